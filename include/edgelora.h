@@ -1,0 +1,177 @@
+/*
+ * edgelora.h -- C ABI of the B200 (sm_100a) batch LoRA inference library.
+ *
+ * One operation sits behind this boundary: a LoRA-augmented linear layer over a
+ * mixed batch of T tokens in which every token names its own adapter,
+ *
+ *     y[t] = W x[t] + s_a * B_a (A_a x[t]),   a = adapter_id[t],   a = -1 => y[t] = W x[t]
+ *
+ * (paper Section 3.4 "Batch LoRA Inference", the displayed batch equation; adapter shapes
+ * A: r x h_in, B: h_out x r from Section 2.1).  Adapters live in a pool of fixed-size
+ * blocks reserved once (Section 3.3 "pre-allocated memory pool", Section 4.2); a token's
+ * adapter id is the index of the block ("slot") that holds its adapter.
+ *
+ * Conventions
+ *   - All matrices are row-major bfloat16 (uint16 bit patterns).  Accumulation is fp32,
+ *     outputs are rounded to nearest-even bfloat16.  Ids are int32.
+ *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers are
+ *     ordinary host memory.  The caller owns W, x, ids and y; the pool owns the slot
+ *     memory (unless the caller lends an arena), its staging buffers, workspaces, side
+ *     stream and events.
+ *   - Every function returns an int: EDGELORA_OK (0) or a negative edgelora_status.
+ *     Nothing throws or aborts across this boundary.  There is no CPU fallback: without
+ *     a CUDA device every compute entry point returns EDGELORA_ERR_CUDA.
+ *   - Conditions only the GPU can see (an id outside [-1, n_slots), an id that names an
+ *     empty slot) never trap: that token is computed base-only, a bit is set in a device
+ *     status word, and edgelora_pool_sync_status() reports it.
+ *   - Shape limits: h_in % 8 == 0, h_out % 8 == 0, 1 <= max_rank <= 64 (rounded up to a
+ *     multiple of 16 internally), n_slots <= 65534, T <= max_tokens <= 32768.
+ */
+#ifndef EDGELORA_H_
+#define EDGELORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  EDGELORA_OK = 0,
+  EDGELORA_ERR_INVALID_ARG = -1,
+  EDGELORA_ERR_BAD_SLOT = -2,
+  EDGELORA_ERR_RANK_TOO_LARGE = -3,
+  EDGELORA_ERR_ARENA_TOO_SMALL = -4,
+  EDGELORA_ERR_CUDA = -5,
+  EDGELORA_ERR_BAD_ADAPTER_ID = -6,
+  EDGELORA_ERR_SLOT_EMPTY = -7,
+  EDGELORA_ERR_TIMEOUT = -8,
+  EDGELORA_ERR_TOO_MANY_TOKENS = -9
+} edgelora_status;
+
+/* Bits of the device status word returned by edgelora_pool_sync_status(). */
+#define EDGELORA_STATUS_BAD_ADAPTER_ID 0x1u /* an id outside [-1, n_slots) was seen     */
+#define EDGELORA_STATUS_SLOT_EMPTY 0x2u     /* an id named a slot with nothing loaded   */
+#define EDGELORA_STATUS_TIMEOUT 0x4u        /* a bounded in-kernel wait gave up         */
+
+typedef struct edgelora_pool edgelora_pool_t; /* opaque, owned by the library */
+typedef struct edgelora_plan edgelora_plan_t; /* opaque, owned by the library */
+
+/* Pool geometry for ONE linear site (one W shape).  Section 3.3: the pool is a set of
+ * fixed blocks, each the size of one adapter; here a block holds A padded to
+ * [max_rank][h_in] and B padded to [h_out][max_rank]. */
+typedef struct {
+  int32_t h_in;       /* input width of the linear site                                  */
+  int32_t h_out;      /* output width                                                    */
+  int32_t n_slots;    /* number of blocks S                                              */
+  int32_t max_rank;   /* largest adapter rank a block can hold                           */
+  int32_t max_tokens; /* largest T of a call; 0 => 8192.  Sizes the workspaces.          */
+  uint32_t flags;     /* EDGELORA_FLAG_*                                                 */
+  void *arena_dev;    /* optional caller-owned device memory for the slot blocks, 256-byte
+                         aligned; NULL => the library allocates and owns it              */
+  size_t arena_bytes; /* size of arena_dev; ignored when arena_dev is NULL               */
+} edgelora_pool_config;
+
+#define EDGELORA_FLAG_NONE 0u
+
+/* Options for edgelora_pool_set_option(). */
+#define EDGELORA_OPT_REGIME 1    /* 0 auto (T <= 256 => decode), 1 force decode, 2 force prefill */
+#define EDGELORA_OPT_PROFILE 2   /* 1 => bracket every kernel with CUDA events (slower)          */
+#define EDGELORA_OPT_PDL 3       /* 1 (default) => programmatic dependent launch between kernels  */
+
+/* Bytes of device memory the slot blocks need for this geometry (what arena_bytes must
+ * be at least).  Host-only arithmetic. */
+int edgelora_pool_bytes_required(const edgelora_pool_config *cfg, size_t *bytes_out);
+
+/* Section 3.3 / 4.2: reserve every block once, at initialisation.  Allocates the slot
+ * blocks (unless an arena is lent), the slot table, pinned staging buffers, a side
+ * stream, events and the per-call workspaces.  All slots start empty. */
+int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool_out);
+
+/* Section 3.3: "when a new adapter is required it is assigned to a free block".
+ * Copies adapter (A_host [rank][h_in], B_host [h_out][rank], dense bf16) into block
+ * `slot`, asynchronously: the data is first copied into pinned staging (so the caller may
+ * free A_host / B_host on return), then moved with cudaMemcpyAsync on the pool's side
+ * stream.  The copy waits for the last edgelora_lora_linear call issued before it, and
+ * later edgelora_lora_linear calls wait for the copy, so a call never sees a half-written
+ * block; the caller must not reload a slot that ids of a still-queued call refer to.
+ * rank must be in [1, max_rank]; scale is s_a. */
+int edgelora_pool_load_slot(edgelora_pool_t *pool, int32_t slot, int32_t rank, float scale,
+                            const uint16_t *A_host, const uint16_t *B_host);
+
+/* Section 4.2: an evicted adapter's block returns to the pool.  Marks `slot` empty
+ * (asynchronously, ordered like a load). */
+int edgelora_pool_evict_slot(edgelora_pool_t *pool, int32_t slot);
+
+/* Blocks the host until every load / evict issued so far has landed in device memory. */
+int edgelora_pool_wait_loads(edgelora_pool_t *pool);
+
+/* Section 3.4: the batched layer.  W_dev [h_out][h_in], x_dev [T][h_in],
+ * adapter_id_dev [T] (slot index or -1), y_dev [T][h_out]; all device memory, 16-byte
+ * aligned.  Enqueues, on `stream` (a cudaStream_t; NULL = legacy default stream):
+ * routing plan -> shrink (z = s_a A_a x) -> base product W x on the tensor cores ->
+ * expand + combine, y written once.  Asynchronous; no host synchronisation, no
+ * allocation.  T == 0 is a no-op.  x_dev / y_dev must not alias. */
+int edgelora_lora_linear(edgelora_pool_t *pool, const void *W_dev, const void *x_dev,
+                         const int32_t *adapter_id_dev, int32_t T, void *y_dev, void *stream);
+
+/* Same layer with HOST buffers: copies x and ids to the device through pinned staging,
+ * runs the layer, copies y back and synchronises `stream` before returning.  W stays a
+ * device pointer (weights are resident model state, like the pool). */
+int edgelora_lora_linear_host(edgelora_pool_t *pool, const void *W_dev, const uint16_t *x_host,
+                              const int32_t *adapter_id_host, int32_t T, uint16_t *y_host,
+                              void *stream);
+
+/* Routing plan (Section 3.4 "u-batch" grouping; Section 4.3 "maps adapter IDs to sample
+ * indices ... scattered back to their original positions").  A plan depends only on the
+ * ids, so one plan can serve every linear site that sees the same batch. */
+int edgelora_plan_create(int32_t max_tokens, int32_t n_slots, edgelora_plan_t **plan_out);
+int edgelora_plan_destroy(edgelora_plan_t *plan);
+/* Builds the plan for adapter_id_dev[T] on `stream` (asynchronous). */
+int edgelora_plan_build(edgelora_plan_t *plan, const int32_t *adapter_id_dev, int32_t T,
+                        void *stream);
+/* Copies the last built plan to host arrays (synchronises `stream`).  Any array may be
+ * NULL.  Sizes: ids_valid[T], perm[T], group_start[T+1], group_adapter[T],
+ * seg_start[T+1], seg_adapter[T]; counts_out = {n_groups, n_segments}.
+ *   segments: maximal runs of equal id in token order;
+ *   groups  : ids ascending with -1 first, token order kept inside a group. */
+int edgelora_plan_export(edgelora_plan_t *plan, void *stream, int32_t *ids_valid,
+                         int32_t *perm, int32_t *group_start, int32_t *group_adapter,
+                         int32_t *seg_start, int32_t *seg_adapter, int32_t counts_out[2]);
+/* The layer with a plan built beforehand by edgelora_plan_build on the same stream for
+ * the same ids (plan.n_slots must equal the pool's). */
+int edgelora_lora_linear_planned(edgelora_pool_t *pool, edgelora_plan_t *plan, const void *W_dev,
+                                 const void *x_dev, int32_t T, void *y_dev, void *stream);
+/* The pool's own plan object (the one edgelora_lora_linear builds each call). */
+int edgelora_pool_plan(edgelora_pool_t *pool, edgelora_plan_t **plan_out);
+
+/* Synchronises the device work issued through this pool, returns the status bits
+ * accumulated since the last call in *bits_out and clears them.  The return value is
+ * EDGELORA_OK, or the error matching the most severe bit. */
+int edgelora_pool_sync_status(edgelora_pool_t *pool, uint32_t *bits_out);
+
+int edgelora_pool_set_option(edgelora_pool_t *pool, int32_t option, int32_t value);
+
+/* Launch bookkeeping for measurement.  info_out[0] = kernels launched by the last
+ * edgelora_lora_linear call, [1] = regime used (1 decode, 2 prefill), [2] = grid of the
+ * base-product kernel, [3] = split-K factor, [4] = pipeline stages, [5] = N tile,
+ * [6] = total kernels launched through this pool, [7] = reserved. */
+int edgelora_pool_last_launch(edgelora_pool_t *pool, int64_t info_out[8]);
+
+/* With EDGELORA_OPT_PROFILE on: accumulated device time per kernel since the last reset,
+ * from CUDA events on the launching stream (synchronises them).  ms_out / launches_out:
+ * [0] plan, [1] shrink (gather-by-token), [2] shrink (segment), [3] base product,
+ * [4] decode combine.  reset != 0 clears the accumulators afterwards. */
+int edgelora_pool_kernel_times(edgelora_pool_t *pool, double ms_out[5], int64_t launches_out[5],
+                               int32_t reset);
+
+/* Releases everything the pool owns (never the caller's arena).  Synchronises first. */
+int edgelora_pool_destroy(edgelora_pool_t *pool);
+
+const char *edgelora_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EDGELORA_H_ */

@@ -1,0 +1,274 @@
+"""Python binding of the C-ABI library (``include/edgelora.h``): argument marshalling only.
+
+Every function here has the name of the C entry point it calls.  Tensors are torch CUDA tensors
+(used for device memory and streams only); the arithmetic all happens in the CUDA kernels of
+``libedgelora.so``.  There is no CPU path: importing works anywhere, but creating a pool without
+the compiled library or without a CUDA device raises.
+"""
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libedgelora.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_BAD_SLOT, ERR_RANK_TOO_LARGE, ERR_ARENA_TOO_SMALL = -1, -2, -3, -4
+ERR_CUDA, ERR_BAD_ADAPTER_ID, ERR_SLOT_EMPTY, ERR_TIMEOUT, ERR_TOO_MANY_TOKENS = -5, -6, -7, -8, -9
+STATUS_BAD_ADAPTER_ID, STATUS_SLOT_EMPTY, STATUS_TIMEOUT = 0x1, 0x2, 0x4
+OPT_REGIME, OPT_PROFILE, OPT_PDL = 1, 2, 3
+KERNEL_NAMES = ("plan", "shrink_bgmv", "shrink_sgmv", "base_gemm", "decode_combine")
+
+EXPORTS = (
+    "edgelora_pool_bytes_required", "edgelora_pool_create", "edgelora_pool_load_slot",
+    "edgelora_pool_evict_slot", "edgelora_pool_wait_loads", "edgelora_lora_linear",
+    "edgelora_lora_linear_host", "edgelora_plan_create", "edgelora_plan_destroy",
+    "edgelora_plan_build", "edgelora_plan_export", "edgelora_lora_linear_planned",
+    "edgelora_pool_plan", "edgelora_pool_sync_status", "edgelora_pool_set_option",
+    "edgelora_pool_last_launch", "edgelora_pool_kernel_times", "edgelora_pool_destroy",
+    "edgelora_strerror",
+)
+
+
+class EdgeLoraError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+
+
+class PoolConfig(ctypes.Structure):
+    _fields_ = [("h_in", ctypes.c_int32), ("h_out", ctypes.c_int32), ("n_slots", ctypes.c_int32),
+                ("max_rank", ctypes.c_int32), ("max_tokens", ctypes.c_int32),
+                ("flags", ctypes.c_uint32), ("arena_dev", ctypes.c_void_p),
+                ("arena_bytes", ctypes.c_size_t)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libedgelora.so (built in-tree by ``python -m paper_2507_01438_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                           "`python -m paper_2507_01438_b200.build` (needs nvcc); there is no fallback")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, cp = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER
+    L.edgelora_pool_bytes_required.argtypes = [cp(PoolConfig), cp(ctypes.c_size_t)]
+    L.edgelora_pool_create.argtypes = [cp(PoolConfig), cp(vp)]
+    L.edgelora_pool_load_slot.argtypes = [vp, i32, i32, ctypes.c_float, vp, vp]
+    L.edgelora_pool_evict_slot.argtypes = [vp, i32]
+    L.edgelora_pool_wait_loads.argtypes = [vp]
+    L.edgelora_lora_linear.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+    L.edgelora_lora_linear_host.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+    L.edgelora_plan_create.argtypes = [i32, i32, cp(vp)]
+    L.edgelora_plan_destroy.argtypes = [vp]
+    L.edgelora_plan_build.argtypes = [vp, vp, i32, vp]
+    L.edgelora_plan_export.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.edgelora_lora_linear_planned.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+    L.edgelora_pool_plan.argtypes = [vp, cp(vp)]
+    L.edgelora_pool_sync_status.argtypes = [vp, cp(ctypes.c_uint32)]
+    L.edgelora_pool_set_option.argtypes = [vp, i32, i32]
+    L.edgelora_pool_last_launch.argtypes = [vp, vp]
+    L.edgelora_pool_kernel_times.argtypes = [vp, vp, vp, i32]
+    L.edgelora_pool_destroy.argtypes = [vp]
+    L.edgelora_strerror.argtypes = [ctypes.c_int]
+    L.edgelora_strerror.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name != "edgelora_strerror":
+            getattr(L, name).restype = ctypes.c_int
+    _lib = L
+    return L
+
+
+def strerror(code: int) -> str:
+    return lib().edgelora_strerror(code).decode()
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != OK:
+        raise EdgeLoraError(rc, what)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dev_ptr(t, dtype_bytes: int, what: str) -> int:
+    assert t.is_cuda and t.is_contiguous() and t.element_size() == dtype_bytes, what
+    return t.data_ptr()
+
+
+def edgelora_pool_bytes_required(h_in, h_out, n_slots, max_rank) -> int:
+    cfg = PoolConfig(h_in, h_out, n_slots, max_rank, 0, 0, None, 0)
+    out = ctypes.c_size_t(0)
+    _check(lib().edgelora_pool_bytes_required(ctypes.byref(cfg), ctypes.byref(out)), "pool_bytes_required")
+    return out.value
+
+
+def edgelora_pool_create(h_in, h_out, n_slots, max_rank, max_tokens=0, arena=None) -> int:
+    """Returns the opaque pool handle.  ``arena`` may be a torch CUDA tensor lent for the slot blocks."""
+    cfg = PoolConfig(h_in, h_out, n_slots, max_rank, max_tokens, 0,
+                     arena.data_ptr() if arena is not None else None,
+                     arena.numel() * arena.element_size() if arena is not None else 0)
+    out = ctypes.c_void_p()
+    _check(lib().edgelora_pool_create(ctypes.byref(cfg), ctypes.byref(out)), "pool_create")
+    return out.value
+
+
+def edgelora_pool_load_slot(pool, slot: int, rank: int, scale: float, A: np.ndarray, B: np.ndarray) -> None:
+    """A: uint16 [rank, h_in], B: uint16 [h_out, rank] (bf16 bit patterns, host memory)."""
+    A = np.ascontiguousarray(A, dtype=np.uint16)
+    B = np.ascontiguousarray(B, dtype=np.uint16)
+    _check(lib().edgelora_pool_load_slot(pool, slot, rank, scale, A.ctypes.data, B.ctypes.data), "pool_load_slot")
+
+
+def edgelora_pool_evict_slot(pool, slot: int) -> None:
+    _check(lib().edgelora_pool_evict_slot(pool, slot), "pool_evict_slot")
+
+
+def edgelora_pool_wait_loads(pool) -> None:
+    _check(lib().edgelora_pool_wait_loads(pool), "pool_wait_loads")
+
+
+def edgelora_lora_linear(pool, W, x, adapter_id, y, stream=None) -> None:
+    """W [h_out,h_in], x [T,h_in], y [T,h_out]: torch bf16 CUDA tensors; adapter_id: int32 [T]."""
+    T = int(x.shape[0])
+    _check(lib().edgelora_lora_linear(pool, _dev_ptr(W, 2, "W"), _dev_ptr(x, 2, "x") if T else None,
+                                      _dev_ptr(adapter_id, 4, "ids") if T else None, T,
+                                      _dev_ptr(y, 2, "y") if T else None, _stream_ptr(stream)),
+           "lora_linear")
+
+
+def edgelora_lora_linear_planned(pool, plan, W, x, y, stream=None) -> None:
+    T = int(x.shape[0])
+    _check(lib().edgelora_lora_linear_planned(pool, plan, _dev_ptr(W, 2, "W"), _dev_ptr(x, 2, "x"), T,
+                                              _dev_ptr(y, 2, "y"), _stream_ptr(stream)),
+           "lora_linear_planned")
+
+
+def edgelora_lora_linear_host(pool, W, x_host: np.ndarray, ids_host: np.ndarray, y_host: np.ndarray,
+                              stream=None) -> None:
+    """Host buffers in and out (numpy uint16 / int32); W stays a device tensor."""
+    assert x_host.dtype == np.uint16 and ids_host.dtype == np.int32 and y_host.dtype == np.uint16
+    assert x_host.flags.c_contiguous and ids_host.flags.c_contiguous and y_host.flags.c_contiguous
+    T = int(x_host.shape[0])
+    _check(lib().edgelora_lora_linear_host(pool, _dev_ptr(W, 2, "W"), x_host.ctypes.data,
+                                           ids_host.ctypes.data, T, y_host.ctypes.data,
+                                           _stream_ptr(stream)), "lora_linear_host")
+
+
+def edgelora_plan_create(max_tokens: int, n_slots: int) -> int:
+    out = ctypes.c_void_p()
+    _check(lib().edgelora_plan_create(max_tokens, n_slots, ctypes.byref(out)), "plan_create")
+    return out.value
+
+
+def edgelora_plan_destroy(plan) -> None:
+    _check(lib().edgelora_plan_destroy(plan), "plan_destroy")
+
+
+def edgelora_plan_build(plan, adapter_id, stream=None) -> None:
+    T = int(adapter_id.shape[0])
+    _check(lib().edgelora_plan_build(plan, _dev_ptr(adapter_id, 4, "ids") if T else None, T,
+                                     _stream_ptr(stream)), "plan_build")
+
+
+def edgelora_plan_export(plan, T: int, stream=None) -> dict:
+    """Host copies of the last built plan, trimmed to their true lengths."""
+    n = max(T, 1)
+    arr = {k: np.zeros(n + 1, dtype=np.int32) for k in
+           ("ids_valid", "perm", "group_start", "group_adapter", "seg_start", "seg_adapter")}
+    counts = np.zeros(2, dtype=np.int32)
+    _check(lib().edgelora_plan_export(plan, _stream_ptr(stream), arr["ids_valid"].ctypes.data,
+                                      arr["perm"].ctypes.data, arr["group_start"].ctypes.data,
+                                      arr["group_adapter"].ctypes.data, arr["seg_start"].ctypes.data,
+                                      arr["seg_adapter"].ctypes.data, counts.ctypes.data), "plan_export")
+    G, NS = int(counts[0]), int(counts[1])
+    return {"ids_valid": arr["ids_valid"][:T].copy(), "perm": arr["perm"][:T].copy(),
+            "group_start": arr["group_start"][:G + 1].copy(), "group_adapter": arr["group_adapter"][:G].copy(),
+            "seg_start": arr["seg_start"][:NS + 1].copy(), "seg_adapter": arr["seg_adapter"][:NS].copy()}
+
+
+def edgelora_pool_plan(pool) -> int:
+    out = ctypes.c_void_p()
+    _check(lib().edgelora_pool_plan(pool, ctypes.byref(out)), "pool_plan")
+    return out.value
+
+
+def edgelora_pool_sync_status(pool):
+    """Returns (return code, status bits); does not raise on device-detected conditions."""
+    bits = ctypes.c_uint32(0)
+    rc = lib().edgelora_pool_sync_status(pool, ctypes.byref(bits))
+    if rc == ERR_CUDA or rc == ERR_INVALID_ARG:
+        raise EdgeLoraError(rc, "pool_sync_status")
+    return rc, bits.value
+
+
+def edgelora_pool_set_option(pool, option: int, value: int) -> None:
+    _check(lib().edgelora_pool_set_option(pool, option, value), "pool_set_option")
+
+
+def edgelora_pool_last_launch(pool) -> dict:
+    info = np.zeros(8, dtype=np.int64)
+    _check(lib().edgelora_pool_last_launch(pool, info.ctypes.data), "pool_last_launch")
+    return {"launches": int(info[0]), "regime": {1: "decode", 2: "prefill"}.get(int(info[1]), "none"),
+            "gemm_grid": int(info[2]), "split_k": int(info[3]), "stages": int(info[4]),
+            "n_tile": int(info[5]), "total_launches": int(info[6])}
+
+
+def edgelora_pool_kernel_times(pool, reset: bool = True) -> dict:
+    ms = np.zeros(5, dtype=np.float64)
+    n = np.zeros(5, dtype=np.int64)
+    _check(lib().edgelora_pool_kernel_times(pool, ms.ctypes.data, n.ctypes.data, 1 if reset else 0),
+           "pool_kernel_times")
+    return {k: {"ms": float(ms[i]), "launches": int(n[i])} for i, k in enumerate(KERNEL_NAMES)}
+
+
+def edgelora_pool_destroy(pool) -> None:
+    _check(lib().edgelora_pool_destroy(pool), "pool_destroy")
+
+
+class Pool:
+    """Small convenience wrapper: owns a pool handle and loads a workload's adapters."""
+
+    def __init__(self, h_in, h_out, n_slots, max_rank, max_tokens=0, arena=None):
+        self.handle = edgelora_pool_create(h_in, h_out, n_slots, max_rank, max_tokens, arena)
+        self.h_in, self.h_out, self.n_slots, self.max_rank = h_in, h_out, n_slots, max_rank
+        self._arena = arena
+
+    def load(self, slot, A, B, scale):
+        edgelora_pool_load_slot(self.handle, slot, int(A.shape[0]), float(scale), A, B)
+
+    def load_all(self, adapters: dict):
+        for slot, ad in adapters.items():
+            self.load(int(slot), ad.A, ad.B, ad.scale)
+        edgelora_pool_wait_loads(self.handle)
+
+    def linear(self, W, x, ids, y=None, stream=None):
+        import torch
+        if y is None:
+            y = torch.empty((x.shape[0], self.h_out), dtype=torch.bfloat16, device=x.device)
+        edgelora_lora_linear(self.handle, W, x, ids, y, stream)
+        return y
+
+    def status(self):
+        return edgelora_pool_sync_status(self.handle)
+
+    def close(self):
+        if self.handle:
+            edgelora_pool_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

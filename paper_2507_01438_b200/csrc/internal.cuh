@@ -1,0 +1,92 @@
+// Structures shared by the kernels and the host launcher of the batch LoRA library.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/edgelora.h"
+
+namespace edgelora {
+
+constexpr int kTileM = 128;        // UMMA M: rows of the TMEM accumulator (one per lane)
+constexpr int kBlockK = 64;        // bf16 elements per K block = one 128-byte swizzled row
+constexpr int kUmmaK = 16;         // K of one tcgen05.mma for 16-bit inputs
+constexpr int kMaxStages = 12;
+constexpr int kSegMin = 32;        // prefill: runs at least this long go through the segment shrink
+constexpr int kDecodeMaxT = 256;   // decode regime: all tokens are one UMMA N tile
+constexpr int kMaxTokensLimit = 32768;
+constexpr int kGemmThreads = 192;  // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+
+// One row of the slot table (paper Section 3.3: one fixed block per resident adapter).
+struct SlotRow {
+  int32_t rank;        // 0 = empty
+  float scale;         // s_a
+  int32_t generation;  // bumped on every load / evict
+  int32_t pad;
+};
+
+// Device arrays of a routing plan.
+struct PlanView {
+  int32_t *ids_valid;      // [maxT]   id, or -1 where the caller's id was out of range
+  int32_t *perm;           // [maxT]   tokens ordered by (id, token)
+  int32_t *group_start;    // [maxT+1]
+  int32_t *group_adapter;  // [maxT]
+  int32_t *seg_start;      // [maxT+1]
+  int32_t *seg_adapter;    // [maxT]
+  int32_t *tok_seg;        // [maxT]   segment index of each token
+  int32_t *perm_short;     // [maxT]   perm restricted to tokens the gather-by-token shrink handles
+  int32_t *gs_short;       // [maxT+1] group boundaries inside perm_short
+  int32_t *sgmv_tiles;     // [max_sgmv_tiles][4] {first token, tokens, slot, 0}
+  int32_t *scratch;        // [maxT+1]
+  int32_t *counts;         // [8]  0: n_groups, 1: n_segments, 2: n_sgmv_tiles
+  uint32_t *status;        // device status word of the plan
+  int32_t max_sgmv_tiles;
+};
+
+enum GemmMode : int32_t { kModePrefill = 0, kModeDecode = 1, kModeSgmv = 2 };
+
+struct GemmParams {
+  int32_t mode;
+  int32_t T, h_in, h_out;
+  int32_t BN;          // UMMA N = rows of the column-operand tile (multiple of 16, <= 256)
+  int32_t stages;      // TMA pipeline depth
+  int32_t n_acc;       // TMEM accumulator buffers (1 or 2)
+  int32_t tmem_cols;   // power of two >= n_acc * BN, >= 32
+  int32_t kb_total;    // K blocks of 64 covering h_in
+  int32_t kb_per;      // K blocks per split
+  int32_t splits;
+  int32_t n_mtiles;    // prefill: token tiles; decode: W row tiles
+  int32_t n_ntiles;    // prefill: W row tiles of BN
+  int32_t R_pad;       // slot block rank stride
+  int32_t zsplits;     // partial z buffers the consumer sums
+  int32_t max_tokens;  // row stride of the z / plan workspaces
+  const int32_t *ids_valid;
+  const SlotRow *slots;
+  const uint16_t *B_pool;   // [S][h_out][R_pad]
+  const float *zws;         // [zsplits][max_tokens][R_pad]   (read by the prefill epilogue)
+  float *zws_out;           // same buffer, written by the segment shrink
+  uint16_t *y;              // [T][h_out]
+  float *ws;                // decode partials [splits][T][h_out]
+  const int32_t *sgmv_tiles;
+  const int32_t *counts;
+  uint32_t *status;
+};
+
+// kernels (defined in plan.cu, shrink.cu, gemm.cu, combine.cu)
+void launch_plan(const int32_t *ids, int32_t T, int32_t n_slots, const PlanView &pv, bool pdl,
+                 cudaStream_t stream);
+void launch_bgmv_shrink(const uint16_t *x, const uint16_t *A_pool, const SlotRow *slots,
+                        const PlanView &pv, float *zws, int32_t T, int32_t h_in, int32_t R_pad,
+                        int32_t n_slots, int32_t zsplits, int32_t max_tokens, uint32_t *status,
+                        bool pdl, cudaStream_t stream);
+void init_plan_kernel();
+cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
+                        const GemmParams &p, int32_t grid, size_t smem_bytes, bool pdl,
+                        cudaStream_t stream);
+cudaError_t gemm_set_smem_limit(size_t smem_bytes);
+void launch_decode_combine(const float *ws, int32_t splits, const float *zws, int32_t zsplits,
+                           int32_t max_tokens, const uint16_t *B_pool, const SlotRow *slots,
+                           const int32_t *ids_valid, uint16_t *y, int32_t T, int32_t h_out,
+                           int32_t R_pad, bool pdl, cudaStream_t stream);
+
+}  // namespace edgelora

@@ -1,0 +1,823 @@
+// Host side of the C ABI: the adapter pool (slot blocks + slot table in HBM, pinned staging,
+// side-stream loads), the routing-plan objects and the launcher of the batched layer.
+// Paper Section 3.3 / 4.2 (pre-allocated pool of fixed blocks, reuse after eviction) and
+// Section 3.4 / 4.3 (batch LoRA inference).
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "internal.cuh"
+
+using namespace edgelora;
+
+namespace {
+
+constexpr int kStagingBuffers = 4;
+constexpr int kMaxZSplits = 8;
+constexpr int kTmapCache = 32;
+constexpr int kProfEvents = 8192;
+constexpr size_t kSmemBudget = 220 * 1024;
+
+#define CUDA_TRY(expr)                                   \
+  do {                                                   \
+    cudaError_t _e = (expr);                             \
+    if (_e != cudaSuccess) {                             \
+      set_last_cuda_error(_e, #expr);                    \
+      return EDGELORA_ERR_CUDA;                          \
+    }                                                    \
+  } while (0)
+
+thread_local char g_last_error[256] = "";
+void set_last_cuda_error(cudaError_t e, const char *what) {
+  snprintf(g_last_error, sizeof g_last_error, "%s: %s", what, cudaGetErrorString(e));
+  if (getenv("EDGELORA_LOG")) fprintf(stderr, "[edgelora] CUDA error: %s\n", g_last_error);
+}
+
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+inline int pad_rank(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : 64); }
+
+// ---- cuTensorMapEncodeTiled through the runtime's driver entry point (no link to libcuda) ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+struct TmapKey {
+  const void *base;
+  uint64_t d0, d1, d2;
+  uint32_t b1;
+  bool operator==(const TmapKey &o) const {
+    return base == o.base && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && b1 == o.b1;
+  }
+};
+struct TmapEntry {
+  TmapKey key;
+  CUtensorMap map;
+};
+
+// bf16 row-major [d2][d1][d0] (d2 == 0 => 2D), box = {64, box_rows, 1}, 128-byte swizzle,
+// out-of-range elements read as zero.
+int encode_tmap(CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1, uint64_t d2,
+                uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return EDGELORA_ERR_CUDA;
+  const cuuint32_t rank = d2 ? 3 : 2;
+  cuuint64_t dims[3] = {d0, d1, d2 ? d2 : 1};
+  cuuint64_t strides[2] = {d0 * 2, d0 * d1 * 2};
+  cuuint32_t box[3] = {static_cast<cuuint32_t>(kBlockK), box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), dims,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(g_last_error, sizeof g_last_error, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+    return EDGELORA_ERR_CUDA;
+  }
+  return EDGELORA_OK;
+}
+
+struct StagingBuf {
+  uint8_t *host = nullptr;  // pinned: [A padded][B padded][SlotRow]
+  cudaEvent_t done = nullptr;
+  bool in_flight = false;
+};
+
+struct ProfRec {
+  int kernel;
+  cudaEvent_t start, stop;
+};
+
+}  // namespace
+
+struct edgelora_plan {
+  int32_t max_tokens = 0, n_slots = 0, last_T = 0;
+  void *block = nullptr;
+  PlanView pv{};
+};
+
+struct edgelora_pool {
+  edgelora_pool_config cfg{};
+  int R_pad = 0, device = 0, sms = 0;
+  bool owns_arena = false;
+  uint8_t *arena = nullptr;
+  uint16_t *A_pool = nullptr, *B_pool = nullptr;
+  size_t a_block = 0, b_block = 0;  // elements per slot
+  SlotRow *slots_dev = nullptr;
+  std::vector<SlotRow> slots_host;
+  StagingBuf staging[kStagingBuffers];
+  int next_staging = 0;
+  cudaStream_t side = nullptr;
+  cudaEvent_t load_ev = nullptr, use_ev = nullptr;
+  uint64_t load_seq = 0, load_seq_waited = 0;
+  bool use_recorded = false;
+  edgelora_plan *plan = nullptr;
+  float *zws = nullptr, *ws = nullptr;
+  size_t ws_floats = 0;
+  uint32_t *status_dev = nullptr;
+  std::vector<TmapEntry> tmaps;
+  size_t tmap_next = 0;
+  int opt_regime = 0, opt_profile = 0, opt_pdl = 1;
+  int64_t last_info[8] = {0};
+  int64_t total_launches = 0;
+  // profiling
+  std::vector<ProfRec> prof;
+  size_t prof_used = 0;
+  double prof_ms[5] = {0};
+  int64_t prof_n[5] = {0};
+  // host-buffer entry point
+  uint16_t *hx = nullptr, *hy = nullptr, *dx = nullptr, *dy = nullptr;
+  int32_t *hids = nullptr, *dids = nullptr;
+};
+
+namespace {
+
+int get_tmap(edgelora_pool *p, const CUtensorMap **out, const void *base, uint64_t d0, uint64_t d1,
+             uint64_t d2, uint32_t box_rows) {
+  TmapKey key{base, d0, d1, d2, box_rows};
+  for (auto &e : p->tmaps)
+    if (e.key == key) {
+      *out = &e.map;
+      return EDGELORA_OK;
+    }
+  TmapEntry e;
+  e.key = key;
+  int rc = encode_tmap(&e.map, base, d0, d1, d2, box_rows);
+  if (rc != EDGELORA_OK) return rc;
+  if (p->tmaps.size() < static_cast<size_t>(kTmapCache)) {
+    p->tmaps.push_back(e);
+    *out = &p->tmaps.back().map;
+  } else {
+    p->tmaps[p->tmap_next] = e;
+    *out = &p->tmaps[p->tmap_next].map;
+    p->tmap_next = (p->tmap_next + 1) % kTmapCache;
+  }
+  return EDGELORA_OK;
+}
+
+bool stream_capturing(cudaStream_t s) {
+  cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &st) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  return st != cudaStreamCaptureStatusNone;
+}
+
+struct ProfScope {
+  edgelora_pool *p;
+  cudaStream_t s;
+  ProfRec *rec = nullptr;
+  ProfScope(edgelora_pool *pool, int kernel, cudaStream_t stream) : p(pool), s(stream) {
+    if (p->opt_profile && p->prof_used < p->prof.size() && !stream_capturing(s)) {
+      rec = &p->prof[p->prof_used++];
+      rec->kernel = kernel;
+      cudaEventRecord(rec->start, s);
+    }
+  }
+  ~ProfScope() {
+    if (rec) cudaEventRecord(rec->stop, s);
+  }
+};
+
+int check_cfg(const edgelora_pool_config *c) {
+  if (!c) return EDGELORA_ERR_INVALID_ARG;
+  if (c->h_in < 8 || c->h_out < 8 || (c->h_in % 8) || (c->h_out % 8)) return EDGELORA_ERR_INVALID_ARG;
+  if (c->n_slots < 1 || c->n_slots > 65534) return EDGELORA_ERR_INVALID_ARG;
+  if (c->max_rank < 1) return EDGELORA_ERR_INVALID_ARG;
+  if (c->max_rank > 64) return EDGELORA_ERR_RANK_TOO_LARGE;
+  if (c->max_tokens < 0 || c->max_tokens > kMaxTokensLimit) return EDGELORA_ERR_TOO_MANY_TOKENS;
+  return EDGELORA_OK;
+}
+
+size_t arena_bytes_for(const edgelora_pool_config *c) {
+  const size_t R = pad_rank(c->max_rank);
+  const size_t per_slot = 2 * R * (static_cast<size_t>(c->h_in) + c->h_out);
+  return per_slot * c->n_slots;
+}
+
+int plan_alloc(edgelora_plan *pl) {
+  const size_t mt = pl->max_tokens;
+  const int max_tiles = pl->max_tokens / kSegMin + 8;
+  // ids_valid, perm, group_adapter, seg_adapter, tok_seg, perm_short: mt each;
+  // group_start, seg_start, gs_short, scratch: mt + 1 each; tiles; counts; status
+  const size_t ints = 6 * mt + 4 * (mt + 1) + 4 * static_cast<size_t>(max_tiles) + 8 + 4;
+  CUDA_TRY(cudaMalloc(&pl->block, ints * 4));
+  CUDA_TRY(cudaMemset(pl->block, 0, ints * 4));
+  int32_t *q = static_cast<int32_t *>(pl->block);
+  PlanView &v = pl->pv;
+  v.ids_valid = q; q += mt;
+  v.perm = q; q += mt;
+  v.group_adapter = q; q += mt;
+  v.seg_adapter = q; q += mt;
+  v.tok_seg = q; q += mt;
+  v.perm_short = q; q += mt;
+  v.group_start = q; q += mt + 1;
+  v.seg_start = q; q += mt + 1;
+  v.gs_short = q; q += mt + 1;
+  v.scratch = q; q += mt + 1;
+  v.sgmv_tiles = q; q += 4 * static_cast<size_t>(max_tiles);
+  v.counts = q; q += 8;
+  v.status = reinterpret_cast<uint32_t *>(q);
+  v.max_sgmv_tiles = max_tiles;
+  return EDGELORA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *edgelora_strerror(int code) {
+  switch (code) {
+    case EDGELORA_OK: return "ok";
+    case EDGELORA_ERR_INVALID_ARG: return "invalid argument";
+    case EDGELORA_ERR_BAD_SLOT: return "slot index out of range";
+    case EDGELORA_ERR_RANK_TOO_LARGE: return "adapter rank exceeds the pool's max_rank (or 64)";
+    case EDGELORA_ERR_ARENA_TOO_SMALL: return "caller arena smaller than edgelora_pool_bytes_required";
+    case EDGELORA_ERR_CUDA: return g_last_error[0] ? g_last_error : "CUDA error";
+    case EDGELORA_ERR_BAD_ADAPTER_ID: return "an adapter id outside [-1, n_slots) was seen (token computed base-only)";
+    case EDGELORA_ERR_SLOT_EMPTY: return "an adapter id named an empty slot (token computed base-only)";
+    case EDGELORA_ERR_TIMEOUT: return "a bounded in-kernel wait gave up";
+    case EDGELORA_ERR_TOO_MANY_TOKENS: return "T exceeds max_tokens (or max_tokens exceeds 32768)";
+    default: return "unknown error";
+  }
+}
+
+int edgelora_pool_bytes_required(const edgelora_pool_config *cfg, size_t *bytes_out) {
+  int rc = check_cfg(cfg);
+  if (rc != EDGELORA_OK) return rc;
+  if (!bytes_out) return EDGELORA_ERR_INVALID_ARG;
+  *bytes_out = arena_bytes_for(cfg);
+  return EDGELORA_OK;
+}
+
+int edgelora_plan_create(int32_t max_tokens, int32_t n_slots, edgelora_plan_t **plan_out) {
+  if (!plan_out || n_slots < 1 || n_slots > 65534) return EDGELORA_ERR_INVALID_ARG;
+  if (max_tokens == 0) max_tokens = 8192;
+  if (max_tokens < 0 || max_tokens > kMaxTokensLimit) return EDGELORA_ERR_TOO_MANY_TOKENS;
+  edgelora_plan *pl = new (std::nothrow) edgelora_plan();
+  if (!pl) return EDGELORA_ERR_INVALID_ARG;
+  pl->max_tokens = max_tokens;
+  pl->n_slots = n_slots;
+  int rc = plan_alloc(pl);
+  if (rc != EDGELORA_OK) {
+    if (pl->block) cudaFree(pl->block);
+    delete pl;
+    return rc;
+  }
+  init_plan_kernel();
+  *plan_out = pl;
+  return EDGELORA_OK;
+}
+
+int edgelora_plan_destroy(edgelora_plan_t *plan) {
+  if (!plan) return EDGELORA_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  if (plan->block) cudaFree(plan->block);
+  delete plan;
+  return EDGELORA_OK;
+}
+
+int edgelora_plan_build(edgelora_plan_t *plan, const int32_t *ids_dev, int32_t T, void *stream) {
+  if (!plan || T < 0 || (T > 0 && !ids_dev)) return EDGELORA_ERR_INVALID_ARG;
+  if (T > plan->max_tokens) return EDGELORA_ERR_TOO_MANY_TOKENS;
+  plan->last_T = T;
+  if (T == 0) return EDGELORA_OK;
+  launch_plan(ids_dev, T, plan->n_slots, plan->pv, false, static_cast<cudaStream_t>(stream));
+  CUDA_TRY(cudaGetLastError());
+  return EDGELORA_OK;
+}
+
+int edgelora_plan_export(edgelora_plan_t *plan, void *stream, int32_t *ids_valid, int32_t *perm,
+                         int32_t *group_start, int32_t *group_adapter, int32_t *seg_start,
+                         int32_t *seg_adapter, int32_t counts_out[2]) {
+  if (!plan) return EDGELORA_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  CUDA_TRY(cudaStreamSynchronize(s));
+  const int T = plan->last_T;
+  int32_t counts[8] = {0};
+  if (T > 0) CUDA_TRY(cudaMemcpy(counts, plan->pv.counts, sizeof counts, cudaMemcpyDeviceToHost));
+  const int G = counts[0], NS = counts[1];
+  auto get = [&](int32_t *dst, const int32_t *src, int n) -> cudaError_t {
+    if (!dst || n <= 0) return cudaSuccess;
+    return cudaMemcpy(dst, src, static_cast<size_t>(n) * 4, cudaMemcpyDeviceToHost);
+  };
+  CUDA_TRY(get(ids_valid, plan->pv.ids_valid, T));
+  CUDA_TRY(get(perm, plan->pv.perm, T));
+  CUDA_TRY(get(group_adapter, plan->pv.group_adapter, G));
+  CUDA_TRY(get(seg_adapter, plan->pv.seg_adapter, NS));
+  if (T > 0) {
+    CUDA_TRY(get(group_start, plan->pv.group_start, G + 1));
+    CUDA_TRY(get(seg_start, plan->pv.seg_start, NS + 1));
+  } else {
+    if (group_start) group_start[0] = 0;
+    if (seg_start) seg_start[0] = 0;
+  }
+  if (counts_out) {
+    counts_out[0] = G;
+    counts_out[1] = NS;
+  }
+  return EDGELORA_OK;
+}
+
+int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool_out) {
+  int rc = check_cfg(cfg);
+  if (rc != EDGELORA_OK) return rc;
+  if (!pool_out) return EDGELORA_ERR_INVALID_ARG;
+  const size_t need = arena_bytes_for(cfg);
+  if (cfg->arena_dev) {
+    if (cfg->arena_bytes < need) return EDGELORA_ERR_ARENA_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(cfg->arena_dev) % 256) return EDGELORA_ERR_INVALID_ARG;
+  }
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) {
+    snprintf(g_last_error, sizeof g_last_error, "device is sm_%d%d; this library is built for sm_100a only",
+             prop.major, prop.minor);
+    return EDGELORA_ERR_CUDA;
+  }
+  if (!get_encode_fn()) {
+    snprintf(g_last_error, sizeof g_last_error, "cuTensorMapEncodeTiled not available from the driver");
+    return EDGELORA_ERR_CUDA;
+  }
+
+  edgelora_pool *p = new (std::nothrow) edgelora_pool();
+  if (!p) return EDGELORA_ERR_INVALID_ARG;
+  p->cfg = *cfg;
+  if (p->cfg.max_tokens == 0) p->cfg.max_tokens = 8192;
+  p->R_pad = pad_rank(cfg->max_rank);
+  p->device = dev;
+  p->sms = prop.multiProcessorCount;
+  p->a_block = static_cast<size_t>(p->R_pad) * cfg->h_in;
+  p->b_block = static_cast<size_t>(cfg->h_out) * p->R_pad;
+  p->slots_host.assign(cfg->n_slots, SlotRow{0, 0.f, 0, 0});
+  p->tmaps.reserve(kTmapCache);
+
+#define POOL_TRY(expr)                         \
+  do {                                         \
+    cudaError_t _e = (expr);                   \
+    if (_e != cudaSuccess) {                   \
+      set_last_cuda_error(_e, #expr);          \
+      edgelora_pool_destroy(p);                \
+      return EDGELORA_ERR_CUDA;                \
+    }                                          \
+  } while (0)
+
+  if (cfg->arena_dev) {
+    p->arena = static_cast<uint8_t *>(cfg->arena_dev);
+  } else {
+    POOL_TRY(cudaMalloc(&p->arena, need));
+    p->owns_arena = true;
+  }
+  p->A_pool = reinterpret_cast<uint16_t *>(p->arena);
+  p->B_pool = p->A_pool + p->a_block * cfg->n_slots;
+  POOL_TRY(cudaMalloc(&p->slots_dev, sizeof(SlotRow) * cfg->n_slots));
+  POOL_TRY(cudaMemset(p->slots_dev, 0, sizeof(SlotRow) * cfg->n_slots));
+  POOL_TRY(cudaMalloc(&p->status_dev, 16));
+  POOL_TRY(cudaMemset(p->status_dev, 0, 16));
+  const size_t stage_bytes = (p->a_block + p->b_block) * 2 + sizeof(SlotRow);
+  for (auto &sb : p->staging) {
+    POOL_TRY(cudaMallocHost(&sb.host, stage_bytes));
+    POOL_TRY(cudaEventCreateWithFlags(&sb.done, cudaEventDisableTiming));
+  }
+  POOL_TRY(cudaStreamCreateWithFlags(&p->side, cudaStreamNonBlocking));
+  POOL_TRY(cudaEventCreateWithFlags(&p->load_ev, cudaEventDisableTiming));
+  POOL_TRY(cudaEventCreateWithFlags(&p->use_ev, cudaEventDisableTiming));
+  POOL_TRY(cudaMalloc(&p->zws, sizeof(float) * kMaxZSplits * static_cast<size_t>(p->cfg.max_tokens) * p->R_pad));
+  // decode partials: splits * T * h_out with splits <= sms / row_tiles + 1 and T <= 256
+  {
+    const int row_tiles = (cfg->h_out + kTileM - 1) / kTileM;
+    const int max_splits = std::max(1, p->sms / row_tiles) + 1;
+    p->ws_floats = static_cast<size_t>(max_splits) * kDecodeMaxT * cfg->h_out;
+    POOL_TRY(cudaMalloc(&p->ws, p->ws_floats * sizeof(float)));
+  }
+  POOL_TRY(gemm_set_smem_limit(kSmemBudget));
+  rc = edgelora_plan_create(p->cfg.max_tokens, cfg->n_slots, &p->plan);
+  if (rc != EDGELORA_OK) {
+    edgelora_pool_destroy(p);
+    return rc;
+  }
+#undef POOL_TRY
+  *pool_out = p;
+  return EDGELORA_OK;
+}
+
+int edgelora_pool_destroy(edgelora_pool_t *p) {
+  if (!p) return EDGELORA_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  if (p->plan) edgelora_plan_destroy(p->plan);
+  if (p->owns_arena && p->arena) cudaFree(p->arena);
+  if (p->slots_dev) cudaFree(p->slots_dev);
+  if (p->status_dev) cudaFree(p->status_dev);
+  for (auto &sb : p->staging) {
+    if (sb.host) cudaFreeHost(sb.host);
+    if (sb.done) cudaEventDestroy(sb.done);
+  }
+  if (p->side) cudaStreamDestroy(p->side);
+  if (p->load_ev) cudaEventDestroy(p->load_ev);
+  if (p->use_ev) cudaEventDestroy(p->use_ev);
+  if (p->zws) cudaFree(p->zws);
+  if (p->ws) cudaFree(p->ws);
+  for (auto &r : p->prof) {
+    cudaEventDestroy(r.start);
+    cudaEventDestroy(r.stop);
+  }
+  if (p->hx) cudaFreeHost(p->hx);
+  if (p->hy) cudaFreeHost(p->hy);
+  if (p->hids) cudaFreeHost(p->hids);
+  if (p->dx) cudaFree(p->dx);
+  if (p->dy) cudaFree(p->dy);
+  if (p->dids) cudaFree(p->dids);
+  cudaGetLastError();
+  delete p;
+  return EDGELORA_OK;
+}
+
+static int stage_and_copy(edgelora_pool *p, int32_t slot, int32_t rank, float scale,
+                          const uint16_t *A_host, const uint16_t *B_host) {
+  StagingBuf &sb = p->staging[p->next_staging];
+  p->next_staging = (p->next_staging + 1) % kStagingBuffers;
+  if (sb.in_flight) {
+    CUDA_TRY(cudaEventSynchronize(sb.done));
+    sb.in_flight = false;
+  }
+  const int h_in = p->cfg.h_in, h_out = p->cfg.h_out, R = p->R_pad;
+  uint16_t *sa = reinterpret_cast<uint16_t *>(sb.host);
+  uint16_t *sbp = sa + p->a_block;
+  SlotRow *srow = reinterpret_cast<SlotRow *>(sbp + p->b_block);
+  SlotRow &mirror = p->slots_host[slot];
+  mirror.rank = rank;
+  mirror.scale = scale;
+  mirror.generation += 1;
+  *srow = mirror;
+  // order against the last layer call that may still read this pool
+  if (p->use_recorded) CUDA_TRY(cudaStreamWaitEvent(p->side, p->use_ev, 0));
+  if (rank > 0) {
+    // A: rows [rank, R) are zero; B: columns [rank, R) are zero
+    memcpy(sa, A_host, static_cast<size_t>(rank) * h_in * 2);
+    memset(sa + static_cast<size_t>(rank) * h_in, 0, static_cast<size_t>(R - rank) * h_in * 2);
+    if (rank == R) {
+      memcpy(sbp, B_host, static_cast<size_t>(h_out) * R * 2);
+    } else {
+      for (int j = 0; j < h_out; ++j) {
+        memcpy(sbp + static_cast<size_t>(j) * R, B_host + static_cast<size_t>(j) * rank, rank * 2);
+        memset(sbp + static_cast<size_t>(j) * R + rank, 0, (R - rank) * 2);
+      }
+    }
+    CUDA_TRY(cudaMemcpyAsync(p->A_pool + p->a_block * slot, sa, p->a_block * 2, cudaMemcpyHostToDevice, p->side));
+    CUDA_TRY(cudaMemcpyAsync(p->B_pool + p->b_block * slot, sbp, p->b_block * 2, cudaMemcpyHostToDevice, p->side));
+  }
+  CUDA_TRY(cudaMemcpyAsync(p->slots_dev + slot, srow, sizeof(SlotRow), cudaMemcpyHostToDevice, p->side));
+  CUDA_TRY(cudaEventRecord(sb.done, p->side));
+  sb.in_flight = true;
+  CUDA_TRY(cudaEventRecord(p->load_ev, p->side));
+  p->load_seq += 1;
+  return EDGELORA_OK;
+}
+
+int edgelora_pool_load_slot(edgelora_pool_t *p, int32_t slot, int32_t rank, float scale,
+                            const uint16_t *A_host, const uint16_t *B_host) {
+  if (!p || !A_host || !B_host) return EDGELORA_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= p->cfg.n_slots) return EDGELORA_ERR_BAD_SLOT;
+  if (rank < 1) return EDGELORA_ERR_INVALID_ARG;
+  if (rank > p->cfg.max_rank) return EDGELORA_ERR_RANK_TOO_LARGE;
+  return stage_and_copy(p, slot, rank, scale, A_host, B_host);
+}
+
+int edgelora_pool_evict_slot(edgelora_pool_t *p, int32_t slot) {
+  if (!p) return EDGELORA_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= p->cfg.n_slots) return EDGELORA_ERR_BAD_SLOT;
+  return stage_and_copy(p, slot, 0, 0.f, nullptr, nullptr);
+}
+
+int edgelora_pool_wait_loads(edgelora_pool_t *p) {
+  if (!p) return EDGELORA_ERR_INVALID_ARG;
+  CUDA_TRY(cudaStreamSynchronize(p->side));
+  for (auto &sb : p->staging) sb.in_flight = false;
+  return EDGELORA_OK;
+}
+
+int edgelora_pool_plan(edgelora_pool_t *p, edgelora_plan_t **plan_out) {
+  if (!p || !plan_out) return EDGELORA_ERR_INVALID_ARG;
+  *plan_out = p->plan;
+  return EDGELORA_OK;
+}
+
+int edgelora_pool_set_option(edgelora_pool_t *p, int32_t option, int32_t value) {
+  if (!p) return EDGELORA_ERR_INVALID_ARG;
+  switch (option) {
+    case EDGELORA_OPT_REGIME:
+      if (value < 0 || value > 2) return EDGELORA_ERR_INVALID_ARG;
+      p->opt_regime = value;
+      return EDGELORA_OK;
+    case EDGELORA_OPT_PROFILE:
+      p->opt_profile = value ? 1 : 0;
+      if (p->opt_profile && p->prof.empty()) {
+        p->prof.resize(kProfEvents);
+        for (auto &r : p->prof) {
+          CUDA_TRY(cudaEventCreate(&r.start));
+          CUDA_TRY(cudaEventCreate(&r.stop));
+        }
+      }
+      return EDGELORA_OK;
+    case EDGELORA_OPT_PDL:
+      p->opt_pdl = value ? 1 : 0;
+      return EDGELORA_OK;
+    default:
+      return EDGELORA_ERR_INVALID_ARG;
+  }
+}
+
+int edgelora_pool_last_launch(edgelora_pool_t *p, int64_t info_out[8]) {
+  if (!p || !info_out) return EDGELORA_ERR_INVALID_ARG;
+  memcpy(info_out, p->last_info, sizeof p->last_info);
+  info_out[6] = p->total_launches;
+  return EDGELORA_OK;
+}
+
+int edgelora_pool_kernel_times(edgelora_pool_t *p, double ms_out[5], int64_t launches_out[5],
+                               int32_t reset) {
+  if (!p) return EDGELORA_ERR_INVALID_ARG;
+  for (size_t i = 0; i < p->prof_used; ++i) {
+    ProfRec &r = p->prof[i];
+    CUDA_TRY(cudaEventSynchronize(r.stop));
+    float ms = 0.f;
+    CUDA_TRY(cudaEventElapsedTime(&ms, r.start, r.stop));
+    p->prof_ms[r.kernel] += ms;
+    p->prof_n[r.kernel] += 1;
+  }
+  p->prof_used = 0;
+  for (int k = 0; k < 5; ++k) {
+    if (ms_out) ms_out[k] = p->prof_ms[k];
+    if (launches_out) launches_out[k] = p->prof_n[k];
+    if (reset) {
+      p->prof_ms[k] = 0;
+      p->prof_n[k] = 0;
+    }
+  }
+  return EDGELORA_OK;
+}
+
+int edgelora_pool_sync_status(edgelora_pool_t *p, uint32_t *bits_out) {
+  if (!p) return EDGELORA_ERR_INVALID_ARG;
+  CUDA_TRY(cudaDeviceSynchronize());
+  uint32_t a = 0, b = 0;
+  CUDA_TRY(cudaMemcpy(&a, p->status_dev, 4, cudaMemcpyDeviceToHost));
+  CUDA_TRY(cudaMemcpy(&b, p->plan->pv.status, 4, cudaMemcpyDeviceToHost));
+  CUDA_TRY(cudaMemset(p->status_dev, 0, 4));
+  CUDA_TRY(cudaMemset(p->plan->pv.status, 0, 4));
+  const uint32_t bits = a | b;
+  if (bits_out) *bits_out = bits;
+  if (bits & EDGELORA_STATUS_TIMEOUT) return EDGELORA_ERR_TIMEOUT;
+  if (bits & EDGELORA_STATUS_BAD_ADAPTER_ID) return EDGELORA_ERR_BAD_ADAPTER_ID;
+  if (bits & EDGELORA_STATUS_SLOT_EMPTY) return EDGELORA_ERR_SLOT_EMPTY;
+  return EDGELORA_OK;
+}
+
+// The layer: plan (optional) -> shrink -> base product -> expand/combine.
+static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_dev,
+                            const void *W_dev, const void *x_dev, int32_t T, void *y_dev,
+                            cudaStream_t stream) {
+  if (!p || !plan || T < 0) return EDGELORA_ERR_INVALID_ARG;
+  if (T == 0) return EDGELORA_OK;
+  if (!W_dev || !x_dev || !y_dev) return EDGELORA_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(W_dev) | reinterpret_cast<uintptr_t>(x_dev) |
+       reinterpret_cast<uintptr_t>(y_dev)) & 15)
+    return EDGELORA_ERR_INVALID_ARG;
+  if (T > p->cfg.max_tokens || T > plan->max_tokens) return EDGELORA_ERR_TOO_MANY_TOKENS;
+  if (plan->n_slots != p->cfg.n_slots) return EDGELORA_ERR_INVALID_ARG;
+  const int h_in = p->cfg.h_in, h_out = p->cfg.h_out, R = p->R_pad;
+  const bool capturing = stream_capturing(stream);
+  const bool pdl = p->opt_pdl && !p->opt_profile;
+  const uint16_t *x = static_cast<const uint16_t *>(x_dev);
+  int launches = 0;
+
+  if (p->load_seq != p->load_seq_waited && !capturing) {
+    CUDA_TRY(cudaStreamWaitEvent(stream, p->load_ev, 0));
+    p->load_seq_waited = p->load_seq;
+  }
+
+  if (ids_dev) {
+    ProfScope ps(p, 0, stream);
+    plan->last_T = T;
+    launch_plan(ids_dev, T, plan->n_slots, plan->pv, pdl, stream);
+    CUDA_TRY(cudaGetLastError());
+    ++launches;
+  } else if (plan->last_T != T) {
+    return EDGELORA_ERR_INVALID_ARG;
+  }
+
+  int regime = (T <= kDecodeMaxT) ? 1 : 2;
+  if (p->opt_regime == 2) regime = 2;
+  if (p->opt_regime == 1 && T > kDecodeMaxT) return EDGELORA_ERR_INVALID_ARG;
+  const bool sgmv = T > kDecodeMaxT;
+  const int kb_total = (h_in + kBlockK - 1) / kBlockK;
+
+  // segment-shrink split-K factor (number of partial z buffers the consumers sum)
+  int zsplits = 1;
+  if (sgmv) {
+    const int tiles_est = std::max(1, T / kTileM);
+    zsplits = std::max(1, std::min({kMaxZSplits, p->sms / tiles_est, kb_total / 4}));
+    const int kb_per = (kb_total + zsplits - 1) / zsplits;
+    zsplits = (kb_total + kb_per - 1) / kb_per;
+  }
+
+  {
+    ProfScope ps(p, 1, stream);
+    launch_bgmv_shrink(x, p->A_pool, p->slots_dev, plan->pv, p->zws, T, h_in, R, p->cfg.n_slots,
+                       zsplits, p->cfg.max_tokens, p->status_dev, pdl, stream);
+    CUDA_TRY(cudaGetLastError());
+    ++launches;
+  }
+
+  GemmParams g{};
+  g.T = T;
+  g.h_in = h_in;
+  g.h_out = h_out;
+  g.kb_total = kb_total;
+  g.R_pad = R;
+  g.zsplits = zsplits;
+  g.max_tokens = p->cfg.max_tokens;
+  g.ids_valid = plan->pv.ids_valid;
+  g.slots = p->slots_dev;
+  g.B_pool = p->B_pool;
+  g.zws = p->zws;
+  g.zws_out = p->zws;
+  g.y = static_cast<uint16_t *>(y_dev);
+  g.ws = p->ws;
+  g.sgmv_tiles = plan->pv.sgmv_tiles;
+  g.counts = plan->pv.counts;
+  g.status = p->status_dev;
+
+  auto smem_for = [](int stages, int BN) {
+    return static_cast<size_t>(1024 + stages * (kTileM * kBlockK * 2 + BN * kBlockK * 2) + 512);
+  };
+  auto stages_for = [&](int BN, int kb_per_cta) {
+    int s = static_cast<int>((kSmemBudget - 1536) / (kTileM * kBlockK * 2 + BN * kBlockK * 2));
+    return std::max(1, std::min({s, kMaxStages, std::max(2, kb_per_cta)}));
+  };
+  auto pow2_cols = [](int cols) {
+    int c = 32;
+    while (c < cols) c <<= 1;
+    return c;
+  };
+
+  if (sgmv) {
+    GemmParams s = g;
+    s.mode = kModeSgmv;
+    s.BN = R;
+    s.splits = zsplits;
+    s.kb_per = (kb_total + zsplits - 1) / zsplits;
+    s.stages = stages_for(R, s.kb_per);
+    s.n_acc = 2;
+    s.tmem_cols = pow2_cols(2 * R);
+    const CUtensorMap *mr, *mc;
+    int rc = get_tmap(p, &mr, x, h_in, T, 0, kTileM);
+    if (rc) return rc;
+    rc = get_tmap(p, &mc, p->A_pool, h_in, R, p->cfg.n_slots, R);
+    if (rc) return rc;
+    const int grid = std::max(1, std::min(p->sms, plan->pv.max_sgmv_tiles * zsplits));
+    ProfScope ps(p, 2, stream);
+    CUDA_TRY(launch_gemm(*mr, *mc, s, grid, smem_for(s.stages, R), pdl, stream));
+    ++launches;
+  }
+
+  if (regime == 1) {
+    const int N = round_up(T, 32);
+    const int row_tiles = (h_out + kTileM - 1) / kTileM;
+    int splits = std::max(1, std::min(p->sms / row_tiles, kb_total / 2));
+    int kb_per = (kb_total + splits - 1) / splits;
+    splits = (kb_total + kb_per - 1) / kb_per;
+    if (static_cast<size_t>(splits) * T * h_out > p->ws_floats) return EDGELORA_ERR_INVALID_ARG;
+    g.mode = kModeDecode;
+    g.BN = N;
+    g.splits = splits;
+    g.kb_per = kb_per;
+    g.n_mtiles = row_tiles;
+    g.n_ntiles = 1;
+    g.stages = stages_for(N, kb_per);
+    g.n_acc = 1;
+    g.tmem_cols = pow2_cols(N);
+    const CUtensorMap *mr, *mc;
+    int rc = get_tmap(p, &mr, W_dev, h_in, h_out, 0, kTileM);
+    if (rc) return rc;
+    rc = get_tmap(p, &mc, x, h_in, T, 0, N);
+    if (rc) return rc;
+    const int grid = row_tiles * splits;
+    {
+      ProfScope ps(p, 3, stream);
+      CUDA_TRY(launch_gemm(*mr, *mc, g, grid, smem_for(g.stages, N), pdl, stream));
+      ++launches;
+    }
+    {
+      ProfScope ps(p, 4, stream);
+      launch_decode_combine(p->ws, splits, p->zws, zsplits, p->cfg.max_tokens, p->B_pool,
+                            p->slots_dev, plan->pv.ids_valid, g.y, T, h_out, R, pdl, stream);
+      CUDA_TRY(cudaGetLastError());
+      ++launches;
+    }
+    p->last_info[2] = grid;
+    p->last_info[3] = splits;
+  } else {
+    const int n_mtiles = (T + kTileM - 1) / kTileM;
+    const int tiles256 = n_mtiles * ((h_out + 255) / 256);
+    int BN = (tiles256 >= p->sms || h_out <= 128) ? 256 : 128;
+    BN = std::min(BN, round_up(h_out, 32));
+    g.mode = kModePrefill;
+    g.BN = BN;
+    g.splits = 1;
+    g.kb_per = kb_total;
+    g.n_mtiles = n_mtiles;
+    g.n_ntiles = (h_out + BN - 1) / BN;
+    g.stages = stages_for(BN, kb_total);
+    g.n_acc = 2;
+    g.tmem_cols = pow2_cols(2 * BN);
+    const CUtensorMap *mr, *mc;
+    int rc = get_tmap(p, &mr, x, h_in, T, 0, kTileM);
+    if (rc) return rc;
+    rc = get_tmap(p, &mc, W_dev, h_in, h_out, 0, BN);
+    if (rc) return rc;
+    const int grid = std::min(p->sms, g.n_mtiles * g.n_ntiles);
+    ProfScope ps(p, 3, stream);
+    CUDA_TRY(launch_gemm(*mr, *mc, g, grid, smem_for(g.stages, BN), pdl, stream));
+    ++launches;
+    p->last_info[2] = grid;
+    p->last_info[3] = 1;
+  }
+
+  if (!capturing) {
+    CUDA_TRY(cudaEventRecord(p->use_ev, stream));
+    p->use_recorded = true;
+  }
+  p->last_info[0] = launches;
+  p->last_info[1] = regime;
+  p->last_info[4] = g.stages;
+  p->last_info[5] = g.BN;
+  p->total_launches += launches;
+  return EDGELORA_OK;
+}
+
+int edgelora_lora_linear(edgelora_pool_t *pool, const void *W_dev, const void *x_dev,
+                         const int32_t *adapter_id_dev, int32_t T, void *y_dev, void *stream) {
+  if (!pool) return EDGELORA_ERR_INVALID_ARG;
+  if (T > 0 && !adapter_id_dev) return EDGELORA_ERR_INVALID_ARG;
+  return lora_linear_impl(pool, pool->plan, adapter_id_dev, W_dev, x_dev, T, y_dev,
+                          static_cast<cudaStream_t>(stream));
+}
+
+int edgelora_lora_linear_planned(edgelora_pool_t *pool, edgelora_plan_t *plan, const void *W_dev,
+                                 const void *x_dev, int32_t T, void *y_dev, void *stream) {
+  if (!pool || !plan) return EDGELORA_ERR_INVALID_ARG;
+  return lora_linear_impl(pool, plan, nullptr, W_dev, x_dev, T, y_dev,
+                          static_cast<cudaStream_t>(stream));
+}
+
+int edgelora_lora_linear_host(edgelora_pool_t *p, const void *W_dev, const uint16_t *x_host,
+                              const int32_t *adapter_id_host, int32_t T, uint16_t *y_host,
+                              void *stream) {
+  if (!p || T < 0) return EDGELORA_ERR_INVALID_ARG;
+  if (T == 0) return EDGELORA_OK;
+  if (!x_host || !adapter_id_host || !y_host) return EDGELORA_ERR_INVALID_ARG;
+  if (T > p->cfg.max_tokens) return EDGELORA_ERR_TOO_MANY_TOKENS;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t mt = p->cfg.max_tokens;
+  if (!p->hx) {  // first use: pinned staging and device mirrors for one batch
+    CUDA_TRY(cudaMallocHost(&p->hx, mt * p->cfg.h_in * 2));
+    CUDA_TRY(cudaMallocHost(&p->hy, mt * p->cfg.h_out * 2));
+    CUDA_TRY(cudaMallocHost(&p->hids, mt * 4));
+    CUDA_TRY(cudaMalloc(&p->dx, mt * p->cfg.h_in * 2));
+    CUDA_TRY(cudaMalloc(&p->dy, mt * p->cfg.h_out * 2));
+    CUDA_TRY(cudaMalloc(&p->dids, mt * 4));
+  }
+  const size_t xb = static_cast<size_t>(T) * p->cfg.h_in * 2, yb = static_cast<size_t>(T) * p->cfg.h_out * 2;
+  memcpy(p->hx, x_host, xb);
+  memcpy(p->hids, adapter_id_host, static_cast<size_t>(T) * 4);
+  CUDA_TRY(cudaMemcpyAsync(p->dx, p->hx, xb, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(cudaMemcpyAsync(p->dids, p->hids, static_cast<size_t>(T) * 4, cudaMemcpyHostToDevice, s));
+  int rc = lora_linear_impl(p, p->plan, p->dids, W_dev, p->dx, T, p->dy, s);
+  if (rc != EDGELORA_OK) return rc;
+  CUDA_TRY(cudaMemcpyAsync(p->hy, p->dy, yb, cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaStreamSynchronize(s));
+  memcpy(y_host, p->hy, yb);
+  return EDGELORA_OK;
+}
+
+}  // extern "C"
