@@ -1,0 +1,109 @@
+"""The task's full-size workloads (gate/up prefill, many-tenant down_proj, the 224-site projection set)
+run in the launch configuration the benchmark uses.  The oracle is too slow for every element at
+these sizes, so each check has two parts:
+  - sampled token rows, full width, element by element (rows chosen to cover every run boundary,
+    every base-only class and the most and least popular adapters), and
+  - for ALL tokens, the projection p[t] = sum_j v[j] y[t][j] against the oracle's projection form.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2507_01438_b200 import binding as B
+from paper_2507_01438_b200 import workloads as wl
+from helpers import adapter_set, assert_parity, oracle_of
+from gpu_helpers import from_dev_bf16, make_pool, run_gpu, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def boundary_rows(ids, extra, seed):
+    """First and last token of every run (capped), plus `extra` random tokens."""
+    start, _ = oracle.segments(ids)
+    rows = set()
+    runs = list(zip(start[:-1], start[1:]))
+    if len(runs) > 24:                                  # many short runs: sample the runs too
+        rng = np.random.Generator(np.random.PCG64(seed))
+        runs = [runs[i] for i in rng.choice(len(runs), 24, replace=False)]
+    for a, b in runs:
+        rows.update((int(a), int(b - 1)))
+    rng = np.random.Generator(np.random.PCG64(seed + 1))
+    rows.update(int(t) for t in rng.choice(len(ids), size=min(extra, len(ids)), replace=False))
+    return np.array(sorted(rows))
+
+
+def projection_check(w, y, seed):
+    """Every token: <v, y[t]> against the oracle, v a seeded +-1 vector.
+
+    Allowed error: the sum of h_out independent bf16 roundings of size <= 2^-9 |y| grows like
+    sqrt(h_out); 1e-2 * sqrt(h_out) * rms(y) is > 5x that and far below the change a dropped or
+    misrouted adapter makes (its term is >= 10 % of rms(y) on every output)."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    v = rng.choice(np.array([-1.0, 1.0]), size=w.h_out)
+    p_ref = oracle.lora_projection(w.W, w.x, w.ids, adapter_set(w.n_slots, w.adapters), v)
+    p_gpu = y.astype(np.float64) @ v
+    rms_y = float(np.sqrt(np.mean(y.astype(np.float64) ** 2)))
+    tol = 1e-2 * np.sqrt(w.h_out) * rms_y
+    bad = np.abs(p_gpu - p_ref) > tol
+    assert not bad.any(), f"{w.name}: projection off for tokens {np.where(bad)[0][:10]}, " \
+                          f"worst {np.abs(p_gpu - p_ref).max() / tol:.2f}x tol"
+
+
+def test_gate_up_prefill_full_size():
+    w = wl.gate_up_prefill()
+    assert (w.T, w.h_in, w.h_out) == (4096, 4096, 14336)
+    y = run_gpu(w)
+    rows = boundary_rows(w.ids, 16, 3)
+    assert_parity(y[rows], oracle_of(w, rows), "gate_up_prefill sampled rows")
+    projection_check(w, y, 3)
+
+
+def test_down_proj_many_tenant_full_size():
+    w = wl.down_proj_many_tenant(only_used=False)       # all 1000 slots resident (2.36 GB)
+    assert (w.T, w.h_in, w.h_out, len(w.adapters)) == (256, 14336, 4096, 1000)
+    y = run_gpu(w)
+    # rows: every base-only token class, the most popular adapter's tokens, singletons, random
+    vals, counts = np.unique(w.ids[w.ids >= 0], return_counts=True)
+    rows = set(np.where(w.ids == -1)[0][:4].tolist())
+    rows.update(np.where(w.ids == vals[np.argmax(counts)])[0][:4].tolist())
+    for a in vals[counts == 1][:6]:
+        rows.update(np.where(w.ids == a)[0].tolist())
+    rows.update(boundary_rows(w.ids, 8, 4).tolist()[:24])
+    rows = np.array(sorted(rows))
+    assert_parity(y[rows], oracle_of(w, rows), "down_proj sampled rows")
+    projection_check(w, y, 4)
+
+
+def full_set_sites():
+    """All 7 sites of layers 0, 15 and 31, and one site (rotating) of every other layer."""
+    sites = [(l, s) for l in (0, 15, 31) for s in range(7)]
+    sites += [(l, l % 7) for l in range(32) if l not in (0, 15, 31)]
+    return sites
+
+
+def test_full_projection_set_sampled_sites():
+    import torch
+    batch = wl.full_set_batch()
+    assert batch.ids.shape[0] == 2112
+    rows = boundary_rows(batch.ids, 4, 5)
+    rows = np.array(sorted(set(rows.tolist()[:10] + [63, 64, 1087, 1088, 2111])))
+    ids_dev = torch.from_numpy(batch.ids).cuda()
+    plan = B.edgelora_plan_create(2112, batch.n_slots)
+    xs = {4096: to_dev_bf16(batch.x4096), 14336: to_dev_bf16(batch.x14336)}
+    try:
+        B.edgelora_plan_build(plan, ids_dev)             # one plan reused by every site
+        for (layer, site) in full_set_sites():
+            w = wl.full_set_site(batch, layer, site)
+            pool = make_pool(w, 2112)
+            try:
+                y = torch.empty((w.T, w.h_out), dtype=torch.bfloat16, device="cuda")
+                B.edgelora_lora_linear_planned(pool.handle, plan, to_dev_bf16(w.W), xs[w.h_in], y)
+                assert pool.status() == (0, 0)
+                yh = from_dev_bf16(y)
+                assert_parity(yh[rows], oracle_of(w, rows), w.name)
+                if layer in (0, 31):
+                    projection_check(w, yh, 5 + site)
+            finally:
+                pool.close()
+    finally:
+        B.edgelora_plan_destroy(plan)
