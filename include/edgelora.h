@@ -146,6 +146,34 @@ int edgelora_lora_linear_planned(edgelora_pool_t *pool, edgelora_plan_t *plan, c
 /* The pool's own plan object (the one edgelora_lora_linear builds each call). */
 int edgelora_pool_plan(edgelora_pool_t *pool, edgelora_plan_t **plan_out);
 
+/* No counterpart in the paper: a routing-plan builder for callers that cannot allocate.
+ *
+ * Some hosts of this library may not call cudaMalloc on the path where they need a plan: a
+ * serving loop that has handed all device memory to its own arena at start-up, code running
+ * inside a region where allocation would synchronise the device or is simply forbidden by the
+ * embedding runtime.  For them this entry point builds the same plan as edgelora_plan_build but
+ * keeps the kernel's working arrays in a fixed array that is part of the library image (about
+ * 66 KB on every GPU that loads the library, for the life of the process).  It calls no
+ * cudaMalloc / cudaFree and no allocating library routine; the caller passes every output.
+ *
+ *   adapter_id_dev [T]     ids as for edgelora_lora_linear (device)
+ *   ids_valid_dev, perm_dev, group_adapter_dev, seg_adapter_dev   [T]   int32, device, written
+ *   group_start_dev, seg_start_dev                                [T+1] int32, device, written
+ *   info_dev [4]           {n_groups, n_segments, status bits (EDGELORA_STATUS_*), 0}, device
+ * Array meanings are those of edgelora_plan_export.  Asynchronous on `stream`.
+ *
+ * Limits and rules: T <= EDGELORA_PLAN_STATIC_MAX_TOKENS, otherwise
+ * EDGELORA_ERR_TOO_MANY_TOKENS and nothing is launched.  The first call on each device looks up
+ * the device address of the built-in array (with that device current); make that first call
+ * outside any stream capture.  All calls on a device share the one array, and it keeps what the
+ * last call left in it, so two calls whose kernels may overlap on the GPU (different streams with
+ * no ordering between them) race: order them on one stream or with events. */
+#define EDGELORA_PLAN_STATIC_MAX_TOKENS 4096
+int edgelora_plan_build_static(const int32_t *adapter_id_dev, int32_t T, int32_t n_slots,
+                               int32_t *ids_valid_dev, int32_t *perm_dev, int32_t *group_start_dev,
+                               int32_t *group_adapter_dev, int32_t *seg_start_dev,
+                               int32_t *seg_adapter_dev, int32_t *info_dev, void *stream);
+
 /* Synchronises the device work issued through this pool, returns the status bits
  * accumulated since the last call in *bits_out and clears them.  The return value is
  * EDGELORA_OK, or the error matching the most severe bit. */

@@ -28,7 +28,7 @@ EXPORTS = (
     "edgelora_plan_build", "edgelora_plan_export", "edgelora_lora_linear_planned",
     "edgelora_pool_plan", "edgelora_pool_sync_status", "edgelora_pool_set_option",
     "edgelora_pool_last_launch", "edgelora_pool_kernel_times", "edgelora_pool_destroy",
-    "edgelora_strerror",
+    "edgelora_strerror", "edgelora_plan_build_static",
 )
 
 
@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
     L.edgelora_plan_build.argtypes = [vp, vp, i32, vp]
     L.edgelora_plan_export.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.edgelora_lora_linear_planned.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+    L.edgelora_plan_build_static.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.edgelora_pool_plan.argtypes = [vp, cp(vp)]
     L.edgelora_pool_sync_status.argtypes = [vp, cp(ctypes.c_uint32)]
     L.edgelora_pool_set_option.argtypes = [vp, i32, i32]
@@ -195,6 +196,22 @@ def edgelora_plan_export(plan, T: int, stream=None) -> dict:
     return {"ids_valid": arr["ids_valid"][:T].copy(), "perm": arr["perm"][:T].copy(),
             "group_start": arr["group_start"][:G + 1].copy(), "group_adapter": arr["group_adapter"][:G].copy(),
             "seg_start": arr["seg_start"][:NS + 1].copy(), "seg_adapter": arr["seg_adapter"][:NS].copy()}
+
+
+PLAN_STATIC_MAX_TOKENS = 4096
+
+
+def edgelora_plan_build_static(adapter_id, n_slots: int, ids_valid, perm, group_start, group_adapter,
+                               seg_start, seg_adapter, info, stream=None) -> int:
+    """The plan builder for callers that cannot allocate device memory (see the header): every
+    array is a caller-owned int32 CUDA tensor ([T] or [T+1]; info is [4]).  Returns the C return
+    code instead of raising, so that callers can test the size limit."""
+    T = int(adapter_id.shape[0])
+    ptr = (lambda t: _dev_ptr(t, 4, "int32 array")) if T else (lambda t: None)
+    return lib().edgelora_plan_build_static(ptr(adapter_id), T, n_slots, ptr(ids_valid), ptr(perm),
+                                            ptr(group_start), ptr(group_adapter), ptr(seg_start),
+                                            ptr(seg_adapter), _dev_ptr(info, 4, "info"),
+                                            _stream_ptr(stream))
 
 
 def edgelora_pool_plan(pool) -> int:
