@@ -235,6 +235,10 @@ def main():
         for i in range(args.warmup):
             step(i)
         stream.synchronize()
+        for pool in pools:
+            rc, bits = pool.status()
+            if rc != 0 or bits != 0:
+                raise SystemExit(f"device status after warm-up: rc={rc} bits={bits:#x} ({B.strerror(rc)})")
         if not args.no_graph:
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph, stream=stream):
@@ -327,8 +331,10 @@ def main():
     gemm_us = 1e3 * kt["base_gemm"]["ms"] / max(kt["base_gemm"]["launches"], 1)
     pk = peaks()
     if bound == "hbm":
-        # the base-product kernel must read W once and x once; its fp32 partials are not counted
-        gemm_bytes = 2 * w.h_in * w.h_out + 2 * w.T * w.h_in
+        # the base-product kernel reads W once, x once and each distinct adapter's B once, and
+        # writes y once; its fp32 split-K partials are not counted
+        gemm_bytes = 2 * w.h_in * w.h_out + 2 * w.T * (w.h_in + w.h_out) + \
+            sum(2 * w.adapters[a].rank * w.h_out for a in w.distinct_adapters())
         achieved = gemm_bytes / (gemm_us * 1e-6) / 1e9
         peak = pk["hbm_gbs"]
         roof = {"bound": "hbm", "kernel": "lora_gemm_kernel (decode mode)", "achieved": achieved, "peak": peak,

@@ -78,7 +78,13 @@ typedef struct {
 /* Options for edgelora_pool_set_option(). */
 #define EDGELORA_OPT_REGIME 1    /* 0 auto (T <= 256 => decode), 1 force decode, 2 force prefill */
 #define EDGELORA_OPT_PROFILE 2   /* 1 => bracket every kernel with CUDA events (slower)          */
-#define EDGELORA_OPT_PDL 3       /* 1 (default) => programmatic dependent launch between kernels  */
+#define EDGELORA_OPT_PDL 3       /* programmatic dependent launch: 0 off; 1 (default) between the
+                                    kernels of one call; 2 also lets the first kernel of a call
+                                    start under the tail of earlier work on the stream -- only
+                                    valid when W, x and the ids of a call are not produced by the
+                                    call before it (independent sites / batches)                  */
+#define EDGELORA_OPT_DECODE_SPLITS 4 /* tuning: K splits per W row tile in decode, 0 = automatic  */
+#define EDGELORA_OPT_SHRINK_ITEMS 5  /* tuning: work items the decode shrink aims for, 0 = auto   */
 
 /* Bytes of device memory the slot blocks need for this geometry (what arena_bytes must
  * be at least).  Host-only arithmetic. */
@@ -110,8 +116,9 @@ int edgelora_pool_wait_loads(edgelora_pool_t *pool);
 /* Section 3.4: the batched layer.  W_dev [h_out][h_in], x_dev [T][h_in],
  * adapter_id_dev [T] (slot index or -1), y_dev [T][h_out]; all device memory, 16-byte
  * aligned.  Enqueues, on `stream` (a cudaStream_t; NULL = legacy default stream):
- * routing plan -> shrink (z = s_a A_a x) -> base product W x on the tensor cores ->
- * expand + combine, y written once.  Asynchronous; no host synchronisation, no
+ * routing plan -> shrink (z = s_a A_a x) -> base product W x on the tensor cores with
+ * the expand B_a z accumulated into the same tile (z rounded to bfloat16 for it) -> y written
+ * once.  Asynchronous; no host synchronisation, no
  * allocation.  T == 0 is a no-op.  x_dev / y_dev must not alias. */
 int edgelora_lora_linear(edgelora_pool_t *pool, const void *W_dev, const void *x_dev,
                          const int32_t *adapter_id_dev, int32_t T, void *y_dev, void *stream);
@@ -153,7 +160,7 @@ int edgelora_pool_plan(edgelora_pool_t *pool, edgelora_plan_t **plan_out);
  * inside a region where allocation would synchronise the device or is simply forbidden by the
  * embedding runtime.  For them this entry point builds the same plan as edgelora_plan_build but
  * keeps the kernel's working arrays in a fixed array that is part of the library image (about
- * 66 KB on every GPU that loads the library, for the life of the process).  It calls no
+ * 100 KB on every GPU that loads the library, for the life of the process).  It calls no
  * cudaMalloc / cudaFree and no allocating library routine; the caller passes every output.
  *
  *   adapter_id_dev [T]     ids as for edgelora_lora_linear (device)
@@ -189,8 +196,8 @@ int edgelora_pool_last_launch(edgelora_pool_t *pool, int64_t info_out[8]);
 
 /* With EDGELORA_OPT_PROFILE on: accumulated device time per kernel since the last reset,
  * from CUDA events on the launching stream (synchronises them).  ms_out / launches_out:
- * [0] plan, [1] shrink (gather-by-token), [2] shrink (segment), [3] base product,
- * [4] decode combine.  reset != 0 clears the accumulators afterwards. */
+ * [0] plan, [1] shrink (gather-by-token), [2] shrink (segment), [3] base product
+ * (expand and combine included), [4] unused.  reset != 0 clears the accumulators afterwards. */
 int edgelora_pool_kernel_times(edgelora_pool_t *pool, double ms_out[5], int64_t launches_out[5],
                                int32_t reset);
 

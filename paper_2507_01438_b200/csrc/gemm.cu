@@ -1,22 +1,28 @@
-// tcgen05 / TMEM / TMA bf16 GEMM for the dense contractions of batch LoRA inference
-// (paper Section 3.4: the base product W [x_0 .. x_n] is batched over every token of the batch).
+// tcgen05 / TMEM / TMA bf16 GEMM for batch LoRA inference (paper Section 3.4): the base product
+// W [x_0 .. x_n] batched over every token, with the low-rank expand B_a z folded into the same
+// accumulator so that y is written once.
 //
-// D[128 x BN] (fp32, in tensor memory) = R[128 x K] * C[BN x K]^T, both operands K-major bf16,
-// fetched by TMA into 128-byte-swizzled shared-memory tiles and multiplied by tcgen05.mma issued
-// from one thread.  The same kernel serves three uses, chosen by GemmParams::mode:
+// D[128 x BN] (fp32, in tensor memory) = R[128 x K] * C[BN x K]^T, both operands K-major bf16 in
+// 128-byte-swizzled shared-memory tiles of 64 K elements ("K blocks"), multiplied by tcgen05.mma
+// issued from one thread.  A tile's K blocks are the K blocks of h_in followed by one "LoRA
+// K block" per adapter the tile touches: its operands are B_a (fetched by TMA, zero-filled beyond
+// the rank stride) and the tokens' z rounded to bf16, masked to the tokens of that adapter and
+// written into the operand tile by four builder warps.  Modes (GemmParams::mode):
 //
-//   prefill  R = 128 tokens of x,  C = BN rows of W.  Epilogue: y = bf16(D + B_a z) per token
-//            (expand fused, y written once).  Persistent over tiles, two TMEM accumulators so the
-//            epilogue of one tile overlaps the main loop of the next.
-//   decode   R = 128 rows of W,    C = all tokens (N = T rounded up).  W is streamed once; K is
-//            split across CTAs so every SM pulls from HBM; fp32 partials go to a workspace that
-//            the combine kernel reduces.
+//   prefill  R = 128 tokens of x,  C = BN rows of W;  LoRA blocks: R = masked z, C = B_a rows.
+//            Persistent over tiles, two TMEM accumulators so the epilogue of one tile overlaps the
+//            main loop of the next.  Epilogue: y = bf16(D).
+//   decode   R = 128 rows of W,    C = all tokens (N = T rounded up); LoRA blocks: R = B_a rows,
+//            C = masked z.  W is streamed once; K and the LoRA groups are split across CTAs so
+//            every SM pulls from HBM; fp32 partials go to a workspace and the CTA that arrives
+//            last at a row tile adds them in a fixed order and writes y.
 //   sgmv     R = 128 tokens of one run, C = A_a (N = rank stride): the segment shrink
-//            z = s_a A_a x for long runs, tile list from the plan.
+//            z = s_a A_a x for long runs, tile list from the plan.  No LoRA blocks.
 //
 // Warp roles: warp 0 issues TMA, warp 1 owns TMEM and issues the MMAs, warps 2..5 are the
-// epilogue (each reads the 32 TMEM lanes of its quadrant).  Every mbarrier wait is bounded; on a
-// timeout the status word gets EDGELORA_STATUS_TIMEOUT and all roles leave their loops.
+// epilogue (each reads the 32 TMEM lanes of its quadrant), warps 6..9 build the z operand.
+// Every mbarrier wait is bounded; on a timeout the status word gets EDGELORA_STATUS_TIMEOUT and
+// all roles leave their loops.
 #include "internal.cuh"
 #include "launch.cuh"
 #include "ptx.cuh"
@@ -30,6 +36,7 @@ struct TileCoord {
   int32_t kb0, kb1;
   int32_t split;
   int32_t nrows;   // sgmv: tokens of the tile that belong to the run
+  int32_t mtile;   // prefill: token tile; decode: W row tile
 };
 
 __device__ __forceinline__ int32_t total_tiles(const GemmParams &p) {
@@ -47,11 +54,13 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams &p, int32_t til
     c.row_r = m * kTileM;
     c.row_c = n * p.BN;
     c.split = 0;
+    c.mtile = m;
   } else if (p.mode == kModeDecode) {
     const int m = tile % p.n_mtiles;
     c.split = tile / p.n_mtiles;
     c.row_r = m * kTileM;
     c.row_c = 0;
+    c.mtile = m;
   } else {
     const int n_t = p.counts[2];
     const int st = tile % n_t;
@@ -60,93 +69,49 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams &p, int32_t til
     c.nrows = p.sgmv_tiles[4 * st + 1];
     c.slot = p.sgmv_tiles[4 * st + 2];
     c.row_c = 0;
+    c.mtile = 0;
   }
   c.kb0 = c.split * p.kb_per;
   c.kb1 = min(p.kb_total, c.kb0 + p.kb_per);
   return c;
 }
 
-// ---- epilogues: each thread owns one accumulator row (TMEM lane) and NC consecutive columns ----
-
-// prefill: row = token, columns = output features n0 + c0 + [0, NC)
-template <int NC>
-__device__ __forceinline__ void epilogue_prefill_chunk(const GemmParams &p, float (&acc)[NC],
-                                                       int32_t t, bool valid, int32_t a,
-                                                       int32_t rank, const float (&z)[64],
-                                                       int32_t col0) {
-  if (a >= 0 && rank > 0) {
-    const uint16_t *Bbase = p.B_pool + (static_cast<size_t>(a) * p.h_out) * p.R_pad;
-#pragma unroll
-    for (int jj = 0; jj < NC; ++jj) {
-      const int j = col0 + jj;
-      if (j < p.h_out) {
-        const uint4 *Brow = reinterpret_cast<const uint4 *>(Bbase + static_cast<size_t>(j) * p.R_pad);
-        float s = 0.f;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          if (c * 8 < rank) {
-            const uint4 b = __ldg(Brow + c);
-            s = fmaf(ptx::bf16_lo(b.x), z[c * 8 + 0], s);
-            s = fmaf(ptx::bf16_hi(b.x), z[c * 8 + 1], s);
-            s = fmaf(ptx::bf16_lo(b.y), z[c * 8 + 2], s);
-            s = fmaf(ptx::bf16_hi(b.y), z[c * 8 + 3], s);
-            s = fmaf(ptx::bf16_lo(b.z), z[c * 8 + 4], s);
-            s = fmaf(ptx::bf16_hi(b.z), z[c * 8 + 5], s);
-            s = fmaf(ptx::bf16_lo(b.w), z[c * 8 + 6], s);
-            s = fmaf(ptx::bf16_hi(b.w), z[c * 8 + 7], s);
-          }
-        }
-        acc[jj] += s;
-      }
-    }
+// The LoRA K blocks of a tile: entries [e0, e1) step `de` of `list`.  Entries whose slot is
+// empty are skipped by every role alike (they all read the same slot table).
+struct LoraList {
+  const int32_t *list;
+  int32_t e0, e1, de;
+};
+__device__ __forceinline__ LoraList lora_list(const GemmParams &p, const TileCoord &tc) {
+  LoraList l;
+  if (p.mode == kModePrefill) {
+    l.list = p.mt_list + tc.mtile * kTileM;
+    l.e0 = 0;
+    l.e1 = p.mt_count[tc.mtile];
+    l.de = 1;
+  } else if (p.mode == kModeDecode) {
+    l.list = p.lg_adapter;
+    l.e0 = tc.split;  // the groups are dealt round-robin to the K splits of a row tile
+    l.e1 = p.counts[4];
+    l.de = p.splits;
+  } else {
+    l.list = nullptr;
+    l.e0 = l.e1 = 0;
+    l.de = 1;
   }
-  if (valid) {
-    uint16_t *yrow = p.y + static_cast<size_t>(t) * p.h_out;
-#pragma unroll
-    for (int q = 0; q < NC; q += 8) {
-      const int j = col0 + q;
-      if (j < p.h_out) {  // h_out is a multiple of 8, so a group of 8 is all in or all out
-        uint4 o;
-        o.x = ptx::pack_bf16x2(acc[q + 0], acc[q + 1]);
-        o.y = ptx::pack_bf16x2(acc[q + 2], acc[q + 3]);
-        o.z = ptx::pack_bf16x2(acc[q + 4], acc[q + 5]);
-        o.w = ptx::pack_bf16x2(acc[q + 6], acc[q + 7]);
-        *reinterpret_cast<uint4 *>(yrow + j) = o;
-      }
-    }
-  }
+  return l;
 }
 
-// decode: row = W row j, columns = tokens c0 + [0, NC); partial sums to ws[split][t][j]
-template <int NC>
-__device__ __forceinline__ void epilogue_decode_chunk(const GemmParams &p, const float (&acc)[NC],
-                                                      int32_t j, int32_t split, int32_t c0) {
-  if (j >= p.h_out) return;
-  float *base = p.ws + (static_cast<size_t>(split) * p.T) * p.h_out + j;
-#pragma unroll
-  for (int jj = 0; jj < NC; ++jj) {
-    const int t = c0 + jj;
-    if (t < p.T) base[static_cast<size_t>(t) * p.h_out] = acc[jj];
-  }
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// sgmv: row = token of the run, columns = rank index; z partial = scale * acc
-template <int NC>
-__device__ __forceinline__ void epilogue_sgmv_chunk(const GemmParams &p, const float (&acc)[NC],
-                                                    int32_t t, bool valid, float scale,
-                                                    int32_t split, int32_t c0) {
-  if (!valid) return;
-  float *zrow = p.zws_out + (static_cast<size_t>(split) * p.max_tokens + t) * p.R_pad + c0;
-#pragma unroll
-  for (int q = 0; q < NC; q += 4) {
-    float4 o = make_float4(scale * acc[q], scale * acc[q + 1], scale * acc[q + 2], scale * acc[q + 3]);
-    *reinterpret_cast<float4 *>(zrow + q) = o;
-  }
-}
-
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(kGemmThreads, 2)
 lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_constant__ CUtensorMap tmap_c,
-                 const GemmParams p) {
+                 const __grid_constant__ CUtensorMap tmap_b, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   // tiles need 1024-byte alignment for the 128-byte swizzle
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -156,25 +121,33 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + static_cast<size_t>(p.stages) * stage_bytes);
   uint64_t *full_bar = bars;                      // [stages]  TMA -> MMA
   uint64_t *empty_bar = bars + kMaxStages;        // [stages]  MMA -> TMA
-  uint64_t *tfull_bar = bars + 2 * kMaxStages;    // [2]       MMA -> epilogue
+  uint64_t *zfull_bar = bars + 2 * kMaxStages;    // [stages]  builder -> MMA (LoRA K blocks)
+  uint64_t *zgo_bar = bars + 3 * kMaxStages;      // [stages]  TMA warp -> builder (stage is free)
+  uint64_t *tfull_bar = bars + 4 * kMaxStages;    // [2]       MMA -> epilogue
   uint64_t *tempty_bar = tfull_bar + 2;           // [2]       epilogue -> MMA
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(tempty_bar + 2);
   volatile uint32_t *abort_flag = tmem_slot + 1;
+  volatile uint32_t *last_flag = tmem_slot + 2;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool has_lora = p.mode != kModeSgmv;
 
   if (threadIdx.x == 0) {
     ptx::prefetch_tensormap(&tmap_r);
     ptx::prefetch_tensormap(&tmap_c);
+    if (has_lora) ptx::prefetch_tensormap(&tmap_b);
     for (int s = 0; s < p.stages; ++s) {
       ptx::mbar_init(&full_bar[s], 1);
       ptx::mbar_init(&empty_bar[s], 1);
+      ptx::mbar_init(&zfull_bar[s], 4);  // one arrival per builder warp
+      ptx::mbar_init(&zgo_bar[s], 1);
     }
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&tfull_bar[i], 1);
       ptx::mbar_init(&tempty_bar[i], 4);  // one arrival per epilogue warp
     }
     *abort_flag = 0;
+    *last_flag = 0;
     ptx::fence_barrier_init();
   }
   if (warp == 1) {
@@ -191,12 +164,13 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
 
   if (p.mode == kModeSgmv) ptx::pdl_wait_prior_grids();  // tile list comes from the plan kernel
   const int32_t n_tiles = total_tiles(p);
+  const uint32_t nstages = static_cast<uint32_t>(p.stages);
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
-      bool ok = true;
+      bool ok = true, waited = p.mode == kModeSgmv;
       for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
         const TileCoord tc = tile_coord(p, tile);
         for (int32_t kb = tc.kb0; kb < tc.kb1; ++kb) {
@@ -211,7 +185,36 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
             ptx::tma_load_3d(sr + r_bytes, &tmap_c, &full_bar[stage], kb * kBlockK, 0, tc.slot);
           else
             ptx::tma_load_2d(sr + r_bytes, &tmap_c, &full_bar[stage], kb * kBlockK, tc.row_c);
-          if (++stage == static_cast<uint32_t>(p.stages)) {
+          if (++stage == nstages) {
+            stage = 0;
+            phase ^= 1;
+          }
+        }
+        if (!ok || !has_lora) continue;
+        if (!waited) {  // the adapter lists come from the kernel before this one
+          ptx::pdl_wait_prior_grids();
+          waited = true;
+        }
+        const LoraList ll = lora_list(p, tc);
+        for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
+          const int32_t a = ll.list[e];
+          if (p.slots[a].rank <= 0) continue;
+          if (!ptx::mbar_wait(&empty_bar[stage], phase ^ 1) || *abort_flag) {
+            ok = false;
+            break;
+          }
+          // The stage is free: let the builder write its half (it follows this warp, never the
+          // stage barriers directly, so it cannot run ahead of the ring).
+          ptx::mbar_arrive(&zgo_bar[stage]);
+          uint8_t *sr = smem + static_cast<size_t>(stage) * stage_bytes;
+          if (p.mode == kModePrefill) {  // C operand: rows [row_c, row_c + BN) of B_a
+            ptx::mbar_arrive_expect_tx(&full_bar[stage], c_bytes);
+            ptx::tma_load_3d(sr + r_bytes, &tmap_b, &full_bar[stage], 0, tc.row_c, a);
+          } else {                       // R operand: rows [row_r, row_r + 128) of B_a
+            ptx::mbar_arrive_expect_tx(&full_bar[stage], r_bytes);
+            ptx::tma_load_3d(sr, &tmap_b, &full_bar[stage], 0, tc.row_r, a);
+          }
+          if (++stage == nstages) {
             stage = 0;
             phase ^= 1;
           }
@@ -226,8 +229,9 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = ptx::umma_idesc_bf16(kTileM, static_cast<uint32_t>(p.BN));
-      uint32_t stage = 0, phase = 0;
-      bool ok = true;
+      const int lora_ksteps = p.R_pad / kUmmaK;
+      uint32_t stage = 0, phase = 0, zphase = 0;  // zphase: one parity bit per stage
+      bool ok = true, waited = p.mode == kModeSgmv;
       int32_t it = 0;
       for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++it) {
         const TileCoord tc = tile_coord(p, tile);
@@ -254,12 +258,40 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
             ptx::umma_bf16(tmem_d, da + 2 * k, db + 2 * k, idesc, (kb > tc.kb0 || k > 0) ? 1u : 0u);
           }
           ptx::umma_commit(&empty_bar[stage]);  // frees the smem stage once these MMAs are done
-          if (++stage == static_cast<uint32_t>(p.stages)) {
+          if (++stage == nstages) {
             stage = 0;
             phase ^= 1;
           }
         }
         if (!ok) break;
+        if (has_lora) {
+          if (!waited) {
+            ptx::pdl_wait_prior_grids();
+            waited = true;
+          }
+          const LoraList ll = lora_list(p, tc);
+          for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
+            const int32_t a = ll.list[e];
+            if (p.slots[a].rank <= 0) continue;
+            if (!ptx::mbar_wait(&full_bar[stage], phase) ||
+                !ptx::mbar_wait(&zfull_bar[stage], (zphase >> stage) & 1u) || *abort_flag) {
+              ok = false;
+              break;
+            }
+            zphase ^= 1u << stage;
+            ptx::tc_fence_after_sync();
+            const uint32_t sr = ptx::smem_u32(smem + static_cast<size_t>(stage) * stage_bytes);
+            const uint64_t da = ptx::umma_desc_k128(sr);
+            const uint64_t db = ptx::umma_desc_k128(sr + r_bytes);
+            for (int k = 0; k < lora_ksteps; ++k) ptx::umma_bf16(tmem_d, da + 2 * k, db + 2 * k, idesc, 1u);
+            ptx::umma_commit(&empty_bar[stage]);
+            if (++stage == nstages) {
+              stage = 0;
+              phase ^= 1;
+            }
+          }
+          if (!ok) break;
+        }
         ptx::umma_commit(&tfull_bar[acc]);  // accumulator complete
       }
       if (!ok) {
@@ -267,83 +299,234 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         atomicOr(p.status, EDGELORA_STATUS_TIMEOUT);
       }
     }
-  } else {
+  } else if (warp < 6) {
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int quad = warp & 3;                      // TMEM lanes [32*quad, 32*quad+32)
     const int row_in_tile = quad * 32 + lane;
-    ptx::pdl_wait_prior_grids();                    // z / plan / workspace owners have finished
+    const int etid = threadIdx.x - 64;              // 0..127
+    const bool reduce_here = p.mode == kModeDecode && p.splits > 1;
+    ptx::pdl_wait_prior_grids();                    // earlier kernels may still read y / the workspace
     bool ok = true;
     int32_t it = 0;
     for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++it) {
       const TileCoord tc = tile_coord(p, tile);
       const uint32_t acc = (p.n_acc == 2) ? (it & 1) : 0;
       const uint32_t use = (p.n_acc == 2) ? (it >> 1) : it;
-
-      // per-row state that does not need the accumulator
-      int32_t a = -1, rank = 0;
-      float scale = 0.f;
-      bool valid = false;
-      float z[64];
       const int32_t row = tc.row_r + row_in_tile;
-      if (p.mode == kModePrefill) {
-        valid = row < p.T;
-        if (valid) a = p.ids_valid[row];
-        if (a >= 0) rank = p.slots[a].rank;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          if (c * 8 < rank) {
-            float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
-            for (int sp = 0; sp < p.zsplits; ++sp) {
-              const float4 *zp = reinterpret_cast<const float4 *>(
-                  p.zws + (static_cast<size_t>(sp) * p.max_tokens + row) * p.R_pad + c * 8);
-              const float4 u = zp[0], v = zp[1];
-              lo.x += u.x; lo.y += u.y; lo.z += u.z; lo.w += u.w;
-              hi.x += v.x; hi.y += v.y; hi.z += v.z; hi.w += v.w;
-            }
-            z[c * 8 + 0] = lo.x; z[c * 8 + 1] = lo.y; z[c * 8 + 2] = lo.z; z[c * 8 + 3] = lo.w;
-            z[c * 8 + 4] = hi.x; z[c * 8 + 5] = hi.y; z[c * 8 + 6] = hi.z; z[c * 8 + 7] = hi.w;
-          } else {
-#pragma unroll
-            for (int q = 0; q < 8; ++q) z[c * 8 + q] = 0.f;
-          }
-        }
-      } else if (p.mode == kModeSgmv) {
-        valid = row_in_tile < tc.nrows;
-        scale = p.slots[tc.slot].scale;
-      }
+      float scale = 0.f;
+      if (p.mode == kModeSgmv) scale = p.slots[tc.slot].scale;
 
-      if (!ptx::mbar_wait(&tfull_bar[acc], use & 1) || *abort_flag) {
+      const bool got = ptx::mbar_wait(&tfull_bar[acc], use & 1) && !*abort_flag;
+      if (!got) {
         ok = false;
-        break;
+        *abort_flag = 1;
+        if (!reduce_here) break;
       }
       ptx::tc_fence_after_sync();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                              acc * static_cast<uint32_t>(p.BN);
-      for (int32_t c0 = 0; c0 < p.BN; c0 += 32) {
+      for (int32_t c0 = 0; got && c0 < p.BN; c0 += 32) {
+        float v[32];
         if (p.BN - c0 >= 32) {
-          float v[32];
           ptx::tmem_ld_32x32(taddr + c0, v);
-          if (p.mode == kModePrefill)
-            epilogue_prefill_chunk<32>(p, v, row, valid, a, rank, z, tc.row_c + c0);
-          else if (p.mode == kModeDecode)
-            epilogue_decode_chunk<32>(p, v, row, tc.split, c0);
-          else
-            epilogue_sgmv_chunk<32>(p, v, row, valid, scale, tc.split, c0);
+        } else {  // sgmv with a rank stride of 16: only 16 columns exist
+          float h[16];
+          ptx::tmem_ld_32x16(taddr + c0, h);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            v[i] = h[i];
+            v[i + 16] = 0.f;
+          }
+        }
+        if (p.mode == kModePrefill) {
+          // row = token, columns = output features row_c + c0 + [0, 32)
+          if (row < p.T) {
+            uint16_t *yrow = p.y + static_cast<size_t>(row) * p.h_out;
+#pragma unroll
+            for (int q = 0; q < 32; q += 8) {
+              const int j = tc.row_c + c0 + q;
+              if (j < p.h_out) {  // h_out is a multiple of 8: a group of 8 is all in or all out
+                uint4 o;
+                o.x = ptx::pack_bf16x2(v[q + 0], v[q + 1]);
+                o.y = ptx::pack_bf16x2(v[q + 2], v[q + 3]);
+                o.z = ptx::pack_bf16x2(v[q + 4], v[q + 5]);
+                o.w = ptx::pack_bf16x2(v[q + 6], v[q + 7]);
+                *reinterpret_cast<uint4 *>(yrow + j) = o;
+              }
+            }
+          }
+        } else if (p.mode == kModeDecode) {
+          // row = W row j, columns = tokens c0 + [0, 32)
+          if (row < p.h_out) {
+            if (p.splits == 1) {
+#pragma unroll
+              for (int jj = 0; jj < 32; ++jj) {
+                const int t = c0 + jj;
+                if (t < p.T)
+                  p.y[static_cast<size_t>(t) * p.h_out + row] =
+                      static_cast<uint16_t>(ptx::pack_bf16x2(v[jj], 0.f) & 0xFFFFu);
+              }
+            } else {
+              float *base = p.ws + (static_cast<size_t>(tc.split) * p.T) * p.h_out + row;
+#pragma unroll
+              for (int jj = 0; jj < 32; ++jj) {
+                const int t = c0 + jj;
+                if (t < p.T) base[static_cast<size_t>(t) * p.h_out] = v[jj];
+              }
+            }
+          }
         } else {
-          float v[16];
-          ptx::tmem_ld_32x16(taddr + c0, v);
-          if (p.mode == kModePrefill)
-            epilogue_prefill_chunk<16>(p, v, row, valid, a, rank, z, tc.row_c + c0);
-          else if (p.mode == kModeDecode)
-            epilogue_decode_chunk<16>(p, v, row, tc.split, c0);
-          else
-            epilogue_sgmv_chunk<16>(p, v, row, valid, scale, tc.split, c0);
+          // sgmv: row = token of the run, columns = rank index; z partial = scale * acc
+          if (row_in_tile < tc.nrows) {
+            float *zrow = p.zws_out + (static_cast<size_t>(tc.split) * p.max_tokens + row) * p.R_pad + c0;
+            const int nc = min(32, p.BN - c0);
+            for (int q = 0; q < nc; q += 4)
+              *reinterpret_cast<float4 *>(zrow + q) =
+                  make_float4(scale * v[q], scale * v[q + 1], scale * v[q + 2], scale * v[q + 3]);
+          }
         }
       }
-      // all TMEM reads of this warp are complete (tcgen05.wait::ld inside the loads)
-      ptx::tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&tempty_bar[acc]);
+      if (got) {
+        // all TMEM reads of this warp are complete (tcgen05.wait::ld inside the loads)
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&tempty_bar[acc]);
+      }
+
+      if (reduce_here) {
+        // Split-K reduction by whichever CTA finishes this row tile last (it never waits).  All
+        // four warps pass the named barriers together even when a wait gave up, and leave the loop
+        // together afterwards.
+        __threadfence();
+        named_bar_sync(1, 128);
+        if (etid == 0) {
+          uint32_t last = 0;
+          if (!*abort_flag) {
+            const int old = atomicAdd(&p.tile_counters[tc.mtile], 1);
+            last = (old == p.splits - 1) ? 1u : 0u;
+            if (last) p.tile_counters[tc.mtile] = 0;  // ready for the next launch
+          }
+          *last_flag = last;
+        }
+        named_bar_sync(1, 128);
+        if (*last_flag) {
+          __threadfence();
+          // unit = (token, 4 adjacent W rows); all partials of a unit are loaded before any is used
+          const int n_units = p.T * 32;
+          const size_t plane = static_cast<size_t>(p.T) * p.h_out;
+          for (int u = etid; u < n_units; u += 128) {
+            const int t = u >> 5, j = tc.row_r + ((u & 31) << 2);
+            if (j >= p.h_out) continue;  // h_out is a multiple of 8: 4 rows are all in or all out
+            const float *src = p.ws + static_cast<size_t>(t) * p.h_out + j;
+            float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int sp0 = 0; sp0 < p.splits; sp0 += 8) {
+              float4 v[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                v[i] = (sp0 + i < p.splits)
+                           ? __ldcg(reinterpret_cast<const float4 *>(src + (sp0 + i) * plane))
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                acc4.x += v[i].x; acc4.y += v[i].y; acc4.z += v[i].z; acc4.w += v[i].w;
+              }
+            }
+            uint2 o;
+            o.x = ptx::pack_bf16x2(acc4.x, acc4.y);
+            o.y = ptx::pack_bf16x2(acc4.z, acc4.w);
+            *reinterpret_cast<uint2 *>(p.y + static_cast<size_t>(t) * p.h_out + j) = o;
+          }
+        }
+        named_bar_sync(1, 128);  // last_flag is rewritten by the next tile
+        if (*abort_flag) ok = false;
+      }
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      atomicOr(p.status, EDGELORA_STATUS_TIMEOUT);
+    }
+  } else if (has_lora) {
+    // ------------------------------------------------------------ z operand builder (warps 6..9)
+    const int btid = threadIdx.x - 192;  // 0..127
+    const int nch = p.R_pad >> 3;        // 16-byte chunks of one operand row that the MMAs read
+    uint32_t count = 0;                  // K blocks so far: stage = count % stages
+    uint32_t gophase = 0;                // one parity bit per stage for zgo_bar
+    const uint32_t zsplits = static_cast<uint32_t>(p.zsplits);
+    bool ok = true, waited = false;
+    for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+      const TileCoord tc = tile_coord(p, tile);
+      count += static_cast<uint32_t>(tc.kb1 - tc.kb0);
+      if (!waited) {  // z and the adapter lists come from the kernels before this one
+        ptx::pdl_wait_prior_grids();
+        waited = true;
+      }
+      const LoraList ll = lora_list(p, tc);
+      const int rows = (p.mode == kModePrefill) ? kTileM : p.BN;
+      const int tok0 = (p.mode == kModePrefill) ? tc.row_r : 0;
+      const uint32_t region = (p.mode == kModePrefill) ? 0u : r_bytes;
+      // the ids of this thread's rows do not change over the tile's LoRA blocks
+      int32_t id_lo = -1, id_hi = -1;
+      if (tok0 + btid < p.T) id_lo = p.ids_valid[tok0 + btid];
+      if (rows > 128 && tok0 + btid + 128 < p.T) id_hi = p.ids_valid[tok0 + btid + 128];
+      for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
+        const int32_t a = ll.list[e];
+        const int32_t rank = p.slots[a].rank;
+        if (rank <= 0) continue;
+        const uint32_t stage = count % nstages;
+        ++count;
+        if (!ptx::mbar_wait(&zgo_bar[stage], (gophase >> stage) & 1u) || *abort_flag) {
+          ok = false;
+          break;
+        }
+        gophase ^= 1u << stage;
+        uint8_t *dst = smem + static_cast<size_t>(stage) * stage_bytes + region;
+        for (int r = btid; r < rows; r += 128) {
+          const bool match = ((r < 128) ? id_lo : id_hi) == a;
+          uint8_t *drow = dst + r * 128;
+          if (!match) {
+            for (int c = 0; c < nch; ++c)
+              *reinterpret_cast<uint4 *>(drow + ((c ^ (r & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+            continue;
+          }
+          // z of this token: sum the partial planes in order, four chunks of a plane in flight
+          const float *zt = p.zws + static_cast<size_t>(tok0 + r) * p.R_pad;
+          const size_t plane = static_cast<size_t>(p.max_tokens) * p.R_pad;
+          for (int c0 = 0; c0 < nch; c0 += 4) {
+            float acc[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+            for (uint32_t sp = 0; sp < zsplits; ++sp) {
+              const float4 *zp = reinterpret_cast<const float4 *>(zt + sp * plane) + 2 * c0;
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                if (c0 + c < nch) {
+                  const float4 u = __ldcg(zp + 2 * c), w = __ldcg(zp + 2 * c + 1);
+                  acc[c * 8 + 0] += u.x; acc[c * 8 + 1] += u.y; acc[c * 8 + 2] += u.z; acc[c * 8 + 3] += u.w;
+                  acc[c * 8 + 4] += w.x; acc[c * 8 + 5] += w.y; acc[c * 8 + 6] += w.z; acc[c * 8 + 7] += w.w;
+                }
+              }
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              if (c0 + c < nch) {
+                uint4 o;
+                // values at or past the true rank are not defined by the shrink: force zero
+#define EL(i) (((c0 + c) * 8 + (i)) < rank ? acc[c * 8 + (i)] : 0.f)
+                o.x = ptx::pack_bf16x2(EL(0), EL(1));
+                o.y = ptx::pack_bf16x2(EL(2), EL(3));
+                o.z = ptx::pack_bf16x2(EL(4), EL(5));
+                o.w = ptx::pack_bf16x2(EL(6), EL(7));
+#undef EL
+                // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
+                *reinterpret_cast<uint4 *>(drow + (((c0 + c) ^ (r & 7)) << 4)) = o;
+              }
+            }
+          }
+        }
+        fence_proxy_async_smem();  // make the generic-proxy writes visible to the tensor core
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&zfull_bar[stage]);
+      }
     }
     if (!ok && lane == 0) {
       *abort_flag = 1;
@@ -365,10 +548,10 @@ cudaError_t gemm_set_smem_limit(size_t smem_bytes) {
 }
 
 cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
-                        const GemmParams &p, int32_t grid, size_t smem_bytes, bool pdl,
-                        cudaStream_t stream) {
+                        const CUtensorMap &tmap_b, const GemmParams &p, int32_t grid,
+                        size_t smem_bytes, bool pdl, cudaStream_t stream) {
   return launch_ex(lora_gemm_kernel, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl,
-                   tmap_row, tmap_col, p);
+                   tmap_row, tmap_col, tmap_b, p);
 }
 
 }  // namespace edgelora

@@ -15,7 +15,9 @@ constexpr int kMaxStages = 12;
 constexpr int kSegMin = 32;        // prefill: runs at least this long go through the segment shrink
 constexpr int kDecodeMaxT = 256;   // decode regime: all tokens are one UMMA N tile
 constexpr int kMaxTokensLimit = 32768;
-constexpr int kGemmThreads = 192;  // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int kGemmThreads = 320;  // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue, warps 6..9 z operand
+constexpr int kMaxZSplits = 16;    // partial z planes (K splits of the shrink); plane 16 = summed z
+constexpr int kShrinkThreads = 256;
 
 // One row of the slot table (paper Section 3.3: one fixed block per resident adapter).
 struct SlotRow {
@@ -38,7 +40,11 @@ struct PlanView {
   int32_t *gs_short;       // [maxT+1] group boundaries inside perm_short
   int32_t *sgmv_tiles;     // [max_sgmv_tiles][4] {first token, tokens, slot, 0}
   int32_t *scratch;        // [maxT+1]
-  int32_t *counts;         // [8]  0: n_groups, 1: n_segments, 2: n_sgmv_tiles
+  int32_t *lg_adapter;     // [maxT]   distinct ids >= 0 of the batch, ascending (the LoRA groups)
+  int32_t *mt_count;       // [maxT/128+1] distinct ids >= 0 inside each 128-token tile
+  int32_t *mt_list;        // [ceil(maxT/128)*128] those ids, tile m at [128 m, 128 m + mt_count[m])
+  int32_t *counts;         // [8]  0: n_groups, 1: n_segments, 2: n_sgmv_tiles, 3: short tokens,
+                           //      4: LoRA groups, 5: K chunks used by the decode shrink
   uint32_t *status;        // device status word of the plan
   int32_t max_sgmv_tiles;
 };
@@ -58,7 +64,7 @@ struct GemmParams {
   int32_t n_mtiles;    // prefill: token tiles; decode: W row tiles
   int32_t n_ntiles;    // prefill: W row tiles of BN
   int32_t R_pad;       // slot block rank stride
-  int32_t zsplits;     // partial z buffers the consumer sums
+  int32_t zsplits;     // partial z planes the consumer sums
   int32_t max_tokens;  // row stride of the z / plan workspaces
   const int32_t *ids_valid;
   const SlotRow *slots;
@@ -69,6 +75,10 @@ struct GemmParams {
   float *ws;                // decode partials [splits][T][h_out]
   const int32_t *sgmv_tiles;
   const int32_t *counts;
+  const int32_t *lg_adapter;  // decode: LoRA groups of the batch
+  const int32_t *mt_count;    // prefill: per 128-token tile
+  const int32_t *mt_list;
+  int32_t *tile_counters;     // decode: arrivals per W row tile (split-K reduction by the last one)
   uint32_t *status;
 };
 
@@ -81,12 +91,13 @@ void launch_bgmv_shrink(const uint16_t *x, const uint16_t *A_pool, const SlotRow
                         bool pdl, cudaStream_t stream);
 void init_plan_kernel();
 cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
-                        const GemmParams &p, int32_t grid, size_t smem_bytes, bool pdl,
-                        cudaStream_t stream);
+                        const CUtensorMap &tmap_b, const GemmParams &p, int32_t grid,
+                        size_t smem_bytes, bool pdl, cudaStream_t stream);
 cudaError_t gemm_set_smem_limit(size_t smem_bytes);
-void launch_decode_combine(const float *ws, int32_t splits, const float *zws, int32_t zsplits,
-                           int32_t max_tokens, const uint16_t *B_pool, const SlotRow *slots,
-                           const int32_t *ids_valid, uint16_t *y, int32_t T, int32_t h_out,
-                           int32_t R_pad, bool pdl, cudaStream_t stream);
+void launch_decode_shrink(const int32_t *ids, const uint16_t *x, const uint16_t *A_pool,
+                          const SlotRow *slots, const PlanView &pv, float *zws,
+                          int32_t *group_counters, int32_t T, int32_t h_in, int32_t R_pad,
+                          int32_t n_slots, int32_t max_tokens, int32_t target_items, int32_t grid,
+                          uint32_t *status, bool pdl, cudaStream_t stream);
 
 }  // namespace edgelora

@@ -137,9 +137,17 @@ plan_kernel(const int32_t *__restrict__ ids, int32_t T, int32_t n_slots, PlanVie
       pv.group_adapter[g] = static_cast<int32_t>(keys[i] >> 16) - 1;
     }
   }
+  const int has_base = (keys[0] >> 16) == 0 ? 1 : 0;  // the group of id -1 sorts first
+  for (int i = tid; i < T; i += kPlanThreads) {
+    const uint32_t id1 = keys[i] >> 16;
+    if (id1 != 0 && (i == 0 || id1 != (keys[i - 1] >> 16)))
+      pv.lg_adapter[pv.scratch[i] - has_base] = static_cast<int32_t>(id1) - 1;
+  }
   if (tid == 0) {
     pv.group_start[n_groups] = T;
     pv.counts[0] = n_groups;
+    pv.counts[4] = n_groups - has_base;
+    pv.counts[5] = 0;
   }
   __syncthreads();
 
@@ -189,6 +197,54 @@ plan_kernel(const int32_t *__restrict__ ids, int32_t T, int32_t n_slots, PlanVie
     }
   }
   if (tid == 0) pv.counts[2] = min(n_tiles, pv.max_sgmv_tiles);
+
+  // 6. the distinct ids >= 0 inside every 128-token tile, in order of first appearance (the LoRA
+  // K blocks of that tile in the base-product kernel).  One warp per tile; lane l holds the ids
+  // of tokens l, l + 32, l + 64, l + 96 of the tile.
+  {
+    const int lane = tid & 31, warp = tid >> 5;
+    const int n_mt = (T + kTileM - 1) / kTileM;
+    for (int m = warp; m < n_mt; m += kPlanThreads / 32) {
+      int32_t id[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int t = m * kTileM + q * 32 + lane;
+        id[q] = t < T ? pv.ids_valid[t] : -1;
+      }
+      const int32_t id0 = __shfl_sync(0xffffffffu, id[0], 0);
+      bool same = true;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) same = same && (id[q] == id0);
+      if (__all_sync(0xffffffffu, same)) {  // the usual prefill tile: one run
+        if (lane == 0) {
+          pv.mt_count[m] = id0 >= 0 ? 1 : 0;
+          pv.mt_list[m * kTileM] = id0;
+        }
+        continue;
+      }
+      bool first[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) first[q] = id[q] >= 0;
+#pragma unroll
+      for (int qq = 0; qq < 4; ++qq) {
+        for (int src = 0; src < 32; ++src) {
+          const int32_t v = __shfl_sync(0xffffffffu, id[qq], src);
+          const int pos = qq * 32 + src;
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (pos < q * 32 + lane && v == id[q]) first[q] = false;
+        }
+      }
+      int base = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint32_t b = __ballot_sync(0xffffffffu, first[q]);
+        if (first[q]) pv.mt_list[m * kTileM + base + __popc(b & ((1u << lane) - 1u))] = id[q];
+        base += __popc(b);
+      }
+      if (lane == 0) pv.mt_count[m] = base;
+    }
+  }
 }
 
 void launch_plan(const int32_t *ids, int32_t T, int32_t n_slots, const PlanView &pv, bool pdl,

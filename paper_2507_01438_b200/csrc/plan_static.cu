@@ -13,11 +13,14 @@ namespace {
 
 constexpr int kStaticMaxTokens = EDGELORA_PLAN_STATIC_MAX_TOKENS;
 constexpr int kStaticMaxTiles = kStaticMaxTokens / kSegMin + 8;
-// tok_seg, perm_short: T each; gs_short, scratch: T + 1 each; tile list; counts[8]; status[4]
-constexpr int kStaticInts = 2 * kStaticMaxTokens + 2 * (kStaticMaxTokens + 1) + 4 * kStaticMaxTiles + 8 + 4;
+constexpr int kStaticTokenTiles = (kStaticMaxTokens + kTileM - 1) / kTileM;
+// tok_seg, perm_short, lg_adapter: T each; gs_short, scratch: T + 1 each; segment tile list;
+// per-token-tile adapter lists; counts[8]; status[4]
+constexpr int kStaticInts = 3 * kStaticMaxTokens + 2 * (kStaticMaxTokens + 1) + 4 * kStaticMaxTiles +
+                            (kStaticTokenTiles + 1) + kStaticTokenTiles * kTileM + 8 + 4;
 constexpr int kMaxDevices = 64;
 
-// Held by every GPU that loads the library, until the process exits (about 66 KB).
+// Held by every GPU that loads the library, until the process exits (about 100 KB).
 static __device__ __align__(256) int32_t g_plan_scratch[kStaticInts];
 
 std::mutex g_mutex;
@@ -73,6 +76,9 @@ extern "C" int edgelora_plan_build_static(const int32_t *adapter_id_dev, int32_t
   pv.gs_short = q; q += kStaticMaxTokens + 1;
   pv.scratch = q; q += kStaticMaxTokens + 1;
   pv.sgmv_tiles = q; q += 4 * kStaticMaxTiles;
+  pv.lg_adapter = q; q += kStaticMaxTokens;
+  pv.mt_count = q; q += kStaticTokenTiles + 1;
+  pv.mt_list = q; q += kStaticTokenTiles * kTileM;
   pv.counts = q; q += 8;
   pv.status = reinterpret_cast<uint32_t *>(q);
   pv.max_sgmv_tiles = kStaticMaxTiles;

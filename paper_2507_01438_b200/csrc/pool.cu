@@ -19,10 +19,10 @@ using namespace edgelora;
 namespace {
 
 constexpr int kStagingBuffers = 4;
-constexpr int kMaxZSplits = 8;
 constexpr int kTmapCache = 32;
 constexpr int kProfEvents = 8192;
 constexpr size_t kSmemBudget = 220 * 1024;
+constexpr int kMaxDecodeSplits = 32;
 
 #define CUDA_TRY(expr)                                   \
   do {                                                   \
@@ -129,6 +129,8 @@ struct edgelora_pool {
   bool use_recorded = false;
   edgelora_plan *plan = nullptr;
   float *zws = nullptr, *ws = nullptr;
+  int32_t *tile_counters = nullptr, *group_counters = nullptr;
+  int opt_decode_splits = 0, opt_shrink_items = 0;
   size_t ws_floats = 0;
   uint32_t *status_dev = nullptr;
   std::vector<TmapEntry> tmaps;
@@ -217,7 +219,10 @@ int plan_alloc(edgelora_plan *pl) {
   const int max_tiles = pl->max_tokens / kSegMin + 8;
   // ids_valid, perm, group_adapter, seg_adapter, tok_seg, perm_short: mt each;
   // group_start, seg_start, gs_short, scratch: mt + 1 each; tiles; counts; status
-  const size_t ints = 6 * mt + 4 * (mt + 1) + 4 * static_cast<size_t>(max_tiles) + 8 + 4;
+  // lg_adapter: mt; mt_count: n_mt + 1; mt_list: n_mt * 128
+  const size_t n_mt = (mt + kTileM - 1) / kTileM;
+  const size_t ints = 7 * mt + 4 * (mt + 1) + 4 * static_cast<size_t>(max_tiles) + (n_mt + 1) +
+                      n_mt * kTileM + 8 + 4;
   CUDA_TRY(cudaMalloc(&pl->block, ints * 4));
   CUDA_TRY(cudaMemset(pl->block, 0, ints * 4));
   int32_t *q = static_cast<int32_t *>(pl->block);
@@ -233,6 +238,9 @@ int plan_alloc(edgelora_plan *pl) {
   v.gs_short = q; q += mt + 1;
   v.scratch = q; q += mt + 1;
   v.sgmv_tiles = q; q += 4 * static_cast<size_t>(max_tiles);
+  v.lg_adapter = q; q += mt;
+  v.mt_count = q; q += n_mt + 1;
+  v.mt_list = q; q += n_mt * kTileM;
   v.counts = q; q += 8;
   v.status = reinterpret_cast<uint32_t *>(q);
   v.max_sgmv_tiles = max_tiles;
@@ -401,13 +409,18 @@ int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool
   POOL_TRY(cudaStreamCreateWithFlags(&p->side, cudaStreamNonBlocking));
   POOL_TRY(cudaEventCreateWithFlags(&p->load_ev, cudaEventDisableTiming));
   POOL_TRY(cudaEventCreateWithFlags(&p->use_ev, cudaEventDisableTiming));
-  POOL_TRY(cudaMalloc(&p->zws, sizeof(float) * kMaxZSplits * static_cast<size_t>(p->cfg.max_tokens) * p->R_pad));
+  // partial planes [0, kMaxZSplits) plus the final plane of the decode shrink
+  POOL_TRY(cudaMalloc(&p->zws, sizeof(float) * (kMaxZSplits + 1) * static_cast<size_t>(p->cfg.max_tokens) * p->R_pad));
+  POOL_TRY(cudaMalloc(&p->group_counters, sizeof(int32_t) * kDecodeMaxT));
+  POOL_TRY(cudaMemset(p->group_counters, 0, sizeof(int32_t) * kDecodeMaxT));
   // decode partials: splits * T * h_out with splits <= sms / row_tiles + 1 and T <= 256
   {
     const int row_tiles = (cfg->h_out + kTileM - 1) / kTileM;
-    const int max_splits = std::max(1, p->sms / row_tiles) + 1;
+    const int max_splits = std::min(kMaxDecodeSplits, std::max(1, 2 * p->sms / row_tiles) + 1);
     p->ws_floats = static_cast<size_t>(max_splits) * kDecodeMaxT * cfg->h_out;
     POOL_TRY(cudaMalloc(&p->ws, p->ws_floats * sizeof(float)));
+    POOL_TRY(cudaMalloc(&p->tile_counters, sizeof(int32_t) * row_tiles));
+    POOL_TRY(cudaMemset(p->tile_counters, 0, sizeof(int32_t) * row_tiles));
   }
   POOL_TRY(gemm_set_smem_limit(kSmemBudget));
   rc = edgelora_plan_create(p->cfg.max_tokens, cfg->n_slots, &p->plan);
@@ -436,6 +449,8 @@ int edgelora_pool_destroy(edgelora_pool_t *p) {
   if (p->use_ev) cudaEventDestroy(p->use_ev);
   if (p->zws) cudaFree(p->zws);
   if (p->ws) cudaFree(p->ws);
+  if (p->tile_counters) cudaFree(p->tile_counters);
+  if (p->group_counters) cudaFree(p->group_counters);
   for (auto &r : p->prof) {
     cudaEventDestroy(r.start);
     cudaEventDestroy(r.stop);
@@ -539,7 +554,16 @@ int edgelora_pool_set_option(edgelora_pool_t *p, int32_t option, int32_t value) 
       }
       return EDGELORA_OK;
     case EDGELORA_OPT_PDL:
-      p->opt_pdl = value ? 1 : 0;
+      if (value < 0 || value > 2) return EDGELORA_ERR_INVALID_ARG;
+      p->opt_pdl = value;
+      return EDGELORA_OK;
+    case EDGELORA_OPT_DECODE_SPLITS:
+      if (value < 0 || value > kMaxDecodeSplits) return EDGELORA_ERR_INVALID_ARG;
+      p->opt_decode_splits = value;
+      return EDGELORA_OK;
+    case EDGELORA_OPT_SHRINK_ITEMS:
+      if (value < 0) return EDGELORA_ERR_INVALID_ARG;
+      p->opt_shrink_items = value;
       return EDGELORA_OK;
     default:
       return EDGELORA_ERR_INVALID_ARG;
@@ -592,7 +616,9 @@ int edgelora_pool_sync_status(edgelora_pool_t *p, uint32_t *bits_out) {
   return EDGELORA_OK;
 }
 
-// The layer: plan (optional) -> shrink -> base product -> expand/combine.
+// The layer.  Decode regime (T <= 256): routing + shrink in one kernel, then the base product with
+// the expand and the split-K reduction fused in.  Prefill regime: plan, gather shrink for short
+// runs, segment shrink for long runs, base product with the expand fused in.
 static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_dev,
                             const void *W_dev, const void *x_dev, int32_t T, void *y_dev,
                             cudaStream_t stream) {
@@ -604,9 +630,11 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     return EDGELORA_ERR_INVALID_ARG;
   if (T > p->cfg.max_tokens || T > plan->max_tokens) return EDGELORA_ERR_TOO_MANY_TOKENS;
   if (plan->n_slots != p->cfg.n_slots) return EDGELORA_ERR_INVALID_ARG;
+  if (!ids_dev && plan->last_T != T) return EDGELORA_ERR_INVALID_ARG;
   const int h_in = p->cfg.h_in, h_out = p->cfg.h_out, R = p->R_pad;
   const bool capturing = stream_capturing(stream);
-  const bool pdl = p->opt_pdl && !p->opt_profile;
+  const bool pdl = p->opt_pdl >= 1 && !p->opt_profile;        // between the kernels of this call
+  const bool pdl_first = p->opt_pdl >= 2 && !p->opt_profile;  // first kernel vs earlier stream work
   const uint16_t *x = static_cast<const uint16_t *>(x_dev);
   int launches = 0;
 
@@ -615,38 +643,10 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     p->load_seq_waited = p->load_seq;
   }
 
-  if (ids_dev) {
-    ProfScope ps(p, 0, stream);
-    plan->last_T = T;
-    launch_plan(ids_dev, T, plan->n_slots, plan->pv, pdl, stream);
-    CUDA_TRY(cudaGetLastError());
-    ++launches;
-  } else if (plan->last_T != T) {
-    return EDGELORA_ERR_INVALID_ARG;
-  }
-
   int regime = (T <= kDecodeMaxT) ? 1 : 2;
   if (p->opt_regime == 2) regime = 2;
   if (p->opt_regime == 1 && T > kDecodeMaxT) return EDGELORA_ERR_INVALID_ARG;
-  const bool sgmv = T > kDecodeMaxT;
   const int kb_total = (h_in + kBlockK - 1) / kBlockK;
-
-  // segment-shrink split-K factor (number of partial z buffers the consumers sum)
-  int zsplits = 1;
-  if (sgmv) {
-    const int tiles_est = std::max(1, T / kTileM);
-    zsplits = std::max(1, std::min({kMaxZSplits, p->sms / tiles_est, kb_total / 4}));
-    const int kb_per = (kb_total + zsplits - 1) / zsplits;
-    zsplits = (kb_total + kb_per - 1) / kb_per;
-  }
-
-  {
-    ProfScope ps(p, 1, stream);
-    launch_bgmv_shrink(x, p->A_pool, p->slots_dev, plan->pv, p->zws, T, h_in, R, p->cfg.n_slots,
-                       zsplits, p->cfg.max_tokens, p->status_dev, pdl, stream);
-    CUDA_TRY(cudaGetLastError());
-    ++launches;
-  }
 
   GemmParams g{};
   g.T = T;
@@ -654,7 +654,6 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
   g.h_out = h_out;
   g.kb_total = kb_total;
   g.R_pad = R;
-  g.zsplits = zsplits;
   g.max_tokens = p->cfg.max_tokens;
   g.ids_valid = plan->pv.ids_valid;
   g.slots = p->slots_dev;
@@ -665,14 +664,18 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
   g.ws = p->ws;
   g.sgmv_tiles = plan->pv.sgmv_tiles;
   g.counts = plan->pv.counts;
+  g.lg_adapter = plan->pv.lg_adapter;
+  g.mt_count = plan->pv.mt_count;
+  g.mt_list = plan->pv.mt_list;
+  g.tile_counters = p->tile_counters;
   g.status = p->status_dev;
 
   auto smem_for = [](int stages, int BN) {
     return static_cast<size_t>(1024 + stages * (kTileM * kBlockK * 2 + BN * kBlockK * 2) + 512);
   };
-  auto stages_for = [&](int BN, int kb_per_cta) {
-    int s = static_cast<int>((kSmemBudget - 1536) / (kTileM * kBlockK * 2 + BN * kBlockK * 2));
-    return std::max(1, std::min({s, kMaxStages, std::max(2, kb_per_cta)}));
+  auto stages_for = [&](int BN, int k_blocks_per_cta, size_t budget) {
+    int s = static_cast<int>((budget - 1536) / (kTileM * kBlockK * 2 + BN * kBlockK * 2));
+    return std::max(1, std::min({s, kMaxStages, std::max(2, k_blocks_per_cta)}));
   };
   auto pow2_cols = [](int cols) {
     int c = 32;
@@ -680,63 +683,103 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     return c;
   };
 
-  if (sgmv) {
-    GemmParams s = g;
-    s.mode = kModeSgmv;
-    s.BN = R;
-    s.splits = zsplits;
-    s.kb_per = (kb_total + zsplits - 1) / zsplits;
-    s.stages = stages_for(R, s.kb_per);
-    s.n_acc = 2;
-    s.tmem_cols = pow2_cols(2 * R);
-    const CUtensorMap *mr, *mc;
-    int rc = get_tmap(p, &mr, x, h_in, T, 0, kTileM);
-    if (rc) return rc;
-    rc = get_tmap(p, &mc, p->A_pool, h_in, R, p->cfg.n_slots, R);
-    if (rc) return rc;
-    const int grid = std::max(1, std::min(p->sms, plan->pv.max_sgmv_tiles * zsplits));
-    ProfScope ps(p, 2, stream);
-    CUDA_TRY(launch_gemm(*mr, *mc, s, grid, smem_for(s.stages, R), pdl, stream));
-    ++launches;
-  }
-
   if (regime == 1) {
+    // ---------------------------------------------------------------- decode
+    const int32_t *ids_in = ids_dev ? ids_dev : plan->pv.ids_valid;
+    plan->last_T = T;
+    {
+      ProfScope ps(p, 1, stream);
+      const int grid = std::max(1, std::min(2 * p->sms, std::min(T, p->cfg.n_slots) * kMaxZSplits));
+      const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : 4 * p->sms;
+      launch_decode_shrink(ids_in, x, p->A_pool, p->slots_dev, plan->pv, p->zws, p->group_counters,
+                           T, h_in, R, p->cfg.n_slots, p->cfg.max_tokens, target, grid,
+                           p->status_dev, pdl_first, stream);
+      CUDA_TRY(cudaGetLastError());
+      ++launches;
+    }
     const int N = round_up(T, 32);
     const int row_tiles = (h_out + kTileM - 1) / kTileM;
-    int splits = std::max(1, std::min(p->sms / row_tiles, kb_total / 2));
-    int kb_per = (kb_total + splits - 1) / splits;
+    const int stage_bytes = kTileM * kBlockK * 2 + N * kBlockK * 2;
+    const int ctas_per_sm = (stage_bytes * 4 + 2048 <= static_cast<int>(kSmemBudget / 2)) ? 2 : 1;
+    int splits = p->opt_decode_splits > 0 ? p->opt_decode_splits
+                                          : std::max(1, (p->sms * ctas_per_sm) / row_tiles);
+    splits = std::max(1, std::min({splits, kMaxDecodeSplits, std::max(1, kb_total / 2)}));
+    const int kb_per = (kb_total + splits - 1) / splits;
     splits = (kb_total + kb_per - 1) / kb_per;
-    if (static_cast<size_t>(splits) * T * h_out > p->ws_floats) return EDGELORA_ERR_INVALID_ARG;
+    if (splits > 1 && static_cast<size_t>(splits) * T * h_out > p->ws_floats) return EDGELORA_ERR_INVALID_ARG;
     g.mode = kModeDecode;
     g.BN = N;
     g.splits = splits;
     g.kb_per = kb_per;
     g.n_mtiles = row_tiles;
     g.n_ntiles = 1;
-    g.stages = stages_for(N, kb_per);
+    g.zsplits = 1;   // the decode shrink leaves the summed z in the plane after the partial ones
+    g.zws = p->zws + static_cast<size_t>(kMaxZSplits) * p->cfg.max_tokens * R;
+    const size_t budget = ctas_per_sm == 2 ? kSmemBudget / 2 : kSmemBudget;
+    g.stages = stages_for(N, kb_per + 8, budget);
     g.n_acc = 1;
     g.tmem_cols = pow2_cols(N);
-    const CUtensorMap *mr, *mc;
+    const CUtensorMap *mr, *mc, *mb;
     int rc = get_tmap(p, &mr, W_dev, h_in, h_out, 0, kTileM);
     if (rc) return rc;
     rc = get_tmap(p, &mc, x, h_in, T, 0, N);
     if (rc) return rc;
+    rc = get_tmap(p, &mb, p->B_pool, R, h_out, p->cfg.n_slots, kTileM);
+    if (rc) return rc;
     const int grid = row_tiles * splits;
     {
       ProfScope ps(p, 3, stream);
-      CUDA_TRY(launch_gemm(*mr, *mc, g, grid, smem_for(g.stages, N), pdl, stream));
-      ++launches;
-    }
-    {
-      ProfScope ps(p, 4, stream);
-      launch_decode_combine(p->ws, splits, p->zws, zsplits, p->cfg.max_tokens, p->B_pool,
-                            p->slots_dev, plan->pv.ids_valid, g.y, T, h_out, R, pdl, stream);
-      CUDA_TRY(cudaGetLastError());
+      CUDA_TRY(launch_gemm(*mr, *mc, *mb, g, grid, smem_for(g.stages, N), pdl, stream));
       ++launches;
     }
     p->last_info[2] = grid;
     p->last_info[3] = splits;
   } else {
+    // ---------------------------------------------------------------- prefill
+    if (ids_dev) {
+      ProfScope ps(p, 0, stream);
+      plan->last_T = T;
+      launch_plan(ids_dev, T, plan->n_slots, plan->pv, pdl_first, stream);
+      CUDA_TRY(cudaGetLastError());
+      ++launches;
+    }
+    const bool sgmv = T > kDecodeMaxT;
+    // segment-shrink split-K factor (number of partial z planes the consumers sum)
+    int zsplits = 1;
+    if (sgmv) {
+      const int tiles_est = std::max(1, T / kTileM);
+      zsplits = std::max(1, std::min({8, p->sms / tiles_est, kb_total / 4}));
+      const int kb_per = (kb_total + zsplits - 1) / zsplits;
+      zsplits = (kb_total + kb_per - 1) / kb_per;
+    }
+    g.zsplits = zsplits;
+    {
+      ProfScope ps(p, 1, stream);
+      launch_bgmv_shrink(x, p->A_pool, p->slots_dev, plan->pv, p->zws, T, h_in, R, p->cfg.n_slots,
+                         zsplits, p->cfg.max_tokens, p->status_dev, ids_dev ? pdl : pdl_first, stream);
+      CUDA_TRY(cudaGetLastError());
+      ++launches;
+    }
+    const CUtensorMap *mx;
+    int rc = get_tmap(p, &mx, x, h_in, T, 0, kTileM);
+    if (rc) return rc;
+    if (sgmv) {
+      GemmParams s = g;
+      s.mode = kModeSgmv;
+      s.BN = R;
+      s.splits = zsplits;
+      s.kb_per = (kb_total + zsplits - 1) / zsplits;
+      s.stages = stages_for(R, s.kb_per, kSmemBudget);
+      s.n_acc = 2;
+      s.tmem_cols = pow2_cols(2 * R);
+      const CUtensorMap *mc;
+      rc = get_tmap(p, &mc, p->A_pool, h_in, R, p->cfg.n_slots, R);
+      if (rc) return rc;
+      const int grid = std::max(1, std::min(p->sms, plan->pv.max_sgmv_tiles * zsplits));
+      ProfScope ps(p, 2, stream);
+      CUDA_TRY(launch_gemm(*mx, *mc, *mc, s, grid, smem_for(s.stages, R), pdl, stream));
+      ++launches;
+    }
     const int n_mtiles = (T + kTileM - 1) / kTileM;
     const int tiles256 = n_mtiles * ((h_out + 255) / 256);
     int BN = (tiles256 >= p->sms || h_out <= 128) ? 256 : 128;
@@ -747,17 +790,17 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     g.kb_per = kb_total;
     g.n_mtiles = n_mtiles;
     g.n_ntiles = (h_out + BN - 1) / BN;
-    g.stages = stages_for(BN, kb_total);
+    g.stages = stages_for(BN, kb_total, kSmemBudget);
     g.n_acc = 2;
     g.tmem_cols = pow2_cols(2 * BN);
-    const CUtensorMap *mr, *mc;
-    int rc = get_tmap(p, &mr, x, h_in, T, 0, kTileM);
-    if (rc) return rc;
+    const CUtensorMap *mc, *mb;
     rc = get_tmap(p, &mc, W_dev, h_in, h_out, 0, BN);
+    if (rc) return rc;
+    rc = get_tmap(p, &mb, p->B_pool, R, h_out, p->cfg.n_slots, BN);
     if (rc) return rc;
     const int grid = std::min(p->sms, g.n_mtiles * g.n_ntiles);
     ProfScope ps(p, 3, stream);
-    CUDA_TRY(launch_gemm(*mr, *mc, g, grid, smem_for(g.stages, BN), pdl, stream));
+    CUDA_TRY(launch_gemm(*mx, *mc, *mb, g, grid, smem_for(g.stages, BN), pdl, stream));
     ++launches;
     p->last_info[2] = grid;
     p->last_info[3] = 1;
