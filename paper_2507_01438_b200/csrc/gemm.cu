@@ -14,8 +14,10 @@
 //            main loop of the next.  Epilogue: y = bf16(D).
 //   decode   R = 128 rows of W,    C = all tokens (N = T rounded up); LoRA blocks: R = B_a rows,
 //            C = masked z.  W is streamed once; K and the LoRA groups are split across CTAs so
-//            every SM pulls from HBM; fp32 partials go to a workspace and the CTA that arrives
-//            last at a row tile adds them in a fixed order and writes y.
+//            every SM pulls from HBM.  The K splits of one row tile form a thread-block cluster:
+//            after the main loop every CTA sends its fp32 partial tile, column block by column
+//            block, into the shared memory of the CTA that owns those tokens (distributed shared
+//            memory), and each owner adds the partials in a fixed order and writes its part of y.
 //   sgmv     R = 128 tokens of one run, C = A_a (N = rank stride): the segment shrink
 //            z = s_a A_a x for long runs, tile list from the plan.  No LoRA blocks.
 //
@@ -56,8 +58,8 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams &p, int32_t til
     c.split = 0;
     c.mtile = m;
   } else if (p.mode == kModeDecode) {
-    const int m = tile % p.n_mtiles;
-    c.split = tile / p.n_mtiles;
+    const int m = tile / p.splits;  // the splits of a row tile are consecutive CTAs: one cluster
+    c.split = tile - m * p.splits;
     c.row_r = m * kTileM;
     c.row_c = 0;
     c.mtile = m;
@@ -102,11 +104,65 @@ __device__ __forceinline__ LoraList lora_list(const GemmParams &p, const TileCoo
   return l;
 }
 
-__device__ __forceinline__ void named_bar_sync(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+// Barrier over every thread of every CTA of the cluster (a hardware barrier: all of them reach it,
+// on the time-out paths too, because no role loop is unbounded).
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
+// z of token t as packed bf16 (eight 16-byte chunks; chunks at or past the rank stride are zero):
+// the partial planes are added in order, values at or past the true rank forced to zero.
+__device__ __forceinline__ void load_z_packed(const GemmParams &p, int32_t t, int32_t rank,
+                                              uint4 (&out)[8]) {
+  const int nch = p.R_pad >> 3;
+  const float *zt = p.zws + static_cast<size_t>(t) * p.R_pad;
+  const size_t plane = static_cast<size_t>(p.max_tokens) * p.R_pad;
+#pragma unroll
+  for (int c0 = 0; c0 < 8; c0 += 4) {
+    float acc[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+    if (c0 < nch) {
+      for (int sp = 0; sp < p.zsplits; ++sp) {
+        const float4 *zp = reinterpret_cast<const float4 *>(zt + sp * plane) + 2 * c0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (c0 + c < nch) {
+            const float4 u = __ldcg(zp + 2 * c), w = __ldcg(zp + 2 * c + 1);
+            acc[c * 8 + 0] += u.x; acc[c * 8 + 1] += u.y; acc[c * 8 + 2] += u.z; acc[c * 8 + 3] += u.w;
+            acc[c * 8 + 4] += w.x; acc[c * 8 + 5] += w.y; acc[c * 8 + 6] += w.z; acc[c * 8 + 7] += w.w;
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+#define EL(i) (((c0 + c) * 8 + (i)) < rank ? acc[c * 8 + (i)] : 0.f)
+      out[c0 + c].x = ptx::pack_bf16x2(EL(0), EL(1));
+      out[c0 + c].y = ptx::pack_bf16x2(EL(2), EL(3));
+      out[c0 + c].z = ptx::pack_bf16x2(EL(4), EL(5));
+      out[c0 + c].w = ptx::pack_bf16x2(EL(6), EL(7));
+#undef EL
+    }
+  }
 }
 
 __global__ void __launch_bounds__(kGemmThreads, 2)
@@ -127,7 +183,6 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   uint64_t *tempty_bar = tfull_bar + 2;           // [2]       epilogue -> MMA
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(tempty_bar + 2);
   volatile uint32_t *abort_flag = tmem_slot + 1;
-  volatile uint32_t *last_flag = tmem_slot + 2;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const bool has_lora = p.mode != kModeSgmv;
@@ -147,7 +202,6 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       ptx::mbar_init(&tempty_bar[i], 4);  // one arrival per epilogue warp
     }
     *abort_flag = 0;
-    *last_flag = 0;
     ptx::fence_barrier_init();
   }
   if (warp == 1) {
@@ -303,8 +357,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int quad = warp & 3;                      // TMEM lanes [32*quad, 32*quad+32)
     const int row_in_tile = quad * 32 + lane;
-    const int etid = threadIdx.x - 64;              // 0..127
-    const bool reduce_here = p.mode == kModeDecode && p.splits > 1;
+    const bool clustered = p.mode == kModeDecode && p.splits > 1;
     ptx::pdl_wait_prior_grids();                    // earlier kernels may still read y / the workspace
     bool ok = true;
     int32_t it = 0;
@@ -320,8 +373,9 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       if (!got) {
         ok = false;
         *abort_flag = 1;
-        if (!reduce_here) break;
+        break;
       }
+      if (clustered) break;  // the accumulator is read after the cluster barrier below
       ptx::tc_fence_after_sync();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                              acc * static_cast<uint32_t>(p.BN);
@@ -356,23 +410,14 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
             }
           }
         } else if (p.mode == kModeDecode) {
-          // row = W row j, columns = tokens c0 + [0, 32)
+          // single K split: row = W row j, columns = tokens c0 + [0, 32), straight to y
           if (row < p.h_out) {
-            if (p.splits == 1) {
 #pragma unroll
-              for (int jj = 0; jj < 32; ++jj) {
-                const int t = c0 + jj;
-                if (t < p.T)
-                  p.y[static_cast<size_t>(t) * p.h_out + row] =
-                      static_cast<uint16_t>(ptx::pack_bf16x2(v[jj], 0.f) & 0xFFFFu);
-              }
-            } else {
-              float *base = p.ws + (static_cast<size_t>(tc.split) * p.T) * p.h_out + row;
-#pragma unroll
-              for (int jj = 0; jj < 32; ++jj) {
-                const int t = c0 + jj;
-                if (t < p.T) base[static_cast<size_t>(t) * p.h_out] = v[jj];
-              }
+            for (int jj = 0; jj < 32; ++jj) {
+              const int t = c0 + jj;
+              if (t < p.T)
+                p.y[static_cast<size_t>(t) * p.h_out + row] =
+                    static_cast<uint16_t>(ptx::pack_bf16x2(v[jj], 0.f) & 0xFFFFu);
             }
           }
         } else {
@@ -393,53 +438,6 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         if (lane == 0) ptx::mbar_arrive(&tempty_bar[acc]);
       }
 
-      if (reduce_here) {
-        // Split-K reduction by whichever CTA finishes this row tile last (it never waits).  All
-        // four warps pass the named barriers together even when a wait gave up, and leave the loop
-        // together afterwards.
-        __threadfence();
-        named_bar_sync(1, 128);
-        if (etid == 0) {
-          uint32_t last = 0;
-          if (!*abort_flag) {
-            const int old = atomicAdd(&p.tile_counters[tc.mtile], 1);
-            last = (old == p.splits - 1) ? 1u : 0u;
-            if (last) p.tile_counters[tc.mtile] = 0;  // ready for the next launch
-          }
-          *last_flag = last;
-        }
-        named_bar_sync(1, 128);
-        if (*last_flag) {
-          __threadfence();
-          // unit = (token, 4 adjacent W rows); all partials of a unit are loaded before any is used
-          const int n_units = p.T * 32;
-          const size_t plane = static_cast<size_t>(p.T) * p.h_out;
-          for (int u = etid; u < n_units; u += 128) {
-            const int t = u >> 5, j = tc.row_r + ((u & 31) << 2);
-            if (j >= p.h_out) continue;  // h_out is a multiple of 8: 4 rows are all in or all out
-            const float *src = p.ws + static_cast<size_t>(t) * p.h_out + j;
-            float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int sp0 = 0; sp0 < p.splits; sp0 += 8) {
-              float4 v[8];
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                v[i] = (sp0 + i < p.splits)
-                           ? __ldcg(reinterpret_cast<const float4 *>(src + (sp0 + i) * plane))
-                           : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                acc4.x += v[i].x; acc4.y += v[i].y; acc4.z += v[i].z; acc4.w += v[i].w;
-              }
-            }
-            uint2 o;
-            o.x = ptx::pack_bf16x2(acc4.x, acc4.y);
-            o.y = ptx::pack_bf16x2(acc4.z, acc4.w);
-            *reinterpret_cast<uint2 *>(p.y + static_cast<size_t>(t) * p.h_out + j) = o;
-          }
-        }
-        named_bar_sync(1, 128);  // last_flag is rewritten by the next tile
-        if (*abort_flag) ok = false;
-      }
     }
     if (!ok && lane == 0) {
       *abort_flag = 1;
@@ -451,7 +449,6 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     const int nch = p.R_pad >> 3;        // 16-byte chunks of one operand row that the MMAs read
     uint32_t count = 0;                  // K blocks so far: stage = count % stages
     uint32_t gophase = 0;                // one parity bit per stage for zgo_bar
-    const uint32_t zsplits = static_cast<uint32_t>(p.zsplits);
     bool ok = true, waited = false;
     for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
       const TileCoord tc = tile_coord(p, tile);
@@ -464,14 +461,19 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       const int rows = (p.mode == kModePrefill) ? kTileM : p.BN;
       const int tok0 = (p.mode == kModePrefill) ? tc.row_r : 0;
       const uint32_t region = (p.mode == kModePrefill) ? 0u : r_bytes;
-      // the ids of this thread's rows do not change over the tile's LoRA blocks
+      // The ids of this thread's rows do not change over the tile's LoRA blocks, so their z is
+      // fetched once per tile (while the base K blocks stream) and kept as packed bf16.
       int32_t id_lo = -1, id_hi = -1;
       if (tok0 + btid < p.T) id_lo = p.ids_valid[tok0 + btid];
       if (rows > 128 && tok0 + btid + 128 < p.T) id_hi = p.ids_valid[tok0 + btid + 128];
+      uint4 z_lo[8], z_hi[8];
+      if (ll.e0 < ll.e1) {
+        if (id_lo >= 0) load_z_packed(p, tok0 + btid, p.slots[id_lo].rank, z_lo);
+        if (id_hi >= 0) load_z_packed(p, tok0 + btid + 128, p.slots[id_hi].rank, z_hi);
+      }
       for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
         const int32_t a = ll.list[e];
-        const int32_t rank = p.slots[a].rank;
-        if (rank <= 0) continue;
+        if (p.slots[a].rank <= 0) continue;
         const uint32_t stage = count % nstages;
         ++count;
         if (!ptx::mbar_wait(&zgo_bar[stage], (gophase >> stage) & 1u) || *abort_flag) {
@@ -480,48 +482,24 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         }
         gophase ^= 1u << stage;
         uint8_t *dst = smem + static_cast<size_t>(stage) * stage_bytes + region;
-        for (int r = btid; r < rows; r += 128) {
-          const bool match = ((r < 128) ? id_lo : id_hi) == a;
-          uint8_t *drow = dst + r * 128;
-          if (!match) {
-            for (int c = 0; c < nch; ++c)
-              *reinterpret_cast<uint4 *>(drow + ((c ^ (r & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
-            continue;
-          }
-          // z of this token: sum the partial planes in order, four chunks of a plane in flight
-          const float *zt = p.zws + static_cast<size_t>(tok0 + r) * p.R_pad;
-          const size_t plane = static_cast<size_t>(p.max_tokens) * p.R_pad;
-          for (int c0 = 0; c0 < nch; c0 += 4) {
-            float acc[32];
+        // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
+        if (btid < rows) {
+          uint8_t *drow = dst + btid * 128;
+          const bool match = id_lo == a;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) acc[i] = 0.f;
-            for (uint32_t sp = 0; sp < zsplits; ++sp) {
-              const float4 *zp = reinterpret_cast<const float4 *>(zt + sp * plane) + 2 * c0;
+          for (int c = 0; c < 8; ++c)
+            if (c < nch)
+              *reinterpret_cast<uint4 *>(drow + ((c ^ (btid & 7)) << 4)) =
+                  match ? z_lo[c] : make_uint4(0u, 0u, 0u, 0u);
+        }
+        if (btid + 128 < rows) {
+          uint8_t *drow = dst + (btid + 128) * 128;
+          const bool match = id_hi == a;
 #pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                if (c0 + c < nch) {
-                  const float4 u = __ldcg(zp + 2 * c), w = __ldcg(zp + 2 * c + 1);
-                  acc[c * 8 + 0] += u.x; acc[c * 8 + 1] += u.y; acc[c * 8 + 2] += u.z; acc[c * 8 + 3] += u.w;
-                  acc[c * 8 + 4] += w.x; acc[c * 8 + 5] += w.y; acc[c * 8 + 6] += w.z; acc[c * 8 + 7] += w.w;
-                }
-              }
-            }
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              if (c0 + c < nch) {
-                uint4 o;
-                // values at or past the true rank are not defined by the shrink: force zero
-#define EL(i) (((c0 + c) * 8 + (i)) < rank ? acc[c * 8 + (i)] : 0.f)
-                o.x = ptx::pack_bf16x2(EL(0), EL(1));
-                o.y = ptx::pack_bf16x2(EL(2), EL(3));
-                o.z = ptx::pack_bf16x2(EL(4), EL(5));
-                o.w = ptx::pack_bf16x2(EL(6), EL(7));
-#undef EL
-                // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
-                *reinterpret_cast<uint4 *>(drow + (((c0 + c) ^ (r & 7)) << 4)) = o;
-              }
-            }
-          }
+          for (int c = 0; c < 8; ++c)
+            if (c < nch)
+              *reinterpret_cast<uint4 *>(drow + ((c ^ (btid & 7)) << 4)) =
+                  match ? z_hi[c] : make_uint4(0u, 0u, 0u, 0u);
         }
         fence_proxy_async_smem();  // make the generic-proxy writes visible to the tensor core
         __syncwarp();
@@ -531,6 +509,59 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     if (!ok && lane == 0) {
       *abort_flag = 1;
       atomicOr(p.status, EDGELORA_STATUS_TIMEOUT);
+    }
+  }
+
+  if (p.mode == kModeDecode && p.splits > 1) {
+    // ---------------------------------------------------------- split-K reduction in the cluster
+    // CTA `rank` of the cluster owns tokens [rank * cols_per, (rank + 1) * cols_per).  Its buffer
+    // buf[src split][token][row] overlays the operand ring, which is idle once every CTA of the
+    // cluster is past its main loop (first barrier).
+    const bool epi = warp >= 2 && warp < 6;
+    const int quad = warp & 3, row_in_tile = quad * 32 + lane, etid = threadIdx.x - 64;
+    const uint32_t my_rank = cluster_cta_rank();
+    const int cols_per = p.BN / p.splits;  // a power of two (BN and splits are)
+    const int shift = 31 - __clz(cols_per);
+    const bool have_acc = epi && !*abort_flag;  // this CTA's accumulator is complete (tfull waited)
+    __syncwarp();
+    cluster_sync_all();
+    if (have_acc) {
+      ptx::tc_fence_after_sync();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+      const uint32_t local = ptx::smem_u32(smem) +
+                             ((my_rank * cols_per) * kTileM + row_in_tile) * 4u;
+      for (int32_t c0 = 0; c0 < p.BN; c0 += 32) {
+        float v[32];
+        ptx::tmem_ld_32x32(taddr + c0, v);
+#pragma unroll
+        for (int jj = 0; jj < 32; ++jj) {
+          const int col = c0 + jj;
+          const uint32_t owner = static_cast<uint32_t>(col >> shift);
+          const uint32_t off = static_cast<uint32_t>(col & (cols_per - 1)) * kTileM * 4u;
+          st_cluster_f32(map_to_cta(local + off, owner), v[jj]);  // a warp writes 128 bytes in a row
+        }
+      }
+    }
+    __syncwarp();
+    cluster_sync_all();
+    if (epi) {
+      const float *buf = reinterpret_cast<const float *>(smem);
+      const int n_units = cols_per * 32;  // (token, 4 adjacent W rows)
+      for (int u = etid; u < n_units; u += 128) {
+        const int cl = u >> 5, r4 = (u & 31) << 2;
+        const int t = static_cast<int>(my_rank) * cols_per + cl;
+        const int j = blockIdx.x / p.splits * kTileM + r4;
+        if (t >= p.T || j >= p.h_out) continue;  // h_out is a multiple of 8: 4 rows are all in or out
+        float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sp = 0; sp < p.splits; ++sp) {
+          const float4 w = *reinterpret_cast<const float4 *>(buf + ((sp * cols_per + cl) * kTileM + r4));
+          acc4.x += w.x; acc4.y += w.y; acc4.z += w.z; acc4.w += w.w;
+        }
+        uint2 o;
+        o.x = ptx::pack_bf16x2(acc4.x, acc4.y);
+        o.y = ptx::pack_bf16x2(acc4.z, acc4.w);
+        *reinterpret_cast<uint2 *>(p.y + static_cast<size_t>(t) * p.h_out + j) = o;
+      }
     }
   }
 
@@ -550,7 +581,8 @@ cudaError_t gemm_set_smem_limit(size_t smem_bytes) {
 cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
                         const CUtensorMap &tmap_b, const GemmParams &p, int32_t grid,
                         size_t smem_bytes, bool pdl, cudaStream_t stream) {
-  return launch_ex(lora_gemm_kernel, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl,
+  const int cluster = (p.mode == kModeDecode && p.splits > 1) ? p.splits : 1;
+  return launch_ex(lora_gemm_kernel, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster,
                    tmap_row, tmap_col, tmap_b, p);
 }
 

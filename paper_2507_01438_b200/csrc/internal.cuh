@@ -72,13 +72,11 @@ struct GemmParams {
   const float *zws;         // [zsplits][max_tokens][R_pad]   (read by the prefill epilogue)
   float *zws_out;           // same buffer, written by the segment shrink
   uint16_t *y;              // [T][h_out]
-  float *ws;                // decode partials [splits][T][h_out]
   const int32_t *sgmv_tiles;
   const int32_t *counts;
   const int32_t *lg_adapter;  // decode: LoRA groups of the batch
   const int32_t *mt_count;    // prefill: per 128-token tile
   const int32_t *mt_list;
-  int32_t *tile_counters;     // decode: arrivals per W row tile (split-K reduction by the last one)
   uint32_t *status;
 };
 

@@ -1,5 +1,6 @@
 // Kernel launch helper: optional programmatic dependent launch (the next kernel's prologue may
-// overlap this kernel's tail; each kernel calls griddepcontrol.wait before its first global write).
+// overlap this kernel's tail; each kernel calls griddepcontrol.wait before its first global write)
+// and an optional thread-block cluster of `cluster` consecutive CTAs along x.
 #pragma once
 #include <cuda_runtime.h>
 
@@ -7,17 +8,24 @@ namespace edgelora {
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                             cudaStream_t stream, bool pdl, Args... args) {
+                             cudaStream_t stream, bool pdl, int cluster, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (cluster > 1) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = static_cast<unsigned>(cluster);
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 

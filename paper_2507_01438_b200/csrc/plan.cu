@@ -251,7 +251,7 @@ void launch_plan(const int32_t *ids, int32_t T, int32_t n_slots, const PlanView 
                  cudaStream_t stream) {
   int npow2 = 32;
   while (npow2 < T) npow2 <<= 1;
-  launch_ex(plan_kernel, dim3(1), dim3(kPlanThreads), static_cast<size_t>(npow2) * 4, stream, pdl,
+  launch_ex(plan_kernel, dim3(1), dim3(kPlanThreads), static_cast<size_t>(npow2) * 4, stream, pdl, 1,
             ids, T, n_slots, pv, npow2);
 }
 

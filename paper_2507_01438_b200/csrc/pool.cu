@@ -22,7 +22,7 @@ constexpr int kStagingBuffers = 4;
 constexpr int kTmapCache = 32;
 constexpr int kProfEvents = 8192;
 constexpr size_t kSmemBudget = 220 * 1024;
-constexpr int kMaxDecodeSplits = 32;
+constexpr int kMaxDecodeSplits = 8;  // K splits of a row tile form one (portable-size) cluster
 
 #define CUDA_TRY(expr)                                   \
   do {                                                   \
@@ -128,10 +128,9 @@ struct edgelora_pool {
   uint64_t load_seq = 0, load_seq_waited = 0;
   bool use_recorded = false;
   edgelora_plan *plan = nullptr;
-  float *zws = nullptr, *ws = nullptr;
-  int32_t *tile_counters = nullptr, *group_counters = nullptr;
+  float *zws = nullptr;
+  int32_t *group_counters = nullptr;
   int opt_decode_splits = 0, opt_shrink_items = 0;
-  size_t ws_floats = 0;
   uint32_t *status_dev = nullptr;
   std::vector<TmapEntry> tmaps;
   size_t tmap_next = 0;
@@ -413,15 +412,6 @@ int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool
   POOL_TRY(cudaMalloc(&p->zws, sizeof(float) * (kMaxZSplits + 1) * static_cast<size_t>(p->cfg.max_tokens) * p->R_pad));
   POOL_TRY(cudaMalloc(&p->group_counters, sizeof(int32_t) * kDecodeMaxT));
   POOL_TRY(cudaMemset(p->group_counters, 0, sizeof(int32_t) * kDecodeMaxT));
-  // decode partials: splits * T * h_out with splits <= sms / row_tiles + 1 and T <= 256
-  {
-    const int row_tiles = (cfg->h_out + kTileM - 1) / kTileM;
-    const int max_splits = std::min(kMaxDecodeSplits, std::max(1, 2 * p->sms / row_tiles) + 1);
-    p->ws_floats = static_cast<size_t>(max_splits) * kDecodeMaxT * cfg->h_out;
-    POOL_TRY(cudaMalloc(&p->ws, p->ws_floats * sizeof(float)));
-    POOL_TRY(cudaMalloc(&p->tile_counters, sizeof(int32_t) * row_tiles));
-    POOL_TRY(cudaMemset(p->tile_counters, 0, sizeof(int32_t) * row_tiles));
-  }
   POOL_TRY(gemm_set_smem_limit(kSmemBudget));
   rc = edgelora_plan_create(p->cfg.max_tokens, cfg->n_slots, &p->plan);
   if (rc != EDGELORA_OK) {
@@ -448,8 +438,6 @@ int edgelora_pool_destroy(edgelora_pool_t *p) {
   if (p->load_ev) cudaEventDestroy(p->load_ev);
   if (p->use_ev) cudaEventDestroy(p->use_ev);
   if (p->zws) cudaFree(p->zws);
-  if (p->ws) cudaFree(p->ws);
-  if (p->tile_counters) cudaFree(p->tile_counters);
   if (p->group_counters) cudaFree(p->group_counters);
   for (auto &r : p->prof) {
     cudaEventDestroy(r.start);
@@ -661,13 +649,11 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
   g.zws = p->zws;
   g.zws_out = p->zws;
   g.y = static_cast<uint16_t *>(y_dev);
-  g.ws = p->ws;
   g.sgmv_tiles = plan->pv.sgmv_tiles;
   g.counts = plan->pv.counts;
   g.lg_adapter = plan->pv.lg_adapter;
   g.mt_count = plan->pv.mt_count;
   g.mt_list = plan->pv.mt_list;
-  g.tile_counters = p->tile_counters;
   g.status = p->status_dev;
 
   auto smem_for = [](int stages, int BN) {
@@ -697,16 +683,21 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
       CUDA_TRY(cudaGetLastError());
       ++launches;
     }
-    const int N = round_up(T, 32);
+    int N = 32;  // tokens on the UMMA N axis: a power of two so that the cluster's owners get
+    while (N < T) N <<= 1;  // equal power-of-two column blocks
     const int row_tiles = (h_out + kTileM - 1) / kTileM;
     const int stage_bytes = kTileM * kBlockK * 2 + N * kBlockK * 2;
     const int ctas_per_sm = (stage_bytes * 4 + 2048 <= static_cast<int>(kSmemBudget / 2)) ? 2 : 1;
-    int splits = p->opt_decode_splits > 0 ? p->opt_decode_splits
-                                          : std::max(1, (p->sms * ctas_per_sm) / row_tiles);
-    splits = std::max(1, std::min({splits, kMaxDecodeSplits, std::max(1, kb_total / 2)}));
-    const int kb_per = (kb_total + splits - 1) / splits;
-    splits = (kb_total + kb_per - 1) / kb_per;
-    if (splits > 1 && static_cast<size_t>(splits) * T * h_out > p->ws_floats) return EDGELORA_ERR_INVALID_ARG;
+    int want = p->opt_decode_splits > 0 ? p->opt_decode_splits
+                                        : std::max(1, (p->sms * ctas_per_sm) / row_tiles);
+    want = std::min({want, kMaxDecodeSplits, std::max(1, kb_total / 2)});
+    int splits = 1;
+    while (splits * 2 <= want) splits <<= 1;
+    int kb_per = (kb_total + splits - 1) / splits;
+    while (splits > 1 && kb_per * (splits - 1) >= kb_total) {  // every split needs a K block
+      splits >>= 1;
+      kb_per = (kb_total + splits - 1) / splits;
+    }
     g.mode = kModeDecode;
     g.BN = N;
     g.splits = splits;
@@ -717,6 +708,8 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     g.zws = p->zws + static_cast<size_t>(kMaxZSplits) * p->cfg.max_tokens * R;
     const size_t budget = ctas_per_sm == 2 ? kSmemBudget / 2 : kSmemBudget;
     g.stages = stages_for(N, kb_per + 8, budget);
+    // the cluster's reduction buffer (N x 128 fp32) overlays the operand ring
+    while (splits > 1 && g.stages * stage_bytes < N * kTileM * 4 && g.stages < kMaxStages) ++g.stages;
     g.n_acc = 1;
     g.tmem_cols = pow2_cols(N);
     const CUtensorMap *mr, *mc, *mb;

@@ -105,7 +105,7 @@ void launch_bgmv_shrink(const uint16_t *x, const uint16_t *A_pool, const SlotRow
                         int32_t n_slots, int32_t zsplits, int32_t max_tokens, uint32_t *status,
                         bool pdl, cudaStream_t stream) {
   const int max_groups = (T < n_slots + 1) ? T : n_slots + 1;
-  launch_ex(bgmv_shrink_kernel, dim3(max_groups * R_pad), dim3(kBgmvThreads), 0, stream, pdl, x,
+  launch_ex(bgmv_shrink_kernel, dim3(max_groups * R_pad), dim3(kBgmvThreads), 0, stream, pdl, 1, x,
             A_pool, slots, pv, zws, T, h_in, R_pad, zsplits, max_tokens, status);
 }
 
@@ -417,7 +417,7 @@ void launch_decode_shrink(const int32_t *ids, const uint16_t *x, const uint16_t 
                           int32_t *group_counters, int32_t T, int32_t h_in, int32_t R_pad,
                           int32_t n_slots, int32_t max_tokens, int32_t target_items, int32_t grid,
                           uint32_t *status, bool pdl, cudaStream_t stream) {
-  launch_ex(decode_shrink_kernel, dim3(grid), dim3(kShrinkThreads), 0, stream, pdl, ids, x, A_pool,
+  launch_ex(decode_shrink_kernel, dim3(grid), dim3(kShrinkThreads), 0, stream, pdl, 1, ids, x, A_pool,
             slots, pv, zws, group_counters, T, h_in, R_pad, n_slots, max_tokens, target_items, status);
 }
 
