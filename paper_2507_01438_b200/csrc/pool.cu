@@ -675,7 +675,7 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     plan->last_T = T;
     {
       ProfScope ps(p, 1, stream);
-      const int grid = std::max(1, std::min(2 * p->sms, std::min(T, p->cfg.n_slots) * kMaxZSplits));
+      const int grid = std::max(1, std::min(p->sms, std::min(T, p->cfg.n_slots) * kMaxZSplits));
       const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : 4 * p->sms;
       launch_decode_shrink(ids_in, x, p->A_pool, p->slots_dev, plan->pv, p->zws, p->group_counters,
                            T, h_in, R, p->cfg.n_slots, p->cfg.max_tokens, target, grid,

@@ -119,8 +119,10 @@ namespace edgelora {
 // A decode step is a few microseconds long, so a separate routing launch would cost as much as
 // the arithmetic.  Here every CTA derives the u-batches (paper Section 3.4) from the ids itself, in
 // shared memory, and then takes its share of the work items (group, K chunk).  An item streams the
-// live rows of A_a over its K chunk once from HBM with 128-bit loads, eight rows in flight per
-// lane, and dots them with the x rows of up to four tokens of the group at a time; lanes are
+// live rows of A_a over its K chunk once from HBM with 16-byte cp.async copies into a private
+// shared-memory ring (two K steps of eight rows ahead per lane), and dots them with the x rows of
+// up to four tokens of the group at a time (a group's tokens are cut into blocks of eight, each
+// block an item of its own, so that a popular adapter does not serialise on one CTA); lanes are
 // reduced by shuffles, K sub-ranges of one item by a small shared-memory stage.  Partial sums go
 // to zws[chunk][token][row]; whichever item finishes a group last adds the chunks in a fixed
 // order into the final plane zws[kMaxZSplits] that the base-product kernel reads.  The last CTA also
@@ -164,34 +166,71 @@ __device__ __forceinline__ int block_scan_256(int v, int *wt /* smem[9] */, int 
   return res;
 }
 
-// Eight rows of A against NT token rows of x over the K steps [step0, step1) with stride `dstep`;
-// one K step is 256 elements, lane l owns elements [8 l, 8 l + 8) of it.
-template <int NT>
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_u32(smem_dst)), "l"(gmem_src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+constexpr int kRingSlots = 8 + kDsTok;  // 16-byte slots of one lane in one ring stage: 8 A rows + x rows
+
+// Eight rows of A against NT token rows of x over the K steps step0, step0 + dstep, ... < step1;
+// one K step is 256 elements, lane l owns elements [8 l, 8 l + 8) of it.  Every lane prefetches
+// its own operands DEPTH - 1 steps ahead into its private slots of a shared-memory ring with
+// cp.async, so that many 16-byte requests per lane are in flight without holding registers.
+template <int NT, int DEPTH>
 __device__ __forceinline__ void shrink_rows8(const uint4 *__restrict__ A0, size_t row_u4,
                                              const uint4 *const (&xr)[kDsTok], int step0, int step1,
-                                             int dstep, int n_u4, int lane, float (&acc)[8 * kDsTok]) {
-#pragma unroll 2
+                                             int dstep, int n_u4, int lane, uint4 *ring /* this thread's slot 0 */,
+                                             float (&acc)[8 * kDsTok]) {
+  constexpr int kStageStride = kRingSlots * kShrinkThreads;  // uint4 between stages
+  auto issue = [&](int step, int stage) {
+    const int k = step * 32 + lane;
+    if (step < step1 && k < n_u4) {
+      uint4 *dst = ring + stage * kStageStride;
+#pragma unroll
+      for (int r = 0; r < 8; ++r) cp_async16(dst + r * kShrinkThreads, A0 + r * row_u4 + k);
+#pragma unroll
+      for (int q = 0; q < NT; ++q) cp_async16(dst + (8 + q) * kShrinkThreads, xr[q] + k);
+    }
+    cp_async_commit();  // an empty group keeps the group count uniform
+  };
+#pragma unroll
+  for (int d = 0; d < DEPTH - 1; ++d) issue(step0 + d * dstep, d);
+  int stage = 0;
   for (int step = step0; step < step1; step += dstep) {
+    int pre = stage + DEPTH - 1;
+    if (pre >= DEPTH) pre -= DEPTH;
+    issue(step + (DEPTH - 1) * dstep, pre);
+    cp_async_wait<DEPTH - 1>();
     const int k = step * 32 + lane;
     if (k < n_u4) {
-      uint4 av[8];
-#pragma unroll
-      for (int r = 0; r < 8; ++r) av[r] = __ldg(A0 + r * row_u4 + k);
+      const uint4 *src = ring + stage * kStageStride;
       float xf[NT][8];
 #pragma unroll
-      for (int q = 0; q < NT; ++q) unpack8(__ldg(xr[q] + k), xf[q]);
+      for (int q = 0; q < NT; ++q) unpack8(src[(8 + q) * kShrinkThreads], xf[q]);
 #pragma unroll
       for (int r = 0; r < 8; ++r) {
         float af[8];
-        unpack8(av[r], af);
+        unpack8(src[r * kShrinkThreads], af);
 #pragma unroll
         for (int q = 0; q < NT; ++q)
 #pragma unroll
           for (int e = 0; e < 8; ++e) acc[r * kDsTok + q] = fmaf(af[e], xf[q][e], acc[r * kDsTok + q]);
       }
     }
+    if (++stage == DEPTH) stage = 0;
   }
+  cp_async_wait<0>();
 }
+
+constexpr int kDsDepth = 3;      // ring stages
+constexpr int kDsBlockTok = 8;   // tokens of one group handled by one work item (two passes of four)
+constexpr size_t kDsRingBytes = static_cast<size_t>(kDsDepth) * kRingSlots * kShrinkThreads * 16;
 
 __global__ void __launch_bounds__(kShrinkThreads)
 decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict__ x,
@@ -199,12 +238,15 @@ decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict
                      PlanView pv, float *__restrict__ zws, int32_t *__restrict__ group_counters,
                      int32_t T, int32_t h_in, int32_t R_pad, int32_t n_slots, int32_t max_tokens,
                      int32_t target_items, uint32_t *status) {
+  extern __shared__ uint4 s_ring[];    // [depth][slot][thread]
   __shared__ int32_t s_id[256];        // validated id of each token
   __shared__ int32_t s_grp[256];       // group (in order of first appearance) of a group's first token
   __shared__ int32_t s_gadapter[256];  // adapter of each group
   __shared__ int32_t s_gstart[257];    // token list boundaries
   __shared__ int32_t s_gtok[256];      // tokens ordered by (group, token)
   __shared__ int32_t s_cnt[256];
+  __shared__ int32_t s_bgrp[256];      // token blocks: group and first position in s_gtok
+  __shared__ int32_t s_btok[256];
   __shared__ int s_wt[9];
   __shared__ float s_red[8][32];
   __shared__ int s_last;
@@ -249,17 +291,29 @@ decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict
   }
   __syncthreads();
   int tot;
-  const int gs = block_scan_256(tid < G ? s_cnt[tid] : 0, s_wt, tot);
+  const int n_mine = tid < G ? s_cnt[tid] : 0;
+  const int gs = block_scan_256(n_mine, s_wt, tot);
   if (tid < G) s_gstart[tid] = gs;
   if (tid == 0) s_gstart[G] = tot;
+  // token blocks of at most kDsBlockTok tokens
+  const int nb_mine = (n_mine + kDsBlockTok - 1) / kDsBlockTok;
+  int NB;
+  const int b0 = block_scan_256(nb_mine, s_wt, NB);
+  for (int b = 0; b < nb_mine; ++b) {
+    s_bgrp[b0 + b] = tid;
+    s_btok[b0 + b] = gs + b * kDsBlockTok;
+  }
   __syncthreads();
   if (mygrp >= 0) s_gtok[s_gstart[mygrp] + pos] = tid;
   const int any_bad = __syncthreads_or(bad ? 1 : 0);
 
-  // K chunks: enough items to occupy the machine, each at least one K step per warp sub-range
+  // K chunks: enough items to occupy the machine, but an item keeps at least about 128 KB of A
+  // (below that the extra pass that adds the chunks costs more than it saves) and one K step per
+  // warp sub-range.
   const int n_ksteps = (h_in + 255) >> 8;
   const int ksubs_nominal = 64 / R_pad;  // 4, 2, 1 for a rank stride of 16, 32, 64
-  int KS = (target_items + max(G, 1) - 1) / max(G, 1);
+  int KS = (target_items + max(NB, 1) - 1) / max(NB, 1);
+  KS = min(KS, max(1, (R_pad * h_in * 2) >> 17));
   KS = max(1, min(min(KS, kMaxZSplits), n_ksteps / ksubs_nominal));
   const int spc = (n_ksteps + KS - 1) / KS;
   KS = (n_ksteps + spc - 1) / spc;
@@ -321,16 +375,20 @@ decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict
     }
   }
 
-  // ---- work items (group, K chunk)
-  const int n_items = G * KS;
+  // ---- work items (token block of a group, K chunk)
+  const int n_items = NB * KS;
   const int n_u4 = h_in >> 3;
   const size_t zplane = static_cast<size_t>(max_tokens) * R_pad;
+  uint4 *my_ring = s_ring + tid;
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const int gi = item / KS, c = item - gi * KS;
+    const int bi = item / KS, c = item - bi * KS;
+    const int gi = s_bgrp[bi];
     const int ad = s_gadapter[gi];
     const SlotRow row = slots[ad];
+    const int t0 = s_btok[bi], g_end = s_gstart[gi + 1];
+    const int t1 = min(t0 + kDsBlockTok, g_end);
     if (row.rank <= 0) {
-      if (tid == 0 && c == 0) atomicOr(status, EDGELORA_STATUS_SLOT_EMPTY);
+      if (tid == 0 && c == 0 && t0 == s_gstart[gi]) atomicOr(status, EDGELORA_STATUS_SLOT_EMPTY);
       continue;
     }
     const int n_rg = (row.rank + 7) >> 3;  // live groups of eight rows
@@ -339,7 +397,6 @@ decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict
     const int ksubs = 8 / rg_p2;
     const int rg = warp % rg_p2, ksub = warp / rg_p2;
     const int step0 = c * spc, step1 = min(n_ksteps, step0 + spc);
-    const int t0 = s_gstart[gi], t1 = s_gstart[gi + 1];
     const uint4 *A0 =
         reinterpret_cast<const uint4 *>(A_pool + (static_cast<size_t>(ad) * R_pad + rg * 8) * h_in);
     for (int tb = t0; tb < t1; tb += kDsTok) {
@@ -353,10 +410,10 @@ decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict
         for (int q = 0; q < kDsTok; ++q)
           xr[q] = reinterpret_cast<const uint4 *>(x + static_cast<size_t>(s_gtok[tb + min(q, nt - 1)]) * h_in);
         const size_t row_u4 = static_cast<size_t>(n_u4);
-        if (nt == 1) shrink_rows8<1>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, acc);
-        else if (nt == 2) shrink_rows8<2>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, acc);
-        else if (nt == 3) shrink_rows8<3>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, acc);
-        else shrink_rows8<4>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, acc);
+        if (nt == 1) shrink_rows8<1, kDsDepth>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, my_ring, acc);
+        else if (nt == 2) shrink_rows8<2, kDsDepth>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, my_ring, acc);
+        else if (nt == 3) shrink_rows8<3, kDsDepth>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, my_ring, acc);
+        else shrink_rows8<4, kDsDepth>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, my_ring, acc);
       }
       // lane L ends with the sum over lanes of value L (= row L / 4, token L % 4)
 #pragma unroll
@@ -385,20 +442,22 @@ decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict
     if (KS > 1) {
       // The item that completes a group adds the K chunks in order into the final plane (it never
       // waits for the others).
+      const int gt0 = s_gstart[gi];
+      const int arrivals = KS * ((g_end - gt0 + kDsBlockTok - 1) / kDsBlockTok);
       __threadfence();
       __syncthreads();
       if (tid == 0) {
         const int old = atomicAdd(&group_counters[gi], 1);
-        s_last = (old == KS - 1) ? 1 : 0;
+        s_last = (old == arrivals - 1) ? 1 : 0;
         if (s_last) group_counters[gi] = 0;  // ready for the next launch
       }
       __syncthreads();
       if (s_last) {
         __threadfence();
         const int live = n_rg * 8;
-        for (int idx = tid; idx < (t1 - t0) * live; idx += kShrinkThreads) {
+        for (int idx = tid; idx < (g_end - gt0) * live; idx += kShrinkThreads) {
           const int q = idx / live, r = idx - q * live;
-          const size_t off = static_cast<size_t>(s_gtok[t0 + q]) * R_pad + r;
+          const size_t off = static_cast<size_t>(s_gtok[gt0 + q]) * R_pad + r;
           float part[kMaxZSplits];
 #pragma unroll
           for (int sp = 0; sp < kMaxZSplits; ++sp) part[sp] = sp < KS ? __ldcg(zws + sp * zplane + off) : 0.f;
@@ -417,7 +476,13 @@ void launch_decode_shrink(const int32_t *ids, const uint16_t *x, const uint16_t 
                           int32_t *group_counters, int32_t T, int32_t h_in, int32_t R_pad,
                           int32_t n_slots, int32_t max_tokens, int32_t target_items, int32_t grid,
                           uint32_t *status, bool pdl, cudaStream_t stream) {
-  launch_ex(decode_shrink_kernel, dim3(grid), dim3(kShrinkThreads), 0, stream, pdl, 1, ids, x, A_pool,
+  static bool configured = false;  // per process; the attribute is per function and device-wide
+  if (!configured) {
+    cudaFuncSetAttribute(decode_shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         static_cast<int>(kDsRingBytes));
+    configured = true;
+  }
+  launch_ex(decode_shrink_kernel, dim3(grid), dim3(kShrinkThreads), kDsRingBytes, stream, pdl, 1, ids, x, A_pool,
             slots, pv, zws, group_counters, T, h_in, R_pad, n_slots, max_tokens, target_items, status);
 }
 
