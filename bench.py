@@ -40,6 +40,9 @@ WORKLOADS = {
     "down_proj_many_tenant": (lambda: wl.down_proj_many_tenant(), "hbm",
                               "configs[3]: down_proj 14336->4096, 1000 adapters r64, T=256 Zipf(1.1), 10% base-only"),
     "tiny": (lambda: wl.tiny(), "hbm", "configs[0]: 256->256, 4 adapters r8, T=16"),
+    # smaller resident pool, same layer and batch recipe: sized for multi-pass ncu captures
+    "down_proj_200_tenants": (lambda: wl.down_proj_many_tenant(n_adapters=200), "hbm",
+                              "profiling-size variant of configs[3]: down_proj 14336->4096, 200 adapters r64, T=256"),
 }
 
 
@@ -181,6 +184,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of CUDA-graph replay")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--pdl", type=int, default=None, help="EDGELORA_OPT_PDL value (0, 1, 2); default: library default")
+    ap.add_argument("--decode-splits", type=int, default=0, help="tuning: EDGELORA_OPT_DECODE_SPLITS")
+    ap.add_argument("--shrink-items", type=int, default=0, help="tuning: EDGELORA_OPT_SHRINK_ITEMS")
     args = ap.parse_args()
 
     builder, bound, desc = WORKLOADS[args.workload]
@@ -220,6 +226,12 @@ def main():
         Ws.append(to_bf16(w.W) if r == 0 else Ws[0].clone())
         pool = B.Pool(w.h_in, w.h_out, w.n_slots, w.max_rank, max_tokens=w.T)
         pool.load_all(w.adapters)
+        if args.pdl is not None:
+            B.edgelora_pool_set_option(pool.handle, B.OPT_PDL, args.pdl)
+        if args.decode_splits:
+            B.edgelora_pool_set_option(pool.handle, B.OPT_DECODE_SPLITS, args.decode_splits)
+        if args.shrink_items:
+            B.edgelora_pool_set_option(pool.handle, B.OPT_SHRINK_ITEMS, args.shrink_items)
         pools.append(pool)
     x = to_bf16(w.x)
     ids = torch.from_numpy(w.ids).cuda()

@@ -18,6 +18,7 @@ constexpr int kMaxTokensLimit = 32768;
 constexpr int kGemmThreads = 320;  // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue, warps 6..9 z operand
 constexpr int kMaxZSplits = 16;    // partial z planes (K splits of the shrink); plane 16 = summed z
 constexpr int kShrinkThreads = 256;
+constexpr int kShrinkStepElems = 256;  // K elements of one shrink step (512 bytes of a row)
 
 // One row of the slot table (paper Section 3.3: one fixed block per resident adapter).
 struct SlotRow {
@@ -92,10 +93,11 @@ cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col
                         const CUtensorMap &tmap_b, const GemmParams &p, int32_t grid,
                         size_t smem_bytes, bool pdl, cudaStream_t stream);
 cudaError_t gemm_set_smem_limit(size_t smem_bytes);
-void launch_decode_shrink(const int32_t *ids, const uint16_t *x, const uint16_t *A_pool,
-                          const SlotRow *slots, const PlanView &pv, float *zws,
-                          int32_t *group_counters, int32_t T, int32_t h_in, int32_t R_pad,
-                          int32_t n_slots, int32_t max_tokens, int32_t target_items, int32_t grid,
-                          uint32_t *status, bool pdl, cudaStream_t stream);
+cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &tmap_x,
+                                 const int32_t *ids, const SlotRow *slots, const PlanView &pv,
+                                 float *zws, int32_t *group_counters, int32_t T, int32_t h_in,
+                                 int32_t R_pad, int32_t n_slots, int32_t max_tokens,
+                                 int32_t target_items, int32_t grid, uint32_t *status, bool pdl,
+                                 cudaStream_t stream);
 
 }  // namespace edgelora

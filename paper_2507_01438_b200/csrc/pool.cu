@@ -62,9 +62,9 @@ EncodeTiledFn get_encode_fn() {
 struct TmapKey {
   const void *base;
   uint64_t d0, d1, d2;
-  uint32_t b1;
+  uint32_t b1, b0;  // box rows, box columns (64 => 128-byte swizzle, otherwise no swizzle)
   bool operator==(const TmapKey &o) const {
-    return base == o.base && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && b1 == o.b1;
+    return base == o.base && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && b1 == o.b1 && b0 == o.b0;
   }
 };
 struct TmapEntry {
@@ -72,19 +72,21 @@ struct TmapEntry {
   CUtensorMap map;
 };
 
-// bf16 row-major [d2][d1][d0] (d2 == 0 => 2D), box = {64, box_rows, 1}, 128-byte swizzle,
-// out-of-range elements read as zero.
+// bf16 row-major [d2][d1][d0] (d2 == 0 => 2D), box = {box_cols, box_rows, 1}; out-of-range
+// elements read as zero.  box_cols == 64: the 128-byte-swizzled operand tiles of the GEMM;
+// otherwise (the shrink's row segments) no swizzle.
 int encode_tmap(CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1, uint64_t d2,
-                uint32_t box_rows) {
+                uint32_t box_rows, uint32_t box_cols) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return EDGELORA_ERR_CUDA;
   const cuuint32_t rank = d2 ? 3 : 2;
   cuuint64_t dims[3] = {d0, d1, d2 ? d2 : 1};
   cuuint64_t strides[2] = {d0 * 2, d0 * d1 * 2};
-  cuuint32_t box[3] = {static_cast<cuuint32_t>(kBlockK), box_rows, 1};
+  cuuint32_t box[3] = {box_cols, box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), dims,
-                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  box_cols == static_cast<uint32_t>(kBlockK) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     snprintf(g_last_error, sizeof g_last_error, "cuTensorMapEncodeTiled failed (%d)", (int)r);
@@ -150,8 +152,8 @@ struct edgelora_pool {
 namespace {
 
 int get_tmap(edgelora_pool *p, const CUtensorMap **out, const void *base, uint64_t d0, uint64_t d1,
-             uint64_t d2, uint32_t box_rows) {
-  TmapKey key{base, d0, d1, d2, box_rows};
+             uint64_t d2, uint32_t box_rows, uint32_t box_cols = kBlockK) {
+  TmapKey key{base, d0, d1, d2, box_rows, box_cols};
   for (auto &e : p->tmaps)
     if (e.key == key) {
       *out = &e.map;
@@ -159,7 +161,7 @@ int get_tmap(edgelora_pool *p, const CUtensorMap **out, const void *base, uint64
     }
   TmapEntry e;
   e.key = key;
-  int rc = encode_tmap(&e.map, base, d0, d1, d2, box_rows);
+  int rc = encode_tmap(&e.map, base, d0, d1, d2, box_rows, box_cols);
   if (rc != EDGELORA_OK) return rc;
   if (p->tmaps.size() < static_cast<size_t>(kTmapCache)) {
     p->tmaps.push_back(e);
@@ -410,8 +412,8 @@ int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool
   POOL_TRY(cudaEventCreateWithFlags(&p->use_ev, cudaEventDisableTiming));
   // partial planes [0, kMaxZSplits) plus the final plane of the decode shrink
   POOL_TRY(cudaMalloc(&p->zws, sizeof(float) * (kMaxZSplits + 1) * static_cast<size_t>(p->cfg.max_tokens) * p->R_pad));
-  POOL_TRY(cudaMalloc(&p->group_counters, sizeof(int32_t) * kDecodeMaxT));
-  POOL_TRY(cudaMemset(p->group_counters, 0, sizeof(int32_t) * kDecodeMaxT));
+  POOL_TRY(cudaMalloc(&p->group_counters, sizeof(int32_t) * (kDecodeMaxT * 8 + 32)));
+  POOL_TRY(cudaMemset(p->group_counters, 0, sizeof(int32_t) * (kDecodeMaxT * 8 + 32)));
   POOL_TRY(gemm_set_smem_limit(kSmemBudget));
   rc = edgelora_plan_create(p->cfg.max_tokens, cfg->n_slots, &p->plan);
   if (rc != EDGELORA_OK) {
@@ -676,11 +678,15 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     {
       ProfScope ps(p, 1, stream);
       const int grid = std::max(1, std::min(p->sms, std::min(T, p->cfg.n_slots) * kMaxZSplits));
-      const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : 4 * p->sms;
-      launch_decode_shrink(ids_in, x, p->A_pool, p->slots_dev, plan->pv, p->zws, p->group_counters,
-                           T, h_in, R, p->cfg.n_slots, p->cfg.max_tokens, target, grid,
-                           p->status_dev, pdl_first, stream);
-      CUDA_TRY(cudaGetLastError());
+      const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : 4 * 8 * p->sms;  // warp items
+      const CUtensorMap *ma, *mx;
+      int rc = get_tmap(p, &ma, p->A_pool, h_in, R, p->cfg.n_slots, 8, kShrinkStepElems);
+      if (rc) return rc;
+      rc = get_tmap(p, &mx, x, h_in, T, 0, 1, kShrinkStepElems);
+      if (rc) return rc;
+      CUDA_TRY(launch_decode_shrink(*ma, *mx, ids_in, p->slots_dev, plan->pv, p->zws, p->group_counters,
+                                    T, h_in, R, p->cfg.n_slots, p->cfg.max_tokens, target, grid,
+                                    p->status_dev, pdl_first, stream));
       ++launches;
     }
     int N = 32;  // tokens on the UMMA N axis: a power of two so that the cluster's owners get
@@ -722,7 +728,10 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     const int grid = row_tiles * splits;
     {
       ProfScope ps(p, 3, stream);
-      CUDA_TRY(launch_gemm(*mr, *mc, *mb, g, grid, smem_for(g.stages, N), pdl, stream));
+      // With one CTA per SM the base product cannot start beside the shrink (both fill an SM's
+      // shared memory), and an early launch then only costs: measured 178 vs 122 us per step on
+      // the 14336 -> 4096, T = 256 workload.
+      CUDA_TRY(launch_gemm(*mr, *mc, *mb, g, grid, smem_for(g.stages, N), pdl && ctas_per_sm == 2, stream));
       ++launches;
     }
     p->last_info[2] = grid;

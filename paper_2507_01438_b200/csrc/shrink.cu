@@ -119,13 +119,14 @@ namespace edgelora {
 // A decode step is a few microseconds long, so a separate routing launch would cost as much as
 // the arithmetic.  Here every CTA derives the u-batches (paper Section 3.4) from the ids itself, in
 // shared memory, and then takes its share of the work items (group, K chunk).  An item streams the
-// live rows of A_a over its K chunk once from HBM with 16-byte cp.async copies into a private
-// shared-memory ring (two K steps of eight rows ahead per lane), and dots them with the x rows of
+// live rows of A_a over its K chunk once from HBM with TMA copies into a private shared-memory
+// ring (three K steps of eight rows ahead per warp), and dots them with the x rows of
 // up to four tokens of the group at a time (a group's tokens are cut into blocks of eight, each
 // block an item of its own, so that a popular adapter does not serialise on one CTA); lanes are
-// reduced by shuffles, K sub-ranges of one item by a small shared-memory stage.  Partial sums go
-// to zws[chunk][token][row]; whichever item finishes a group last adds the chunks in a fixed
-// order into the final plane zws[kMaxZSplits] that the base-product kernel reads.  The last CTA also
+// reduced by shuffles.  Items belong to single warps, which run independently so that the fixed
+// latencies of one overlap the streaming of the others.  Partial sums go to
+// zws[chunk][token][row]; whichever warp finishes a (group, eight rows) last adds the chunks in a
+// fixed order into the final plane zws[kMaxZSplits] that the base-product kernel reads.  The last CTA also
 // writes the routing plan in its canonical form for the base-product kernel and for export.
 
 constexpr int kDsTok = 4;
@@ -166,79 +167,74 @@ __device__ __forceinline__ int block_scan_256(int v, int *wt /* smem[9] */, int 
   return res;
 }
 
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_u32(smem_dst)), "l"(gmem_src)
-               : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
+constexpr int kDsDepth = 4;                         // ring stages per warp
+constexpr int kDsRowBytes = kShrinkStepElems * 2;   // 512: one row segment of one K step
+constexpr int kDsStageBytes = (8 + kDsTok) * kDsRowBytes;  // 8 rows of A, then up to 4 rows of x
 
-constexpr int kRingSlots = 8 + kDsTok;  // 16-byte slots of one lane in one ring stage: 8 A rows + x rows
-
-// Eight rows of A against NT token rows of x over the K steps step0, step0 + dstep, ... < step1;
-// one K step is 256 elements, lane l owns elements [8 l, 8 l + 8) of it.  Every lane prefetches
-// its own operands DEPTH - 1 steps ahead into its private slots of a shared-memory ring with
-// cp.async, so that many 16-byte requests per lane are in flight without holding registers.
-template <int NT, int DEPTH>
-__device__ __forceinline__ void shrink_rows8(const uint4 *__restrict__ A0, size_t row_u4,
-                                             const uint4 *const (&xr)[kDsTok], int step0, int step1,
-                                             int dstep, int n_u4, int lane, uint4 *ring /* this thread's slot 0 */,
-                                             float (&acc)[8 * kDsTok]) {
-  constexpr int kStageStride = kRingSlots * kShrinkThreads;  // uint4 between stages
+// Eight rows of A against NT token rows of x over the K steps [step0, step1).  One K step is 256
+// elements; lane l owns elements [8 l, 8 l + 8) of it.  The warp's lane 0 keeps kDsDepth - 1 steps
+// in flight with TMA copies (one box of 8 x 512 bytes of A and one 512-byte row of x per token)
+// into the warp's private ring; columns past h_in arrive as zeros.  `phase` holds one parity bit
+// per ring stage and lives across calls.  Returns false if a wait gave up.
+template <int NT>
+__device__ __forceinline__ bool shrink_rows8(const CUtensorMap *tmap_a, const CUtensorMap *tmap_x,
+                                             int32_t slot, int32_t row0, const int32_t (&tok)[kDsTok],
+                                             int step0, int step1, uint8_t *ring, uint64_t *bars,
+                                             uint32_t &phase, int lane, float (&acc)[8 * kDsTok]) {
   auto issue = [&](int step, int stage) {
-    const int k = step * 32 + lane;
-    if (step < step1 && k < n_u4) {
-      uint4 *dst = ring + stage * kStageStride;
+    if (lane == 0 && step < step1) {
+      uint8_t *dst = ring + stage * kDsStageBytes;
+      ptx::mbar_arrive_expect_tx(&bars[stage], (8 + NT) * kDsRowBytes);
+      ptx::tma_load_3d(dst, tmap_a, &bars[stage], step * kShrinkStepElems, row0, slot);
 #pragma unroll
-      for (int r = 0; r < 8; ++r) cp_async16(dst + r * kShrinkThreads, A0 + r * row_u4 + k);
-#pragma unroll
-      for (int q = 0; q < NT; ++q) cp_async16(dst + (8 + q) * kShrinkThreads, xr[q] + k);
+      for (int q = 0; q < NT; ++q)
+        ptx::tma_load_2d(dst + (8 + q) * kDsRowBytes, tmap_x, &bars[stage], step * kShrinkStepElems, tok[q]);
     }
-    cp_async_commit();  // an empty group keeps the group count uniform
   };
 #pragma unroll
-  for (int d = 0; d < DEPTH - 1; ++d) issue(step0 + d * dstep, d);
+  for (int d = 0; d < kDsDepth - 1; ++d) issue(step0 + d, d);
   int stage = 0;
-  for (int step = step0; step < step1; step += dstep) {
-    int pre = stage + DEPTH - 1;
-    if (pre >= DEPTH) pre -= DEPTH;
-    issue(step + (DEPTH - 1) * dstep, pre);
-    cp_async_wait<DEPTH - 1>();
-    const int k = step * 32 + lane;
-    if (k < n_u4) {
-      const uint4 *src = ring + stage * kStageStride;
-      float xf[NT][8];
+  for (int step = step0; step < step1; ++step) {
+    __syncwarp();  // every lane has finished reading the stage that is refilled next
+    issue(step + kDsDepth - 1, (stage + kDsDepth - 1) % kDsDepth);
+    if (!ptx::mbar_wait(&bars[stage], (phase >> stage) & 1u)) return false;
+    phase ^= 1u << stage;
+    const uint4 *src = reinterpret_cast<const uint4 *>(ring + stage * kDsStageBytes) + lane;
+    float xf[NT][8];
 #pragma unroll
-      for (int q = 0; q < NT; ++q) unpack8(src[(8 + q) * kShrinkThreads], xf[q]);
+    for (int q = 0; q < NT; ++q) unpack8(src[(8 + q) * (kDsRowBytes / 16)], xf[q]);
 #pragma unroll
-      for (int r = 0; r < 8; ++r) {
-        float af[8];
-        unpack8(src[r * kShrinkThreads], af);
+    for (int r = 0; r < 8; ++r) {
+      float af[8];
+      unpack8(src[r * (kDsRowBytes / 16)], af);
 #pragma unroll
-        for (int q = 0; q < NT; ++q)
+      for (int q = 0; q < NT; ++q)
 #pragma unroll
-          for (int e = 0; e < 8; ++e) acc[r * kDsTok + q] = fmaf(af[e], xf[q][e], acc[r * kDsTok + q]);
-      }
+        for (int e = 0; e < 8; ++e) acc[r * kDsTok + q] = fmaf(af[e], xf[q][e], acc[r * kDsTok + q]);
     }
-    if (++stage == DEPTH) stage = 0;
+    if (++stage == kDsDepth) stage = 0;
   }
-  cp_async_wait<0>();
+  return true;
 }
 
-constexpr int kDsDepth = 3;      // ring stages
-constexpr int kDsBlockTok = 8;   // tokens of one group handled by one work item (two passes of four)
-constexpr size_t kDsRingBytes = static_cast<size_t>(kDsDepth) * kRingSlots * kShrinkThreads * 16;
+constexpr int kDsBlockTok = kDsTok;  // tokens of one group handled by one work item (one pass)
+constexpr int kDsTicket = kDecodeMaxT * 8;  // index of the work-item ticket counter in group_counters
 
-__global__ void __launch_bounds__(kShrinkThreads)
-decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict__ x,
-                     const uint16_t *__restrict__ A_pool, const SlotRow *__restrict__ slots,
+__device__ __forceinline__ int atomic_add_acq_rel(int32_t *p, int v) {
+  int old;
+  asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
+constexpr size_t kDsRingBytes = static_cast<size_t>(kShrinkThreads / 32) * kDsDepth * kDsStageBytes + 1024;
+
+__global__ void __launch_bounds__(kShrinkThreads, 1)
+decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_x,
+                     const int32_t *__restrict__ ids, const SlotRow *__restrict__ slots,
                      PlanView pv, float *__restrict__ zws, int32_t *__restrict__ group_counters,
                      int32_t T, int32_t h_in, int32_t R_pad, int32_t n_slots, int32_t max_tokens,
                      int32_t target_items, uint32_t *status) {
-  extern __shared__ uint4 s_ring[];    // [depth][slot][thread]
+  extern __shared__ uint8_t s_ring_raw[];  // [warp][stage][8 A rows + 4 x rows][512 bytes]
+  __shared__ uint64_t s_bars[kShrinkThreads / 32][kDsDepth];
   __shared__ int32_t s_id[256];        // validated id of each token
   __shared__ int32_t s_grp[256];       // group (in order of first appearance) of a group's first token
   __shared__ int32_t s_gadapter[256];  // adapter of each group
@@ -248,11 +244,16 @@ decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict
   __shared__ int32_t s_bgrp[256];      // token blocks: group and first position in s_gtok
   __shared__ int32_t s_btok[256];
   __shared__ int s_wt[9];
-  __shared__ float s_red[8][32];
-  __shared__ int s_last;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   ptx::pdl_launch_dependents();
+  if (tid == 0) {
+    ptx::prefetch_tensormap(&tmap_a);
+    ptx::prefetch_tensormap(&tmap_x);
+    for (int w = 0; w < kShrinkThreads / 32; ++w)
+      for (int d = 0; d < kDsDepth; ++d) ptx::mbar_init(&s_bars[w][d], 1);
+    ptx::fence_barrier_init();
+  }
 
   // ---- routing, in shared memory (reads only the caller's ids)
   int a = -1;
@@ -307,14 +308,13 @@ decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict
   if (mygrp >= 0) s_gtok[s_gstart[mygrp] + pos] = tid;
   const int any_bad = __syncthreads_or(bad ? 1 : 0);
 
-  // K chunks: enough items to occupy the machine, but an item keeps at least about 128 KB of A
-  // (below that the extra pass that adds the chunks costs more than it saves) and one K step per
-  // warp sub-range.
+  // Work items are per warp: (token block, K chunk, group of eight rank rows).  K chunks: enough
+  // items for every warp of the grid, but a chunk keeps at least four K steps (1024 elements)
+  // unless h_in is shorter, so that the ring's ramp-up is amortised.
   const int n_ksteps = (h_in + 255) >> 8;
-  const int ksubs_nominal = 64 / R_pad;  // 4, 2, 1 for a rank stride of 16, 32, 64
-  int KS = (target_items + max(NB, 1) - 1) / max(NB, 1);
-  KS = min(KS, max(1, (R_pad * h_in * 2) >> 17));
-  KS = max(1, min(min(KS, kMaxZSplits), n_ksteps / ksubs_nominal));
+  const int n_rgn = R_pad >> 3;  // row groups of the rank stride: 2, 4 or 8
+  int KS = (target_items + max(NB * n_rgn, 1) - 1) / max(NB * n_rgn, 1);
+  KS = max(1, min(min(KS, kMaxZSplits), n_ksteps / 4));
   const int spc = (n_ksteps + KS - 1) / KS;
   KS = (n_ksteps + spc - 1) / spc;
 
@@ -375,46 +375,56 @@ decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict
     }
   }
 
-  // ---- work items (token block of a group, K chunk)
-  const int n_items = NB * KS;
-  const int n_u4 = h_in >> 3;
+  // ---- per-warp work items, no CTA-wide synchronisation from here on
+  const int n_items = NB * KS * n_rgn;
   const size_t zplane = static_cast<size_t>(max_tokens) * R_pad;
-  uint4 *my_ring = s_ring + tid;
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const int bi = item / KS, c = item - bi * KS;
+  uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(s_ring_raw) + 127) & ~uintptr_t(127)) +
+                  static_cast<size_t>(warp) * kDsDepth * kDsStageBytes;
+  uint64_t *bars = s_bars[warp];
+  uint32_t phase = 0;
+  bool ok = true;
+  // Items are drawn from a ticket counter so that warps stay busy whatever the items cost; the
+  // next ticket is drawn before the current item is processed.  The very last draw of the launch
+  // (item number n_items + warps - 1) puts the counter back to zero.
+  const int warps_total = gridDim.x * (kShrinkThreads / 32);
+  int32_t *ticket = group_counters + kDsTicket;
+  int item = blockIdx.x * (kShrinkThreads / 32) + warp;  // first round is static
+  while (ok && item < n_items) {
+    int next = 0;
+    if (lane == 0) next = warps_total + atomicAdd(ticket, 1);
+    next = __shfl_sync(0xffffffffu, next, 0);
+    const int cur = item;
+    item = next;
+    const int rg = cur % n_rgn;
+    const int bc = cur / n_rgn;
+    const int bi = bc / KS, c = bc - bi * KS;
     const int gi = s_bgrp[bi];
     const int ad = s_gadapter[gi];
     const SlotRow row = slots[ad];
-    const int t0 = s_btok[bi], g_end = s_gstart[gi + 1];
-    const int t1 = min(t0 + kDsBlockTok, g_end);
+    const int gt0 = s_gstart[gi], g_end = s_gstart[gi + 1];
+    const int t0 = s_btok[bi], t1 = min(t0 + kDsBlockTok, g_end);
     if (row.rank <= 0) {
-      if (tid == 0 && c == 0 && t0 == s_gstart[gi]) atomicOr(status, EDGELORA_STATUS_SLOT_EMPTY);
+      if (lane == 0 && c == 0 && rg == 0 && t0 == gt0) atomicOr(status, EDGELORA_STATUS_SLOT_EMPTY);
       continue;
     }
     const int n_rg = (row.rank + 7) >> 3;  // live groups of eight rows
-    int rg_p2 = 1;
-    while (rg_p2 < n_rg) rg_p2 <<= 1;
-    const int ksubs = 8 / rg_p2;
-    const int rg = warp % rg_p2, ksub = warp / rg_p2;
+    if (rg >= n_rg) continue;               // rows past the rank are zero padding: nothing to do
     const int step0 = c * spc, step1 = min(n_ksteps, step0 + spc);
-    const uint4 *A0 =
-        reinterpret_cast<const uint4 *>(A_pool + (static_cast<size_t>(ad) * R_pad + rg * 8) * h_in);
-    for (int tb = t0; tb < t1; tb += kDsTok) {
+    const int q = lane & 3, r = rg * 8 + (lane >> 2);
+    for (int tb = t0; ok && tb < t1; tb += kDsTok) {
       const int nt = min(kDsTok, t1 - tb);
       float acc[8 * kDsTok];
 #pragma unroll
       for (int i = 0; i < 8 * kDsTok; ++i) acc[i] = 0.f;
-      if (rg < n_rg) {
-        const uint4 *xr[kDsTok];
+      int32_t tok[kDsTok];
 #pragma unroll
-        for (int q = 0; q < kDsTok; ++q)
-          xr[q] = reinterpret_cast<const uint4 *>(x + static_cast<size_t>(s_gtok[tb + min(q, nt - 1)]) * h_in);
-        const size_t row_u4 = static_cast<size_t>(n_u4);
-        if (nt == 1) shrink_rows8<1, kDsDepth>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, my_ring, acc);
-        else if (nt == 2) shrink_rows8<2, kDsDepth>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, my_ring, acc);
-        else if (nt == 3) shrink_rows8<3, kDsDepth>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, my_ring, acc);
-        else shrink_rows8<4, kDsDepth>(A0, row_u4, xr, step0 + ksub, step1, ksubs, n_u4, lane, my_ring, acc);
-      }
+      for (int qq = 0; qq < kDsTok; ++qq) tok[qq] = s_gtok[tb + min(qq, nt - 1)];
+      if (nt == 1) ok = shrink_rows8<1>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
+      else if (nt == 2) ok = shrink_rows8<2>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
+      else if (nt == 3) ok = shrink_rows8<3>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
+      else ok = shrink_rows8<4>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       // lane L ends with the sum over lanes of value L (= row L / 4, token L % 4)
 #pragma unroll
       for (int off = 16, cnt = 16; off >= 1; off >>= 1, cnt >>= 1) {
@@ -426,38 +436,24 @@ decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict
           acc[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
         }
       }
-      float v = acc[0];
-      if (ksubs > 1) {
-        s_red[warp][lane] = v;
-        __syncthreads();
-        if (ksub == 0)
-          for (int j = 1; j < ksubs; ++j) v += s_red[warp + j * rg_p2][lane];
-        __syncthreads();
-      }
-      const int q = lane & 3, r = rg * 8 + (lane >> 2);
-      if (ksub == 0 && rg < n_rg && q < nt)
+      if (q < nt)
         zws[(KS > 1 ? c : kMaxZSplits) * zplane + static_cast<size_t>(s_gtok[tb + q]) * R_pad + r] =
-            row.scale * v;
+            row.scale * acc[0];
     }
+    if (!ok) break;
     if (KS > 1) {
-      // The item that completes a group adds the K chunks in order into the final plane (it never
-      // waits for the others).
-      const int gt0 = s_gstart[gi];
+      // The warp that completes (group, row group) adds the K chunks in order into the final plane;
+      // it never waits for the others.
       const int arrivals = KS * ((g_end - gt0 + kDsBlockTok - 1) / kDsBlockTok);
-      __threadfence();
-      __syncthreads();
-      if (tid == 0) {
-        const int old = atomicAdd(&group_counters[gi], 1);
-        s_last = (old == arrivals - 1) ? 1 : 0;
-        if (s_last) group_counters[gi] = 0;  // ready for the next launch
-      }
-      __syncthreads();
-      if (s_last) {
-        __threadfence();
-        const int live = n_rg * 8;
-        for (int idx = tid; idx < (g_end - gt0) * live; idx += kShrinkThreads) {
-          const int q = idx / live, r = idx - q * live;
-          const size_t off = static_cast<size_t>(s_gtok[gt0 + q]) * R_pad + r;
+      __syncwarp();  // the lanes' z stores happen before lane 0's release
+      int old = 0;
+      if (lane == 0) old = atomic_add_acq_rel(&group_counters[gi * 8 + rg], 1);
+      old = __shfl_sync(0xffffffffu, old, 0);
+      if (old == arrivals - 1) {
+        if (lane == 0) group_counters[gi * 8 + rg] = 0;  // ready for the next launch
+        for (int idx = lane; idx < (g_end - gt0) * 8; idx += 32) {
+          const int tq = idx >> 3;
+          const size_t off = static_cast<size_t>(s_gtok[gt0 + tq]) * R_pad + rg * 8 + (idx & 7);
           float part[kMaxZSplits];
 #pragma unroll
           for (int sp = 0; sp < kMaxZSplits; ++sp) part[sp] = sp < KS ? __ldcg(zws + sp * zplane + off) : 0.f;
@@ -469,21 +465,32 @@ decode_shrink_kernel(const int32_t *__restrict__ ids, const uint16_t *__restrict
       }
     }
   }
+  // Every warp stops at its first ticket >= n_items, so exactly n_items - (first round) + warps
+  // draws happen; the one that drew the last ticket resets the counter for the next launch.
+  if (lane == 0 && ok) {
+    const int first_round = min(n_items, warps_total);
+    const int last_ticket = warps_total + (n_items - first_round) + first_round - 1;
+    if (item == last_ticket) *ticket = 0;
+  }
+  if (!ok && lane == 0) atomicOr(status, EDGELORA_STATUS_TIMEOUT);
 }
 
-void launch_decode_shrink(const int32_t *ids, const uint16_t *x, const uint16_t *A_pool,
-                          const SlotRow *slots, const PlanView &pv, float *zws,
-                          int32_t *group_counters, int32_t T, int32_t h_in, int32_t R_pad,
-                          int32_t n_slots, int32_t max_tokens, int32_t target_items, int32_t grid,
-                          uint32_t *status, bool pdl, cudaStream_t stream) {
+cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &tmap_x,
+                                 const int32_t *ids, const SlotRow *slots, const PlanView &pv,
+                                 float *zws, int32_t *group_counters, int32_t T, int32_t h_in,
+                                 int32_t R_pad, int32_t n_slots, int32_t max_tokens,
+                                 int32_t target_items, int32_t grid, uint32_t *status, bool pdl,
+                                 cudaStream_t stream) {
   static bool configured = false;  // per process; the attribute is per function and device-wide
   if (!configured) {
-    cudaFuncSetAttribute(decode_shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         static_cast<int>(kDsRingBytes));
+    cudaError_t e = cudaFuncSetAttribute(decode_shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kDsRingBytes));
+    if (e != cudaSuccess) return e;
     configured = true;
   }
-  launch_ex(decode_shrink_kernel, dim3(grid), dim3(kShrinkThreads), kDsRingBytes, stream, pdl, 1, ids, x, A_pool,
-            slots, pv, zws, group_counters, T, h_in, R_pad, n_slots, max_tokens, target_items, status);
+  return launch_ex(decode_shrink_kernel, dim3(grid), dim3(kShrinkThreads), kDsRingBytes, stream, pdl, 1,
+                   tmap_a, tmap_x, ids, slots, pv, zws, group_counters, T, h_in, R_pad, n_slots,
+                   max_tokens, target_items, status);
 }
 
 }  // namespace edgelora
