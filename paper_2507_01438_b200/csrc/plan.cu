@@ -7,9 +7,12 @@
 //   groups      tokens ordered by (id, token): ids ascending with -1 first, token order kept,
 //   short lists the groups restricted to tokens the gather-by-token shrink handles,
 //   sgmv tiles  in batches above kDecodeMaxT tokens, for runs of >= kSegMin tokens on a real
-//               adapter: 128-token tiles of the run (work list of the segment shrink).
-// The order is produced by a bitonic sort of the unique keys ((id + 1) << 16 | token) in shared
-// memory, so it is exact and the same on every run.
+//               adapter: 128-token tiles of the run (work list of the segment shrink),
+//   tile lists  the distinct ids >= 0 inside every 128-token tile (the LoRA K blocks of that tile).
+// Tokens of one run stay together in the group order, so the runs are sorted, not the tokens: a
+// bitonic sort of the unique keys ((id + 1) << 16 | run index) in shared memory, exact and the
+// same on every launch.  Prefix sums run in rounds of one element per thread (warp shuffles plus
+// one shared-memory stage), so nothing but the outputs goes through global memory.
 #include "internal.cuh"
 #include "launch.cuh"
 #include "ptx.cuh"
@@ -18,74 +21,88 @@ namespace edgelora {
 
 constexpr int kPlanThreads = 1024;
 
-// In-place exclusive prefix sum of data[0..n) by the whole CTA; returns the total.
-__device__ int block_exclusive_scan(int32_t *data, int n, int *warp_sums) {
-  const int tid = threadIdx.x;
-  const int per = (n + kPlanThreads - 1) / kPlanThreads;
-  const int lo = min(n, tid * per), hi = min(n, lo + per);
-  int local = 0;
-  for (int i = lo; i < hi; ++i) local += data[i];
-  // inclusive scan of `local` across the CTA
-  int incl = local;
-  const int lane = tid & 31, warp = tid >> 5;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    int v = __shfl_up_sync(0xffffffffu, incl, d);
-    if (lane >= d) incl += v;
-  }
-  if (lane == 31) warp_sums[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    int w = warp_sums[lane];
-    int wi = w;
+// Exclusive prefix sum over i in [0, n) of value(i), one element per thread per round;
+// consume(i, prefix) is called for every i.  Returns the total.  `wt` is shared memory [34].
+template <typename Value, typename Consume>
+__device__ __forceinline__ int scan_rounds(int n, int *wt, Value value, Consume consume) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int base = 0;
+  for (int i0 = 0; i0 < n; i0 += kPlanThreads) {
+    const int i = i0 + tid;
+    const int v = i < n ? value(i) : 0;
+    int incl = v;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
-      int v = __shfl_up_sync(0xffffffffu, wi, d);
-      if (lane >= d) wi += v;
+      const int o = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += o;
     }
-    warp_sums[lane] = wi - w;  // exclusive prefix of the warp totals
-    if (lane == 31) warp_sums[32] = wi;
+    if (lane == 31) wt[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const int w = wt[lane];
+      int wi = w;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, wi, d);
+        if (lane >= d) wi += o;
+      }
+      wt[lane] = wi - w;
+      if (lane == 31) wt[32] = wi;
+    }
+    __syncthreads();
+    if (i < n) consume(i, base + wt[warp] + incl - v);
+    base += wt[32];
+    __syncthreads();
   }
-  __syncthreads();
-  int run = warp_sums[warp] + incl - local;
-  for (int i = lo; i < hi; ++i) {
-    int v = data[i];
-    data[i] = run;
-    run += v;
-  }
-  const int total = warp_sums[32];
-  __syncthreads();
-  return total;
+  return base;
 }
 
 __global__ void __launch_bounds__(kPlanThreads)
-plan_kernel(const int32_t *__restrict__ ids, int32_t T, int32_t n_slots, PlanView pv, int32_t npow2) {
-  extern __shared__ uint32_t keys[];
-  __shared__ int warp_sums[33];
+plan_kernel(const int32_t *__restrict__ ids, int32_t T, int32_t n_slots, PlanView pv) {
+  extern __shared__ uint32_t keys[];  // one key per run, padded to a power of two
+  __shared__ int wt[34];
   const int tid = threadIdx.x;
 
   ptx::pdl_launch_dependents();
   ptx::pdl_wait_prior_grids();  // earlier kernels on the stream may still read the plan arrays
 
-  // 1. validate, build keys
+  // 1. validate
   bool bad = false;
-  for (int i = tid; i < npow2; i += kPlanThreads) {
-    uint32_t key = 0xFFFFFFFFu;
-    if (i < T) {
-      int32_t a = ids[i];
-      if (a < -1 || a >= n_slots) {
-        a = -1;
-        bad = true;
-      }
-      pv.ids_valid[i] = a;
-      key = (static_cast<uint32_t>(a + 1) << 16) | static_cast<uint32_t>(i);
+  for (int t = tid; t < T; t += kPlanThreads) {
+    int32_t a = ids[t];
+    if (a < -1 || a >= n_slots) {
+      a = -1;
+      bad = true;
     }
-    keys[i] = key;
+    pv.ids_valid[t] = a;
   }
-  if (bad) atomicOr(pv.status, EDGELORA_STATUS_BAD_ADAPTER_ID);
+  if (__syncthreads_or(bad ? 1 : 0) && tid == 0) atomicOr(pv.status, EDGELORA_STATUS_BAD_ADAPTER_ID);
+
+  // 2. segments = maximal runs of equal id in token order
+  auto is_head = [&](int t) { return (t == 0 || pv.ids_valid[t] != pv.ids_valid[t - 1]) ? 1 : 0; };
+  const int n_segs = scan_rounds(
+      T, wt, is_head, [&](int t, int before) {
+        const int head = is_head(t);
+        const int s = before + head - 1;
+        pv.tok_seg[t] = s;
+        if (head) {
+          pv.seg_start[s] = t;
+          pv.seg_adapter[s] = pv.ids_valid[t];
+        }
+      });
+  if (tid == 0) {
+    pv.seg_start[n_segs] = T;
+    pv.counts[1] = n_segs;
+  }
   __syncthreads();
 
-  // 2. bitonic sort, ascending
+  // 3. runs ordered by (id, run index): -1 first, token order kept (runs are in token order)
+  int npow2 = 32;
+  while (npow2 < n_segs) npow2 <<= 1;
+  for (int i = tid; i < npow2; i += kPlanThreads)
+    keys[i] = i < n_segs ? ((static_cast<uint32_t>(pv.seg_adapter[i] + 1) << 16) | static_cast<uint32_t>(i))
+                         : 0xFFFFFFFFu;
+  __syncthreads();
   for (int k = 2; k <= npow2; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
       for (int i = tid; i < npow2; i += kPlanThreads) {
@@ -103,102 +120,88 @@ plan_kernel(const int32_t *__restrict__ ids, int32_t T, int32_t n_slots, PlanVie
     }
   }
 
-  // 3. segments
-  for (int t = tid; t < T; t += kPlanThreads)
-    pv.scratch[t] = (t == 0 || pv.ids_valid[t] != pv.ids_valid[t - 1]) ? 1 : 0;
-  __syncthreads();
-  const int n_segs = block_exclusive_scan(pv.scratch, T, warp_sums);
+  // 4. groups: the runs in sorted order, concatenated.  out_start[j] (in pv.scratch) is where the
+  // j-th sorted run begins in perm; inv (borrowing pv.mt_list until step 8) maps a run to j.
+  int32_t *out_start = pv.scratch, *inv = pv.mt_list, *gidx = pv.perm_short;  // gidx: until step 6
+  auto run_of = [&](int j) { return static_cast<int>(keys[j] & 0xFFFFu); };
+  auto run_len = [&](int j) {
+    const int s = run_of(j);
+    return pv.seg_start[s + 1] - pv.seg_start[s];
+  };
+  scan_rounds(n_segs, wt, run_len, [&](int j, int before) {
+    out_start[j] = before;
+    inv[run_of(j)] = j;
+  });
   for (int t = tid; t < T; t += kPlanThreads) {
-    const bool head = (t == 0 || pv.ids_valid[t] != pv.ids_valid[t - 1]);
-    const int s = pv.scratch[t] + (head ? 1 : 0) - 1;
-    pv.tok_seg[t] = s;
+    const int s = pv.tok_seg[t];
+    pv.perm[out_start[inv[s]] + (t - pv.seg_start[s])] = t;
+  }
+  auto is_ghead = [&](int j) { return (j == 0 || (keys[j] >> 16) != (keys[j - 1] >> 16)) ? 1 : 0; };
+  const int has_base = (n_segs > 0 && (keys[0] >> 16) == 0) ? 1 : 0;  // the group of id -1 sorts first
+  const int n_groups = scan_rounds(n_segs, wt, is_ghead, [&](int j, int before) {
+    const int head = is_ghead(j);
+    const int g = before + head - 1;
+    gidx[j] = g;
     if (head) {
-      pv.seg_start[s] = t;
-      pv.seg_adapter[s] = pv.ids_valid[t];
+      const int32_t a = static_cast<int32_t>(keys[j] >> 16) - 1;
+      pv.group_start[g] = out_start[j];
+      pv.group_adapter[g] = a;
+      if (a >= 0) pv.lg_adapter[g - has_base] = a;
     }
-  }
-  if (tid == 0) {
-    pv.seg_start[n_segs] = T;
-    pv.counts[1] = n_segs;
-  }
-  __syncthreads();
-
-  // 4. groups
-  for (int i = tid; i < T; i += kPlanThreads) {
-    pv.perm[i] = static_cast<int32_t>(keys[i] & 0xFFFFu);
-    pv.scratch[i] = (i == 0 || (keys[i] >> 16) != (keys[i - 1] >> 16)) ? 1 : 0;
-  }
-  __syncthreads();
-  const int n_groups = block_exclusive_scan(pv.scratch, T, warp_sums);
-  for (int i = tid; i < T; i += kPlanThreads) {
-    if (i == 0 || (keys[i] >> 16) != (keys[i - 1] >> 16)) {
-      const int g = pv.scratch[i];
-      pv.group_start[g] = i;
-      pv.group_adapter[g] = static_cast<int32_t>(keys[i] >> 16) - 1;
-    }
-  }
-  const int has_base = (keys[0] >> 16) == 0 ? 1 : 0;  // the group of id -1 sorts first
-  for (int i = tid; i < T; i += kPlanThreads) {
-    const uint32_t id1 = keys[i] >> 16;
-    if (id1 != 0 && (i == 0 || id1 != (keys[i - 1] >> 16)))
-      pv.lg_adapter[pv.scratch[i] - has_base] = static_cast<int32_t>(id1) - 1;
-  }
+  });
   if (tid == 0) {
     pv.group_start[n_groups] = T;
     pv.counts[0] = n_groups;
     pv.counts[4] = n_groups - has_base;
     pv.counts[5] = 0;
   }
-  __syncthreads();
 
-  // 4b. the same groups restricted to "short" tokens: every token of a small batch, otherwise
-  // the tokens of runs shorter than kSegMin (long runs go to the segment shrink)
+  // 5. the same groups restricted to "short" tokens: every token of a small batch, otherwise the
+  // tokens of runs shorter than kSegMin (long runs go to the segment shrink).  sstart[j] replaces
+  // out_start[j] in pv.scratch.
   const bool all_short = T <= kDecodeMaxT;
-  for (int i = tid; i < T; i += kPlanThreads) {
-    const int t = static_cast<int>(keys[i] & 0xFFFFu);
+  auto short_len = [&](int j) {
+    const int len = run_len(j);
+    return (all_short || len < kSegMin) ? len : 0;
+  };
+  const int n_short = scan_rounds(n_segs, wt, short_len, [&](int j, int before) {
+    out_start[j] = before;
+    if (is_ghead(j)) pv.gs_short[gidx[j]] = before;
+  });
+  // 6. (gidx is dead from here: perm_short takes its final content)
+  for (int t = tid; t < T; t += kPlanThreads) {
     const int s = pv.tok_seg[t];
-    pv.scratch[i] = (all_short || (pv.seg_start[s + 1] - pv.seg_start[s]) < kSegMin) ? 1 : 0;
+    const int len = pv.seg_start[s + 1] - pv.seg_start[s];
+    if (all_short || len < kSegMin) pv.perm_short[out_start[inv[s]] + (t - pv.seg_start[s])] = t;
   }
-  __syncthreads();
-  const int n_short = block_exclusive_scan(pv.scratch, T, warp_sums);
-  for (int i = tid; i < T; i += kPlanThreads) {
-    const int t = static_cast<int>(keys[i] & 0xFFFFu);
-    const int s = pv.tok_seg[t];
-    if (all_short || (pv.seg_start[s + 1] - pv.seg_start[s]) < kSegMin) pv.perm_short[pv.scratch[i]] = t;
-  }
-  for (int g = tid; g < n_groups; g += kPlanThreads) pv.gs_short[g] = pv.scratch[pv.group_start[g]];
   if (tid == 0) {
     pv.gs_short[n_groups] = n_short;
     pv.counts[3] = n_short;
   }
-  __syncthreads();
 
-  // 5. 128-token tiles of the long runs (segment shrink work list)
-  for (int s = tid; s < n_segs; s += kPlanThreads) {
+  // 7. 128-token tiles of the long runs (segment shrink work list), in token order
+  auto run_tiles = [&](int s) {
     const int len = pv.seg_start[s + 1] - pv.seg_start[s];
-    pv.scratch[s] =
-        (!all_short && pv.seg_adapter[s] >= 0 && len >= kSegMin) ? (len + kTileM - 1) / kTileM : 0;
-  }
-  __syncthreads();
-  const int n_tiles = block_exclusive_scan(pv.scratch, n_segs, warp_sums);
-  for (int s = tid; s < n_segs; s += kPlanThreads) {
+    return (!all_short && pv.seg_adapter[s] >= 0 && len >= kSegMin) ? (len + kTileM - 1) / kTileM : 0;
+  };
+  const int n_tiles = scan_rounds(n_segs, wt, run_tiles, [&](int s, int before) {
     const int t0 = pv.seg_start[s];
     const int len = pv.seg_start[s + 1] - t0;
-    if (!all_short && pv.seg_adapter[s] >= 0 && len >= kSegMin) {
-      int tile = pv.scratch[s];
-      for (int o = 0; o < len; o += kTileM, ++tile) {
-        if (tile < pv.max_sgmv_tiles) {
-          pv.sgmv_tiles[4 * tile + 0] = t0 + o;
-          pv.sgmv_tiles[4 * tile + 1] = min(kTileM, len - o);
-          pv.sgmv_tiles[4 * tile + 2] = pv.seg_adapter[s];
-          pv.sgmv_tiles[4 * tile + 3] = 0;
-        }
+    const int nt = run_tiles(s);
+    for (int i = 0; i < nt; ++i) {
+      const int tile = before + i;
+      if (tile < pv.max_sgmv_tiles) {
+        pv.sgmv_tiles[4 * tile + 0] = t0 + i * kTileM;
+        pv.sgmv_tiles[4 * tile + 1] = min(kTileM, len - i * kTileM);
+        pv.sgmv_tiles[4 * tile + 2] = pv.seg_adapter[s];
+        pv.sgmv_tiles[4 * tile + 3] = 0;
       }
     }
-  }
+  });
   if (tid == 0) pv.counts[2] = min(n_tiles, pv.max_sgmv_tiles);
+  __syncthreads();  // inv (in pv.mt_list) is dead from here
 
-  // 6. the distinct ids >= 0 inside every 128-token tile, in order of first appearance (the LoRA
+  // 8. the distinct ids >= 0 inside every 128-token tile, in order of first appearance (the LoRA
   // K blocks of that tile in the base-product kernel).  One warp per tile; lane l holds the ids
   // of tokens l, l + 32, l + 64, l + 96 of the tile.
   {
@@ -249,10 +252,10 @@ plan_kernel(const int32_t *__restrict__ ids, int32_t T, int32_t n_slots, PlanVie
 
 void launch_plan(const int32_t *ids, int32_t T, int32_t n_slots, const PlanView &pv, bool pdl,
                  cudaStream_t stream) {
-  int npow2 = 32;
+  int npow2 = 32;  // the number of runs is only known on the device: size for the worst case
   while (npow2 < T) npow2 <<= 1;
   launch_ex(plan_kernel, dim3(1), dim3(kPlanThreads), static_cast<size_t>(npow2) * 4, stream, pdl, 1,
-            ids, T, n_slots, pv, npow2);
+            ids, T, n_slots, pv);
 }
 
 void init_plan_kernel() {
