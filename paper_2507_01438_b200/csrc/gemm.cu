@@ -78,13 +78,19 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams &p, int32_t til
   return c;
 }
 
+// decode: first W row of the tile this CTA works on
+__device__ __forceinline__ int32_t tc_row0(const GemmParams &p) {
+  return static_cast<int32_t>(blockIdx.x) / p.splits * kTileM;
+}
+
 // The LoRA K blocks of a tile: entries [e0, e1) step `de` of `list`.  Entries whose slot is
 // empty are skipped by every role alike (they all read the same slot table).
 struct LoraList {
   const int32_t *list;
   int32_t e0, e1, de;
 };
-__device__ __forceinline__ LoraList lora_list(const GemmParams &p, const TileCoord &tc) {
+__device__ __forceinline__ LoraList lora_list(const GemmParams &p, const TileCoord &tc,
+                                              const int32_t *s_lg, const volatile int32_t *s_nlg) {
   LoraList l;
   if (p.mode == kModePrefill) {
     l.list = p.mt_list + tc.mtile * kTileM;
@@ -92,9 +98,9 @@ __device__ __forceinline__ LoraList lora_list(const GemmParams &p, const TileCoo
     l.e1 = p.mt_count[tc.mtile];
     l.de = 1;
   } else if (p.mode == kModeDecode) {
-    l.list = p.lg_adapter;
+    l.list = s_lg;    // built by this CTA from the ids (see the builder warps)
     l.e0 = tc.split;  // the groups are dealt round-robin to the K splits of a row tile
-    l.e1 = p.counts[4];
+    l.e1 = *s_nlg;
     l.de = p.splits;
   } else {
     l.list = nullptr;
@@ -104,6 +110,9 @@ __device__ __forceinline__ LoraList lora_list(const GemmParams &p, const TileCoo
   return l;
 }
 
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -165,7 +174,10 @@ __device__ __forceinline__ void load_z_packed(const GemmParams &p, int32_t t, in
   }
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 2)
+// kMinBlocks = 2 caps the registers so that two CTAs share an SM (small decode tiles); with 1 the
+// builder keeps both of its z rows in registers without spilling.
+template <int kMinBlocks>
+__global__ void __launch_bounds__(kGemmThreads, kMinBlocks)
 lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_constant__ CUtensorMap tmap_c,
                  const __grid_constant__ CUtensorMap tmap_b, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -183,9 +195,22 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   uint64_t *tempty_bar = tfull_bar + 2;           // [2]       epilogue -> MMA
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(tempty_bar + 2);
   volatile uint32_t *abort_flag = tmem_slot + 1;
+  // decode extras, 512 bytes after the barriers: which 32-token column blocks a LoRA K block
+  // touches, and the batch's adapter list derived from the ids by the builder warps
+  uint8_t *extra = reinterpret_cast<uint8_t *>(bars) + 512;
+  volatile uint8_t *s_cmask = extra;                                        // [stages][4]
+  volatile int32_t *s_nlg = reinterpret_cast<volatile int32_t *>(extra + 64);
+  uint64_t *lg_bar = reinterpret_cast<uint64_t *>(extra + 72);              // builder -> TMA, MMA
+  int32_t *s_lg = reinterpret_cast<int32_t *>(extra + 128);                 // [256] ids ascending
+  int32_t *s_vid = reinterpret_cast<int32_t *>(extra + 1152);               // [256] validated ids
+  uint8_t *s_head = extra + 2176;                                           // [256]
+  uint32_t *s_key = reinterpret_cast<uint32_t *>(extra + 2432);             // [256] sort keys
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const bool has_lora = p.mode != kModeSgmv;
+  // LoRA K blocks: prefill always; decode unless the batch is small enough for the expand to be
+  // added by the owners of the cluster reduction (then z is needed only at the very end and the
+  // whole main loop overlaps the shrink kernel)
+  const bool has_lora = p.mode == kModePrefill || (p.mode == kModeDecode && !p.expand_in_reduce);
 
   if (threadIdx.x == 0) {
     ptx::prefetch_tensormap(&tmap_r);
@@ -201,7 +226,9 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       ptx::mbar_init(&tfull_bar[i], 1);
       ptx::mbar_init(&tempty_bar[i], 4);  // one arrival per epilogue warp
     }
+    ptx::mbar_init(lg_bar, 1);
     *abort_flag = 0;
+    *s_nlg = 0;
     ptx::fence_barrier_init();
   }
   if (warp == 1) {
@@ -245,14 +272,21 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
           }
         }
         if (!ok || !has_lora) continue;
-        if (!waited) {  // the adapter lists come from the kernel before this one
-          ptx::pdl_wait_prior_grids();
+        if (!waited) {
+          if (p.mode == kModeDecode) {  // the builder warps derive the adapter list from the ids
+            if (!ptx::mbar_wait(lg_bar, 0)) {
+              ok = false;
+              break;
+            }
+          } else {                      // the tile lists come from the plan kernel
+            ptx::pdl_wait_prior_grids();
+          }
           waited = true;
         }
-        const LoraList ll = lora_list(p, tc);
+        const LoraList ll = lora_list(p, tc, s_lg, s_nlg);
         for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
           const int32_t a = ll.list[e];
-          if (p.slots[a].rank <= 0) continue;
+          if (p.mode != kModeDecode && p.slots[a].rank <= 0) continue;
           if (!ptx::mbar_wait(&empty_bar[stage], phase ^ 1) || *abort_flag) {
             ok = false;
             break;
@@ -320,13 +354,20 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         if (!ok) break;
         if (has_lora) {
           if (!waited) {
-            ptx::pdl_wait_prior_grids();
+            if (p.mode == kModeDecode) {
+              if (!ptx::mbar_wait(lg_bar, 0)) {
+                ok = false;
+                break;
+              }
+            } else {
+              ptx::pdl_wait_prior_grids();
+            }
             waited = true;
           }
-          const LoraList ll = lora_list(p, tc);
+          const LoraList ll = lora_list(p, tc, s_lg, s_nlg);
           for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
             const int32_t a = ll.list[e];
-            if (p.slots[a].rank <= 0) continue;
+            if (p.mode != kModeDecode && p.slots[a].rank <= 0) continue;
             if (!ptx::mbar_wait(&full_bar[stage], phase) ||
                 !ptx::mbar_wait(&zfull_bar[stage], (zphase >> stage) & 1u) || *abort_flag) {
               ok = false;
@@ -337,7 +378,26 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
             const uint32_t sr = ptx::smem_u32(smem + static_cast<size_t>(stage) * stage_bytes);
             const uint64_t da = ptx::umma_desc_k128(sr);
             const uint64_t db = ptx::umma_desc_k128(sr + r_bytes);
-            for (int k = 0; k < lora_ksteps; ++k) ptx::umma_bf16(tmem_d, da + 2 * k, db + 2 * k, idesc, 1u);
+            if (p.mode == kModePrefill) {
+              for (int k = 0; k < lora_ksteps; ++k) ptx::umma_bf16(tmem_d, da + 2 * k, db + 2 * k, idesc, 1u);
+            } else {
+              // decode: only the 32-token column blocks that hold tokens of this adapter; the
+              // builder wrote those blocks of the z operand and left a flag per block
+              const uint32_t idesc32 = ptx::umma_idesc_bf16(kTileM, 32);
+#pragma unroll
+              for (int w = 0; w < 4; ++w) {
+                const uint32_t flags = s_cmask[stage * 4 + w];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                  if (flags & (1u << h)) {
+                    const uint32_t cb = static_cast<uint32_t>(h * 4 + w);  // tokens [32 cb, 32 cb + 32)
+                    const uint64_t dbc = ptx::umma_desc_k128(sr + r_bytes + cb * 4096u);
+                    for (int k = 0; k < lora_ksteps; ++k)
+                      ptx::umma_bf16(tmem_d + cb * 32u, da + 2 * k, dbc + 2 * k, idesc32, 1u);
+                  }
+                }
+              }
+            }
             ptx::umma_commit(&empty_bar[stage]);
             if (++stage == nstages) {
               stage = 0;
@@ -358,7 +418,36 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     const int quad = warp & 3;                      // TMEM lanes [32*quad, 32*quad+32)
     const int row_in_tile = quad * 32 + lane;
     const bool clustered = p.mode == kModeDecode && p.splits > 1;
-    ptx::pdl_wait_prior_grids();                    // earlier kernels may still read y / the workspace
+    if (clustered && p.expand_in_reduce) {
+      // This CTA will finish tokens [rank * cols_per, ...) of its row tile; pull the B_a rows they
+      // need into L2 now (the ids are the caller's input, the pool is not written by the shrink).
+      const int cols_per = p.BN / p.splits;
+      const int t0 = static_cast<int>(cluster_cta_rank()) * cols_per;
+      for (int cl = quad; cl < cols_per; cl += 4) {  // one warp per token
+        int32_t a = -1, rank = 0;
+        if (t0 + cl < p.T) {
+          a = p.ids[t0 + cl];
+          if (a < 0 || a >= p.n_slots) a = -1;
+          if (a >= 0) rank = p.slots[a].rank;
+        }
+        if (lane == 0) {  // kept for the expand at the end
+          s_vid[cl] = rank > 0 ? a : -1;
+          s_lg[cl] = rank;
+        }
+        if (t0 + cl < p.T) {
+          if (a >= 0 && a < p.n_slots) {
+            const uint8_t *rows = reinterpret_cast<const uint8_t *>(
+                p.B_pool + (static_cast<size_t>(a) * p.h_out + tc_row0(p)) * p.R_pad);
+            const int bytes = min(kTileM, p.h_out - tc_row0(p)) * p.R_pad * 2;  // this tile's rows, contiguous
+            for (int off = lane * 128; off < bytes; off += 32 * 128)
+              asm volatile("prefetch.global.L2 [%0];" ::"l"(rows + off));
+          }
+        }
+      }
+    }
+    // Earlier kernels may still read y, and z comes from the shrink kernel.  With the expand in
+    // the reduction both matter only at the very end, so that wait moves there.
+    if (!(clustered && p.expand_in_reduce)) ptx::pdl_wait_prior_grids();
     bool ok = true;
     int32_t it = 0;
     for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++it) {
@@ -446,34 +535,98 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   } else if (has_lora) {
     // ------------------------------------------------------------ z operand builder (warps 6..9)
     const int btid = threadIdx.x - 192;  // 0..127
+    const int bwarp = warp - 6;
     const int nch = p.R_pad >> 3;        // 16-byte chunks of one operand row that the MMAs read
     uint32_t count = 0;                  // K blocks so far: stage = count % stages
     uint32_t gophase = 0;                // one parity bit per stage for zgo_bar
     bool ok = true, waited = false;
+    if (p.mode == kModeDecode) {
+      // The batch's adapters (paper Section 3.4: one u-batch per adapter), distinct and ascending,
+      // straight from the caller's ids so that the B_a tiles can be fetched before the shrink
+      // kernel has finished.  Thread b looks after tokens b and b + 128.
+      // Keys (id << 8 | token) of the tokens that carry an adapter are sorted (bitonic, BN keys);
+      // the first key of every id that names a loaded slot joins the list.
+      const int nk = p.BN;  // a power of two, 32..256
+      for (int t = btid; t < 256; t += 128) {
+        int32_t a = -1;
+        if (t < p.T) {
+          a = p.ids[t];
+          if (a < -1 || a >= p.n_slots) a = -1;
+        }
+        s_vid[t] = a;
+        s_key[t] = a >= 0 ? ((static_cast<uint32_t>(a) << 8) | static_cast<uint32_t>(t)) : 0xFFFFFFFFu;
+      }
+      named_bar_sync(2, 128);
+      for (int k = 2; k <= nk; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+          for (int i = btid; i < nk; i += 128) {
+            const int ixj = i ^ j;
+            if (ixj > i) {
+              const uint32_t ka = s_key[i], kb = s_key[ixj];
+              if ((ka > kb) == ((i & k) == 0)) {
+                s_key[i] = kb;
+                s_key[ixj] = ka;
+              }
+            }
+          }
+          named_bar_sync(2, 128);
+        }
+      }
+      for (int i = btid; i < nk; i += 128) {
+        const uint32_t key = s_key[i];
+        bool head = key != 0xFFFFFFFFu && (i == 0 || (s_key[i - 1] >> 8) != (key >> 8));
+        if (head) head = p.slots[key >> 8].rank > 0;  // empty slots stay base-only (the shrink flags them)
+        s_head[i] = head ? 1 : 0;
+      }
+      named_bar_sync(2, 128);
+      if (bwarp == 0) {  // 32 lanes x 8 consecutive keys: positions by a warp prefix sum
+        int c = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) c += (lane * 8 + q < nk) ? s_head[lane * 8 + q] : 0;
+        int incl = c;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const int o = __shfl_up_sync(0xffffffffu, incl, d);
+          if (lane >= d) incl += o;
+        }
+        int pos = incl - c;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const int i = lane * 8 + q;
+          if (i < nk && s_head[i]) s_lg[pos++] = static_cast<int32_t>(s_key[i] >> 8);
+        }
+        if (lane == 31) *s_nlg = incl;
+      }
+      named_bar_sync(2, 128);
+      if (btid == 0) ptx::mbar_arrive(lg_bar);
+    }
     for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
       const TileCoord tc = tile_coord(p, tile);
       count += static_cast<uint32_t>(tc.kb1 - tc.kb0);
-      if (!waited) {  // z and the adapter lists come from the kernels before this one
+      if (!waited) {  // z (and in prefill the tile lists) come from the kernels before this one
         ptx::pdl_wait_prior_grids();
         waited = true;
       }
-      const LoraList ll = lora_list(p, tc);
-      const int rows = (p.mode == kModePrefill) ? kTileM : p.BN;
+      const LoraList ll = lora_list(p, tc, s_lg, s_nlg);
       const int tok0 = (p.mode == kModePrefill) ? tc.row_r : 0;
       const uint32_t region = (p.mode == kModePrefill) ? 0u : r_bytes;
       // The ids of this thread's rows do not change over the tile's LoRA blocks, so their z is
       // fetched once per tile (while the base K blocks stream) and kept as packed bf16.
       int32_t id_lo = -1, id_hi = -1;
-      if (tok0 + btid < p.T) id_lo = p.ids_valid[tok0 + btid];
-      if (rows > 128 && tok0 + btid + 128 < p.T) id_hi = p.ids_valid[tok0 + btid + 128];
+      if (p.mode == kModeDecode) {
+        id_lo = s_vid[btid];
+        if (kMinBlocks == 1) id_hi = s_vid[btid + 128];  // the two-per-SM variant runs with BN <= 128
+      } else if (tok0 + btid < p.T) {
+        id_lo = p.ids_valid[tok0 + btid];
+      }
       uint4 z_lo[8], z_hi[8];
       if (ll.e0 < ll.e1) {
         if (id_lo >= 0) load_z_packed(p, tok0 + btid, p.slots[id_lo].rank, z_lo);
-        if (id_hi >= 0) load_z_packed(p, tok0 + btid + 128, p.slots[id_hi].rank, z_hi);
+        if (kMinBlocks == 1 && id_hi >= 0) load_z_packed(p, tok0 + btid + 128, p.slots[id_hi].rank, z_hi);
       }
       for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
         const int32_t a = ll.list[e];
-        if (p.slots[a].rank <= 0) continue;
+        if (p.mode != kModeDecode && p.slots[a].rank <= 0) continue;
         const uint32_t stage = count % nstages;
         ++count;
         if (!ptx::mbar_wait(&zgo_bar[stage], (gophase >> stage) & 1u) || *abort_flag) {
@@ -482,25 +635,29 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         }
         gophase ^= 1u << stage;
         uint8_t *dst = smem + static_cast<size_t>(stage) * stage_bytes + region;
-        // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
-        if (btid < rows) {
+        // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8.
+        // Prefill: all 128 token rows are written.  Decode: warp w owns the 32-token column
+        // blocks w and 4 + w and writes a block only if one of its tokens uses this adapter.
+        const bool m_lo = id_lo == a, m_hi = id_hi == a;
+        const bool w_lo = p.mode == kModePrefill || __any_sync(0xffffffffu, m_lo);
+        const bool w_hi = kMinBlocks == 1 && p.mode == kModeDecode && __any_sync(0xffffffffu, m_hi);
+        if (w_lo) {
           uint8_t *drow = dst + btid * 128;
-          const bool match = id_lo == a;
 #pragma unroll
           for (int c = 0; c < 8; ++c)
             if (c < nch)
               *reinterpret_cast<uint4 *>(drow + ((c ^ (btid & 7)) << 4)) =
-                  match ? z_lo[c] : make_uint4(0u, 0u, 0u, 0u);
+                  m_lo ? z_lo[c] : make_uint4(0u, 0u, 0u, 0u);
         }
-        if (btid + 128 < rows) {
+        if (w_hi) {
           uint8_t *drow = dst + (btid + 128) * 128;
-          const bool match = id_hi == a;
 #pragma unroll
           for (int c = 0; c < 8; ++c)
             if (c < nch)
               *reinterpret_cast<uint4 *>(drow + ((c ^ (btid & 7)) << 4)) =
-                  match ? z_hi[c] : make_uint4(0u, 0u, 0u, 0u);
+                  m_hi ? z_hi[c] : make_uint4(0u, 0u, 0u, 0u);
         }
+        if (lane == 0) s_cmask[stage * 4 + bwarp] = static_cast<uint8_t>((w_lo ? 1 : 0) | (w_hi ? 2 : 0));
         fence_proxy_async_smem();  // make the generic-proxy writes visible to the tensor core
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&zfull_bar[stage]);
@@ -542,6 +699,15 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         }
       }
     }
+    float *s_z = reinterpret_cast<float *>(smem + static_cast<size_t>(p.BN) * kTileM * 4);  // [cols_per][R_pad]
+    if (epi && p.expand_in_reduce) {
+      // z of this owner's tokens: the shrink kernel has to be complete from here on
+      ptx::pdl_wait_prior_grids();
+      for (int i = etid; i < cols_per * p.R_pad; i += 128) {
+        const int t = static_cast<int>(my_rank) * cols_per + i / p.R_pad;
+        s_z[i] = t < p.T ? __ldcg(p.zws + static_cast<size_t>(t) * p.R_pad + (i % p.R_pad)) : 0.f;
+      }
+    }
     __syncwarp();
     cluster_sync_all();
     if (epi) {
@@ -556,6 +722,39 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         for (int sp = 0; sp < p.splits; ++sp) {
           const float4 w = *reinterpret_cast<const float4 *>(buf + ((sp * cols_per + cl) * kTileM + r4));
           acc4.x += w.x; acc4.y += w.y; acc4.z += w.z; acc4.w += w.w;
+        }
+        if (p.expand_in_reduce) {
+          // expand on the CUDA cores: y[t][j..j+3] += B_a[j..j+3][0..r) . z[t]  (z carries s_a)
+          const int32_t a = s_vid[cl], rank = s_lg[cl];  // stored by the epilogue warps at the start
+          if (a >= 0) {
+            const uint4 *Brow = reinterpret_cast<const uint4 *>(
+                p.B_pool + (static_cast<size_t>(a) * p.h_out + j) * p.R_pad);
+            const int nch = p.R_pad >> 3;
+            const float *zt = s_z + cl * p.R_pad;
+            float add[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              if (c < nch && c * 8 < rank) {
+                uint4 b[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) b[r] = __ldg(Brow + r * nch + c);
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                  float s4 = add[r];
+                  s4 = fmaf(ptx::bf16_lo(b[r].x), zt[c * 8 + 0], s4);
+                  s4 = fmaf(ptx::bf16_hi(b[r].x), zt[c * 8 + 1], s4);
+                  s4 = fmaf(ptx::bf16_lo(b[r].y), zt[c * 8 + 2], s4);
+                  s4 = fmaf(ptx::bf16_hi(b[r].y), zt[c * 8 + 3], s4);
+                  s4 = fmaf(ptx::bf16_lo(b[r].z), zt[c * 8 + 4], s4);
+                  s4 = fmaf(ptx::bf16_hi(b[r].z), zt[c * 8 + 5], s4);
+                  s4 = fmaf(ptx::bf16_lo(b[r].w), zt[c * 8 + 6], s4);
+                  s4 = fmaf(ptx::bf16_hi(b[r].w), zt[c * 8 + 7], s4);
+                  add[r] = s4;
+                }
+              }
+            }
+            acc4.x += add[0]; acc4.y += add[1]; acc4.z += add[2]; acc4.w += add[3];
+          }
         }
         uint2 o;
         o.x = ptx::pack_bf16x2(acc4.x, acc4.y);
@@ -574,7 +773,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
 }
 
 cudaError_t gemm_set_smem_limit(size_t smem_bytes) {
-  return cudaFuncSetAttribute(lora_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(lora_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(smem_bytes));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(lora_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               static_cast<int>(smem_bytes));
 }
 
@@ -582,7 +784,10 @@ cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col
                         const CUtensorMap &tmap_b, const GemmParams &p, int32_t grid,
                         size_t smem_bytes, bool pdl, cudaStream_t stream) {
   const int cluster = (p.mode == kModeDecode && p.splits > 1) ? p.splits : 1;
-  return launch_ex(lora_gemm_kernel, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster,
+  if (smem_bytes * 2 <= 225 * 1024 && p.BN <= 128)  // two CTAs fit an SM: registers within half the file
+    return launch_ex(lora_gemm_kernel<2>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster,
+                     tmap_row, tmap_col, tmap_b, p);
+  return launch_ex(lora_gemm_kernel<1>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster,
                    tmap_row, tmap_col, tmap_b, p);
 }
 

@@ -66,8 +66,12 @@ struct GemmParams {
   int32_t n_ntiles;    // prefill: W row tiles of BN
   int32_t R_pad;       // slot block rank stride
   int32_t zsplits;     // partial z planes the consumer sums
+  int32_t expand_in_reduce;  // decode, small batches: B_a z is added by the owners of the cluster
+                             // reduction on the CUDA cores instead of by LoRA K blocks
   int32_t max_tokens;  // row stride of the z / plan workspaces
   const int32_t *ids_valid;
+  const int32_t *ids;       // decode: the caller's ids (validated again inside the kernel)
+  int32_t n_slots;
   const SlotRow *slots;
   const uint16_t *B_pool;   // [S][h_out][R_pad]
   const float *zws;         // [zsplits][max_tokens][R_pad]   (read by the prefill epilogue)
@@ -75,7 +79,6 @@ struct GemmParams {
   uint16_t *y;              // [T][h_out]
   const int32_t *sgmv_tiles;
   const int32_t *counts;
-  const int32_t *lg_adapter;  // decode: LoRA groups of the batch
   const int32_t *mt_count;    // prefill: per 128-token tile
   const int32_t *mt_list;
   uint32_t *status;

@@ -167,7 +167,7 @@ __device__ __forceinline__ int block_scan_256(int v, int *wt /* smem[9] */, int 
   return res;
 }
 
-constexpr int kDsDepth = 4;                         // ring stages per warp
+constexpr int kDsMaxDepth = 4;                      // ring stages per warp: 4, or 2 for small batches
 constexpr int kDsRowBytes = kShrinkStepElems * 2;   // 512: one row segment of one K step
 constexpr int kDsStageBytes = (8 + kDsTok) * kDsRowBytes;  // 8 rows of A, then up to 4 rows of x
 
@@ -176,7 +176,7 @@ constexpr int kDsStageBytes = (8 + kDsTok) * kDsRowBytes;  // 8 rows of A, then 
 // in flight with TMA copies (one box of 8 x 512 bytes of A and one 512-byte row of x per token)
 // into the warp's private ring; columns past h_in arrive as zeros.  `phase` holds one parity bit
 // per ring stage and lives across calls.  Returns false if a wait gave up.
-template <int NT>
+template <int NT, int kDsDepth>
 __device__ __forceinline__ bool shrink_rows8(const CUtensorMap *tmap_a, const CUtensorMap *tmap_x,
                                              int32_t slot, int32_t row0, const int32_t (&tok)[kDsTok],
                                              int step0, int step1, uint8_t *ring, uint64_t *bars,
@@ -225,8 +225,13 @@ __device__ __forceinline__ int atomic_add_acq_rel(int32_t *p, int v) {
   asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
   return old;
 }
-constexpr size_t kDsRingBytes = static_cast<size_t>(kShrinkThreads / 32) * kDsDepth * kDsStageBytes + 1024;
+constexpr size_t ds_ring_bytes(int depth) {
+  return static_cast<size_t>(kShrinkThreads / 32) * depth * kDsStageBytes + 1024;
+}
 
+// kDsDepth = 4 fills an SM's shared memory (large batches: bandwidth); kDsDepth = 2 leaves room
+// for a CTA of the base-product kernel beside it (small batches: the two kernels overlap).
+template <int kDsDepth>
 __global__ void __launch_bounds__(kShrinkThreads, 1)
 decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_x,
                      const int32_t *__restrict__ ids, const SlotRow *__restrict__ slots,
@@ -234,7 +239,7 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                      int32_t T, int32_t h_in, int32_t R_pad, int32_t n_slots, int32_t max_tokens,
                      int32_t target_items, uint32_t *status) {
   extern __shared__ uint8_t s_ring_raw[];  // [warp][stage][8 A rows + 4 x rows][512 bytes]
-  __shared__ uint64_t s_bars[kShrinkThreads / 32][kDsDepth];
+  __shared__ uint64_t s_bars[kShrinkThreads / 32][kDsMaxDepth];
   __shared__ int32_t s_id[256];        // validated id of each token
   __shared__ int32_t s_grp[256];       // group (in order of first appearance) of a group's first token
   __shared__ int32_t s_gadapter[256];  // adapter of each group
@@ -243,6 +248,8 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   __shared__ int32_t s_cnt[256];
   __shared__ int32_t s_bgrp[256];      // token blocks: group and first position in s_gtok
   __shared__ int32_t s_btok[256];
+  __shared__ int32_t s_grank[256];     // rank and scale of each group's slot
+  __shared__ float s_gscale[256];
   __shared__ int s_wt[9];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -250,8 +257,9 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   if (tid == 0) {
     ptx::prefetch_tensormap(&tmap_a);
     ptx::prefetch_tensormap(&tmap_x);
-    for (int w = 0; w < kShrinkThreads / 32; ++w)
-      for (int d = 0; d < kDsDepth; ++d) ptx::mbar_init(&s_bars[w][d], 1);
+  }
+  if (lane < kDsDepth) {  // every warp sets up its own ring barriers
+    ptx::mbar_init(&s_bars[warp][lane], 1);
     ptx::fence_barrier_init();
   }
 
@@ -292,6 +300,11 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   }
   __syncthreads();
   int tot;
+  if (tid < G) {  // in flight during the prefix sums below
+    const SlotRow row = slots[s_gadapter[tid]];
+    s_grank[tid] = row.rank;
+    s_gscale[tid] = row.scale;
+  }
   const int n_mine = tid < G ? s_cnt[tid] : 0;
   const int gs = block_scan_256(n_mine, s_wt, tot);
   if (tid < G) s_gstart[tid] = gs;
@@ -318,10 +331,14 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   const int spc = (n_ksteps + KS - 1) / KS;
   KS = (n_ksteps + spc - 1) / spc;
 
-  ptx::pdl_wait_prior_grids();  // earlier kernels may still read the plan and z
+  // Earlier kernels on the stream may still read the plan and z, so every write to them below comes
+  // after griddepcontrol.wait; the operand loads (the pool and x are not written by this library's
+  // kernels) start before it.
+  const bool publisher = blockIdx.x == gridDim.x - 1;
+  if (publisher) ptx::pdl_wait_prior_grids();
 
   // ---- the last CTA publishes the plan in canonical order (ids ascending, -1 first)
-  if (blockIdx.x == gridDim.x - 1) {
+  if (publisher) {
     if (any_bad && tid == 0) atomicOr(pv.status, EDGELORA_STATUS_BAD_ADAPTER_ID);
     const uint32_t key = (static_cast<uint32_t>(a + 1) << 16) | static_cast<uint32_t>(tid);
     int rp = 0;
@@ -382,7 +399,7 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                   static_cast<size_t>(warp) * kDsDepth * kDsStageBytes;
   uint64_t *bars = s_bars[warp];
   uint32_t phase = 0;
-  bool ok = true;
+  bool ok = true, waited = publisher;
   // Items are drawn from a ticket counter so that warps stay busy whatever the items cost; the
   // next ticket is drawn before the current item is processed.  The very last draw of the launch
   // (item number n_items + warps - 1) puts the counter back to zero.
@@ -400,14 +417,15 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     const int bi = bc / KS, c = bc - bi * KS;
     const int gi = s_bgrp[bi];
     const int ad = s_gadapter[gi];
-    const SlotRow row = slots[ad];
+    const int rank = s_grank[gi];
+    const float scale = s_gscale[gi];
     const int gt0 = s_gstart[gi], g_end = s_gstart[gi + 1];
     const int t0 = s_btok[bi], t1 = min(t0 + kDsBlockTok, g_end);
-    if (row.rank <= 0) {
+    if (rank <= 0) {
       if (lane == 0 && c == 0 && rg == 0 && t0 == gt0) atomicOr(status, EDGELORA_STATUS_SLOT_EMPTY);
       continue;
     }
-    const int n_rg = (row.rank + 7) >> 3;  // live groups of eight rows
+    const int n_rg = (rank + 7) >> 3;  // live groups of eight rows
     if (rg >= n_rg) continue;               // rows past the rank are zero padding: nothing to do
     const int step0 = c * spc, step1 = min(n_ksteps, step0 + spc);
     const int q = lane & 3, r = rg * 8 + (lane >> 2);
@@ -419,10 +437,10 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       int32_t tok[kDsTok];
 #pragma unroll
       for (int qq = 0; qq < kDsTok; ++qq) tok[qq] = s_gtok[tb + min(qq, nt - 1)];
-      if (nt == 1) ok = shrink_rows8<1>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
-      else if (nt == 2) ok = shrink_rows8<2>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
-      else if (nt == 3) ok = shrink_rows8<3>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
-      else ok = shrink_rows8<4>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
+      if (nt == 1) ok = shrink_rows8<1, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
+      else if (nt == 2) ok = shrink_rows8<2, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
+      else if (nt == 3) ok = shrink_rows8<3, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
+      else ok = shrink_rows8<4, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       // lane L ends with the sum over lanes of value L (= row L / 4, token L % 4)
@@ -436,9 +454,13 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
           acc[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
         }
       }
+      if (!waited) {  // first write of this warp to memory that earlier kernels may read
+        ptx::pdl_wait_prior_grids();
+        waited = true;
+      }
       if (q < nt)
         zws[(KS > 1 ? c : kMaxZSplits) * zplane + static_cast<size_t>(s_gtok[tb + q]) * R_pad + r] =
-            row.scale * acc[0];
+            scale * acc[0];
     }
     if (!ok) break;
     if (KS > 1) {
@@ -483,12 +505,19 @@ cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &t
                                  cudaStream_t stream) {
   static bool configured = false;  // per process; the attribute is per function and device-wide
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(decode_shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(kDsRingBytes));
+    cudaError_t e = cudaFuncSetAttribute(decode_shrink_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(ds_ring_bytes(4)));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(decode_shrink_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(ds_ring_bytes(2)));
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  return launch_ex(decode_shrink_kernel, dim3(grid), dim3(kShrinkThreads), kDsRingBytes, stream, pdl, 1,
+  if (T <= 64)
+    return launch_ex(decode_shrink_kernel<2>, dim3(grid), dim3(kShrinkThreads), ds_ring_bytes(2), stream, pdl, 1,
+                     tmap_a, tmap_x, ids, slots, pv, zws, group_counters, T, h_in, R_pad, n_slots,
+                     max_tokens, target_items, status);
+  return launch_ex(decode_shrink_kernel<4>, dim3(grid), dim3(kShrinkThreads), ds_ring_bytes(4), stream, pdl, 1,
                    tmap_a, tmap_x, ids, slots, pv, zws, group_counters, T, h_in, R_pad, n_slots,
                    max_tokens, target_items, status);
 }
