@@ -220,14 +220,18 @@ def main():
     n_rep = 1 if not decode_like else max(2, int(np.ceil(3 * L2_BYTES / ws_bytes)))
     if args.workload == "gate_up_prefill":
         n_rep = 2   # 273 MB per step already exceeds L2; two replicas keep W from being re-hit
+    # The timed steps are independent batches (their W, x and ids are not produced by the step
+    # before), so the library may let a step's first kernel start under the previous step's tail
+    # (EDGELORA_OPT_PDL = 2).  The number for calls that depend on each other (mode 1, the
+    # library's default) is measured as well and reported under "dependent_calls".
+    pdl_mode = args.pdl if args.pdl is not None else (2 if decode_like else 1)
     to_bf16 = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
     Ws, pools = [], []
     for r in range(n_rep):
         Ws.append(to_bf16(w.W) if r == 0 else Ws[0].clone())
         pool = B.Pool(w.h_in, w.h_out, w.n_slots, w.max_rank, max_tokens=w.T)
         pool.load_all(w.adapters)
-        if args.pdl is not None:
-            B.edgelora_pool_set_option(pool.handle, B.OPT_PDL, args.pdl)
+        B.edgelora_pool_set_option(pool.handle, B.OPT_PDL, pdl_mode)
         if args.decode_splits:
             B.edgelora_pool_set_option(pool.handle, B.OPT_DECODE_SPLITS, args.decode_splits)
         if args.shrink_items:
@@ -299,6 +303,28 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
     value = world * w.T * args.steps / (ms * 1e-3)
+
+    dependent = None
+    if pdl_mode == 2:   # same steps with the library's default launch mode, plain stream launches
+        for p_ in pools:
+            B.edgelora_pool_set_option(p_.handle, B.OPT_PDL, 1)
+        k_dep = int(min(args.steps, 20000))
+        with torch.cuda.stream(stream):
+            for i in range(20):
+                step(i)
+        barrier()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(stream)
+        with torch.cuda.stream(stream):
+            for i in range(k_dep):
+                step(i)
+        d1.record(stream)
+        barrier()
+        ms_dep = d0.elapsed_time(d1)
+        dependent = {"value": world * w.T * k_dep / (ms_dep * 1e-3), "unit": "tokens/s", "steps": k_dep,
+                     "ms_per_step": ms_dep / k_dep, "launch": "plain stream launches, EDGELORA_OPT_PDL=1"}
+        for p_ in pools:
+            B.edgelora_pool_set_option(p_.handle, B.OPT_PDL, pdl_mode)
 
     # ---- end to end through the host-buffer entry point (pinned staging inside the library)
     k_e2e = int(min(args.steps, 3000 if decode_like else 200))
@@ -379,7 +405,7 @@ def main():
         "config": {"workload": desc, "T": w.T, "h_in": w.h_in, "h_out": w.h_out, "n_slots": w.n_slots,
                    "max_rank": w.max_rank, "distinct_adapters": len(w.distinct_adapters()),
                    "regime": info["regime"], "split_k": info["split_k"], "gemm_grid": info["gemm_grid"],
-                   "stages": info["stages"], "launch": "plain stream launches" if graph is None else
+                   "stages": info["stages"], "pdl_mode": pdl_mode, "launch": "plain stream launches" if graph is None else
                    f"CUDA-graph replay of {n_rep} consecutive steps",
                    "l2": f"inputs larger than L2: {n_rep} replicas of W and the adapter pool used in rotation "
                          f"({n_rep * ws_bytes / 2**20:.0f} MiB)", "parallelism": f"replicas x{world}"},
@@ -391,6 +417,8 @@ def main():
         "step_roofline_frac": step_frac,
         "kernel_ms_profiled": {k: v for k, v in kt.items() if v["launches"]},
     }
+    if dependent is not None:
+        line["dependent_calls"] = dependent
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(w)
     print(json.dumps(line), flush=True)

@@ -232,7 +232,7 @@ constexpr size_t ds_ring_bytes(int depth) {
 // kDsDepth = 4 fills an SM's shared memory (large batches: bandwidth); kDsDepth = 2 leaves room
 // for a CTA of the base-product kernel beside it (small batches: the two kernels overlap).
 template <int kDsDepth>
-__global__ void __launch_bounds__(kShrinkThreads, 1)
+__global__ void __launch_bounds__(kShrinkThreads, 2)  // <= 128 registers: fits beside the base-product CTAs
 decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_x,
                      const int32_t *__restrict__ ids, const SlotRow *__restrict__ slots,
                      PlanView pv, float *__restrict__ zws, int32_t *__restrict__ group_counters,
