@@ -128,6 +128,22 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(value, world, device):
+    """The slowest rank's time: every rank runs its own replica, the job is as fast as the slowest."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(tokens_per_rank_step, steps, world, seconds):
+    """Whole-job throughput of `world` replicas that each did `steps` steps in `seconds` (max over ranks)."""
+    return world * tokens_per_rank_step * steps / seconds
+
+
 def time_oracle(w, tokens, reps):
     import oracle
     from oracle import AdapterSet
@@ -298,11 +314,8 @@ def main():
     barrier()
     windows.append((t_start, time.time()))
     ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * w.T * args.steps / (ms * 1e-3)
+    ms = max_over_ranks(ms, world, "cuda")
+    value = aggregate_tokens_per_s(w.T, args.steps, world, ms * 1e-3)
 
     dependent = None
     if pdl_mode == 2:   # same steps with the library's default launch mode, plain stream launches
@@ -340,10 +353,7 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     windows.append((t_start, time.time()))
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s, world, "cuda")
     e2e = {"value": world * w.T * k_e2e / e2e_s, "unit": "tokens/s", "steps": k_e2e,
            "h2d_bytes_per_step": int(w.x.nbytes + w.ids.nbytes), "d2h_bytes_per_step": int(y_host.nbytes),
            "api": "edgelora_lora_linear_host"}
