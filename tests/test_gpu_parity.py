@@ -87,6 +87,19 @@ def test_ragged_ranks(max_rank, ranks, T):
     assert_parity(run_gpu(w), oracle_of(w), f"ranks {ranks}")
 
 
+@pytest.mark.parametrize("T,h_in,h_out,max_rank,ranks", [
+    (24, 2048, 1024, 64, [64, 40, 8, 33, 64]),      # 8 K splits, expand by the reduction owners, rank 64
+    (64, 2048, 1024, 16, [16, 8, 3, 16, 12, 16]),   # same path at its largest token count
+    (64, 1024, 2048, 64, [64, 64, 17]),             # too many B loads per owner: LoRA K blocks, 64 tokens
+    (200, 1024, 1024, 32, [32, 8, 24, 16]),         # LoRA K blocks with both halves of the 256-token tile
+])
+def test_small_and_medium_decode_paths(T, h_in, h_out, max_rank, ranks):
+    w = random_workload(T + h_out + max_rank, T, h_in, h_out, ranks=ranks, max_rank=max_rank)
+    y, plan = run_gpu(w, 1, return_plan=True)
+    assert_parity(y, oracle_of(w), f"decode T={T} {h_in}->{h_out} ranks {ranks}")
+    check_plan(plan, w.ids, w.n_slots)
+
+
 @pytest.mark.parametrize("mode", ["base", "0", "2"])
 @pytest.mark.parametrize("T", [40, 384])
 def test_degenerate_batches(mode, T):
