@@ -263,6 +263,9 @@ def main():
         B.edgelora_lora_linear(pools[r].handle, Ws[r], x, ids, ys[r], stream)
 
     graph = None
+    # a graph holds several rotations of the replicas, so that the gap between two replays
+    # (about 20 us) is spread over many steps
+    per_graph = n_rep * (10 if decode_like else 1)
     with torch.cuda.stream(stream):
         for i in range(args.warmup):
             step(i)
@@ -274,7 +277,7 @@ def main():
         if not args.no_graph:
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph, stream=stream):
-                for i in range(n_rep):
+                for i in range(per_graph):
                     step(i)
             for _ in range(3):
                 graph.replay()
@@ -284,9 +287,9 @@ def main():
     def run_steps(k):
         with torch.cuda.stream(stream):
             if graph is not None:
-                for _ in range(k // n_rep):
+                for _ in range(k // per_graph):
                     graph.replay()
-                for i in range(k % n_rep):
+                for i in range(k % per_graph):
                     step(i)
             else:
                 for i in range(k):
@@ -416,7 +419,7 @@ def main():
                    "max_rank": w.max_rank, "distinct_adapters": len(w.distinct_adapters()),
                    "regime": info["regime"], "split_k": info["split_k"], "gemm_grid": info["gemm_grid"],
                    "stages": info["stages"], "pdl_mode": pdl_mode, "launch": "plain stream launches" if graph is None else
-                   f"CUDA-graph replay of {n_rep} consecutive steps",
+                   f"CUDA-graph replay of {per_graph} consecutive steps",
                    "l2": f"inputs larger than L2: {n_rep} replicas of W and the adapter pool used in rotation "
                          f"({n_rep * ws_bytes / 2**20:.0f} MiB)", "parallelism": f"replicas x{world}"},
         "clocks": sampler.summary(windows),

@@ -699,67 +699,95 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         }
       }
     }
-    float *s_z = reinterpret_cast<float *>(smem + static_cast<size_t>(p.BN) * kTileM * 4);  // [cols_per][R_pad]
-    if (epi && p.expand_in_reduce) {
-      // z of this owner's tokens: the shrink kernel has to be complete from here on
-      ptx::pdl_wait_prior_grids();
-      for (int i = etid; i < cols_per * p.R_pad; i += 128) {
-        const int t = static_cast<int>(my_rank) * cols_per + i / p.R_pad;
-        s_z[i] = t < p.T ? __ldcg(p.zws + static_cast<size_t>(t) * p.R_pad + (i % p.R_pad)) : 0.f;
-      }
-    }
     __syncwarp();
     cluster_sync_all();
     if (epi) {
       const float *buf = reinterpret_cast<const float *>(smem);
-      const int n_units = cols_per * 32;  // (token, 4 adjacent W rows)
-      for (int u = etid; u < n_units; u += 128) {
-        const int cl = u >> 5, r4 = (u & 31) << 2;
-        const int t = static_cast<int>(my_rank) * cols_per + cl;
-        const int j = blockIdx.x / p.splits * kTileM + r4;
-        if (t >= p.T || j >= p.h_out) continue;  // h_out is a multiple of 8: 4 rows are all in or out
+      const int n_units = cols_per * 32;  // unit = (token, 4 adjacent W rows)
+      const int row0 = blockIdx.x / p.splits * kTileM;
+      auto sum_partials = [&](int cl, int r4) {
         float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int sp = 0; sp < p.splits; ++sp) {
           const float4 w = *reinterpret_cast<const float4 *>(buf + ((sp * cols_per + cl) * kTileM + r4));
           acc4.x += w.x; acc4.y += w.y; acc4.z += w.z; acc4.w += w.w;
         }
-        if (p.expand_in_reduce) {
-          // expand on the CUDA cores: y[t][j..j+3] += B_a[j..j+3][0..r) . z[t]  (z carries s_a)
+        return acc4;
+      };
+      auto store4 = [&](int t, int j, const float4 &v) {
+        uint2 o;
+        o.x = ptx::pack_bf16x2(v.x, v.y);
+        o.y = ptx::pack_bf16x2(v.z, v.w);
+        *reinterpret_cast<uint2 *>(p.y + static_cast<size_t>(t) * p.h_out + j) = o;
+      };
+      if (!p.expand_in_reduce) {
+        for (int u = etid; u < n_units; u += 128) {
+          const int cl = u >> 5, r4 = (u & 31) << 2;
+          const int t = static_cast<int>(my_rank) * cols_per + cl, j = row0 + r4;
+          if (t >= p.T || j >= p.h_out) continue;  // h_out is a multiple of 8: 4 rows are all in or out
+          store4(t, j, sum_partials(cl, r4));
+        }
+      } else {
+        // Small batches.  Everything that does not need z first: the base product's sums stay in
+        // registers (at most 4 units per thread: cols_per <= 16).  Then wait for the shrink kernel
+        // (and for earlier readers of y), fetch z and the B_a rows in one round trip, add
+        // B_a[j..j+3][0..r) . z[t] in fp32 (z carries s_a) and write y.
+        float4 base[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int u = etid + i * 128;
+          base[i] = u < n_units ? sum_partials(u >> 5, (u & 31) << 2) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        ptx::pdl_wait_prior_grids();
+        const int nch = p.R_pad >> 3;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int u = etid + i * 128;
+          if (u >= n_units) break;
+          const int cl = u >> 5, r4 = (u & 31) << 2;
+          const int t = static_cast<int>(my_rank) * cols_per + cl, j = row0 + r4;
+          if (t >= p.T || j >= p.h_out) continue;
+          float4 acc4 = base[i];
           const int32_t a = s_vid[cl], rank = s_lg[cl];  // stored by the epilogue warps at the start
           if (a >= 0) {
             const uint4 *Brow = reinterpret_cast<const uint4 *>(
                 p.B_pool + (static_cast<size_t>(a) * p.h_out + j) * p.R_pad);
-            const int nch = p.R_pad >> 3;
-            const float *zt = s_z + cl * p.R_pad;
+            const float4 *zt = reinterpret_cast<const float4 *>(p.zws + static_cast<size_t>(t) * p.R_pad);
             float add[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int c0 = 0; c0 < nch && c0 * 8 < rank; c0 += 2) {
+              uint4 b[2][4];
+              float4 z4[2][2];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              if (c < nch && c * 8 < rank) {
-                uint4 b[4];
+              for (int cc = 0; cc < 2; ++cc) {  // two chunks of 8 rank values: 12 loads in flight
+                const int c = c0 + cc;
+                const bool on = c < nch && c * 8 < rank;
 #pragma unroll
-                for (int r = 0; r < 4; ++r) b[r] = __ldg(Brow + r * nch + c);
+                for (int r = 0; r < 4; ++r) b[cc][r] = on ? __ldg(Brow + r * nch + c) : make_uint4(0u, 0u, 0u, 0u);
+                z4[cc][0] = on ? __ldcg(zt + 2 * c) : make_float4(0.f, 0.f, 0.f, 0.f);
+                z4[cc][1] = on ? __ldcg(zt + 2 * c + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+              }
+#pragma unroll
+              for (int cc = 0; cc < 2; ++cc) {
+                const float4 u0 = z4[cc][0], u1 = z4[cc][1];
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
+                  const uint4 bb = b[cc][r];
                   float s4 = add[r];
-                  s4 = fmaf(ptx::bf16_lo(b[r].x), zt[c * 8 + 0], s4);
-                  s4 = fmaf(ptx::bf16_hi(b[r].x), zt[c * 8 + 1], s4);
-                  s4 = fmaf(ptx::bf16_lo(b[r].y), zt[c * 8 + 2], s4);
-                  s4 = fmaf(ptx::bf16_hi(b[r].y), zt[c * 8 + 3], s4);
-                  s4 = fmaf(ptx::bf16_lo(b[r].z), zt[c * 8 + 4], s4);
-                  s4 = fmaf(ptx::bf16_hi(b[r].z), zt[c * 8 + 5], s4);
-                  s4 = fmaf(ptx::bf16_lo(b[r].w), zt[c * 8 + 6], s4);
-                  s4 = fmaf(ptx::bf16_hi(b[r].w), zt[c * 8 + 7], s4);
+                  s4 = fmaf(ptx::bf16_lo(bb.x), u0.x, s4);
+                  s4 = fmaf(ptx::bf16_hi(bb.x), u0.y, s4);
+                  s4 = fmaf(ptx::bf16_lo(bb.y), u0.z, s4);
+                  s4 = fmaf(ptx::bf16_hi(bb.y), u0.w, s4);
+                  s4 = fmaf(ptx::bf16_lo(bb.z), u1.x, s4);
+                  s4 = fmaf(ptx::bf16_hi(bb.z), u1.y, s4);
+                  s4 = fmaf(ptx::bf16_lo(bb.w), u1.z, s4);
+                  s4 = fmaf(ptx::bf16_hi(bb.w), u1.w, s4);
                   add[r] = s4;
                 }
               }
             }
             acc4.x += add[0]; acc4.y += add[1]; acc4.z += add[2]; acc4.w += add[3];
           }
+          store4(t, j, acc4);
         }
-        uint2 o;
-        o.x = ptx::pack_bf16x2(acc4.x, acc4.y);
-        o.y = ptx::pack_bf16x2(acc4.z, acc4.w);
-        *reinterpret_cast<uint2 *>(p.y + static_cast<size_t>(t) * p.h_out + j) = o;
       }
     }
   }

@@ -679,11 +679,16 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     plan->last_T = T;
     {
       ProfScope ps(p, 1, stream);
+      // When calls overlap (EDGELORA_OPT_PDL = 2) a small batch's shrink runs under the previous
+      // call's base product, so its length does not matter but its tail does: one K chunk per
+      // item (no pass that adds chunks) and few CTAs (they take SM resources from the base product).
+      const bool overlapped = pdl_first && T <= 64;
+      const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : (overlapped ? 1 : 4 * 8 * p->sms);
       // at most T token blocks x (R / 8) row groups x K chunks warp items, eight warps per CTA
       const int n_ksteps = (h_in + kShrinkStepElems - 1) / kShrinkStepElems;
-      const int max_items = std::min(T, p->cfg.n_slots) * (R / 8) * std::max(1, std::min(kMaxZSplits, n_ksteps / 4));
-      const int grid = std::max(1, std::min(p->sms, (max_items + 7) / 8));
-      const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : 4 * 8 * p->sms;  // warp items
+      const int max_chunks = target == 1 ? 1 : std::max(1, std::min(kMaxZSplits, n_ksteps / 4));
+      const int max_items = std::min(T, p->cfg.n_slots) * (R / 8) * max_chunks;
+      const int grid = std::max(1, std::min(p->sms - 1, (max_items + 7) / 8)) + 1;  // + the publishing CTA
       const CUtensorMap *ma, *mx;
       int rc = get_tmap(p, &ma, p->A_pool, h_in, R, p->cfg.n_slots, 8, kShrinkStepElems);
       if (rc) return rc;
@@ -721,7 +726,7 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     g.stages = stages_for(N, kb_per + 8, budget);
     // Small batches: the expand moves to the owners of the cluster reduction (at most 64 16-byte
     // loads of B per thread), so the main loop does not depend on the shrink at all.
-    g.expand_in_reduce = (splits > 1 && N <= 64 && (N / splits) * (R / 8) <= 64) ? 1 : 0;
+    g.expand_in_reduce = (splits > 1 && N <= 64 && (N / splits) <= 16 && (N / splits) * (R / 8) <= 64) ? 1 : 0;
     if (g.expand_in_reduce && p->opt_decode_splits == 0) {
       // one CTA per SM leaves room for the shrink kernel's CTAs, so that the two kernels run side
       // by side (measured on 4096 -> 4096, T = 32: 18.4 us per step with 4 splits, 24.4 with 8)
@@ -729,7 +734,7 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
       kb_per = (kb_total + splits - 1) / splits;
       g.splits = splits;
       g.kb_per = kb_per;
-      g.expand_in_reduce = (splits > 1 && (N / splits) * (R / 8) <= 64) ? 1 : 0;
+      g.expand_in_reduce = (splits > 1 && (N / splits) <= 16 && (N / splits) * (R / 8) <= 64) ? 1 : 0;
       g.stages = stages_for(N, kb_per + 8, budget);
     }
     // the cluster's reduction buffer (N x 128 fp32, plus z of the owner's tokens) overlays the ring

@@ -403,9 +403,10 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   // Items are drawn from a ticket counter so that warps stay busy whatever the items cost; the
   // next ticket is drawn before the current item is processed.  The very last draw of the launch
   // (item number n_items + warps - 1) puts the counter back to zero.
-  const int warps_total = gridDim.x * (kShrinkThreads / 32);
+  // (the publishing CTA takes no items: nothing that the next kernel waits for queues behind it)
+  const int warps_total = (gridDim.x - 1) * (kShrinkThreads / 32);
   int32_t *ticket = group_counters + kDsTicket;
-  int item = blockIdx.x * (kShrinkThreads / 32) + warp;  // first round is static
+  int item = publisher ? n_items : blockIdx.x * (kShrinkThreads / 32) + warp;  // first round is static
   while (ok && item < n_items) {
     int next = 0;
     if (lane == 0) next = warps_total + atomicAdd(ticket, 1);
@@ -489,7 +490,7 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   }
   // Every warp stops at its first ticket >= n_items, so exactly n_items - (first round) + warps
   // draws happen; the one that drew the last ticket resets the counter for the next launch.
-  if (lane == 0 && ok) {
+  if (lane == 0 && ok && !publisher) {
     const int first_round = min(n_items, warps_total);
     const int last_ticket = warps_total + (n_items - first_round) + first_round - 1;
     if (item == last_ticket) *ticket = 0;
