@@ -335,11 +335,10 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   // after griddepcontrol.wait; the operand loads (the pool and x are not written by this library's
   // kernels) start before it.
   const bool publisher = blockIdx.x == gridDim.x - 1;
-  if (publisher) ptx::pdl_wait_prior_grids();
 
-  // ---- the last CTA publishes the plan in canonical order (ids ascending, -1 first)
+  // ---- the last CTA publishes the plan in canonical order (ids ascending, -1 first): everything
+  // is worked out in shared memory and registers first, the stores come after the wait
   if (publisher) {
-    if (any_bad && tid == 0) atomicOr(pv.status, EDGELORA_STATUS_BAD_ADAPTER_ID);
     const uint32_t key = (static_cast<uint32_t>(a + 1) << 16) | static_cast<uint32_t>(tid);
     int rp = 0;
     if (tid < T)
@@ -358,6 +357,12 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     int n_groups;
     const int gi = block_scan_256(head ? 1 : 0, s_wt, n_groups);
     const int has_base = (T > 0 && s_id[s_cnt[0]] < 0) ? 1 : 0;
+    const bool shead = tid < T && (tid == 0 || s_id[tid - 1] != a);
+    int n_segs;
+    const int si = block_scan_256(shead ? 1 : 0, s_wt, n_segs);
+
+    ptx::pdl_wait_prior_grids();
+    if (any_bad && tid == 0) atomicOr(pv.status, EDGELORA_STATUS_BAD_ADAPTER_ID);
     if (tid < T) {
       pv.ids_valid[tid] = a;
       pv.perm[tid] = tok;
@@ -368,11 +373,6 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         pv.group_adapter[gi] = ida;
         if (ida >= 0) pv.lg_adapter[gi - has_base] = ida;
       }
-    }
-    const bool shead = tid < T && (tid == 0 || s_id[tid - 1] != a);
-    int n_segs;
-    const int si = block_scan_256(shead ? 1 : 0, s_wt, n_segs);
-    if (tid < T) {
       pv.tok_seg[tid] = si + (shead ? 1 : 0) - 1;
       if (shead) {
         pv.seg_start[si] = tid;
