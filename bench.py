@@ -196,7 +196,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="q_proj_decode", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="q_proj_decode", choices=sorted(WORKLOADS) + ["full_projection_set"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of CUDA-graph replay")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -204,6 +204,17 @@ def main():
     ap.add_argument("--decode-splits", type=int, default=0, help="tuning: EDGELORA_OPT_DECODE_SPLITS")
     ap.add_argument("--shrink-items", type=int, default=0, help="tuning: EDGELORA_OPT_SHRINK_ITEMS")
     args = ap.parse_args()
+
+    if args.workload == "full_projection_set":   # configs[4]: 224 sites, its own driver
+        if args.impl == "reference" or int(os.environ.get("WORLD_SIZE", "1")) > 1:
+            raise SystemExit("full_projection_set: single GPU, --impl ours only")
+        import torch
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+        torch.cuda.set_device(0)
+        from paper_2507_01438_b200 import full_set_bench
+        print(json.dumps(full_set_bench.run(args, peaks(), ClockSampler, max_over_ranks)), flush=True)
+        return
 
     builder, bound, desc = WORKLOADS[args.workload]
     decode_like = bound == "hbm"
