@@ -195,10 +195,9 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   uint64_t *tempty_bar = tfull_bar + 2;           // [2]       epilogue -> MMA
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(tempty_bar + 2);
   volatile uint32_t *abort_flag = tmem_slot + 1;
-  // decode extras, 512 bytes after the barriers: which 32-token column blocks a LoRA K block
-  // touches, and the batch's adapter list derived from the ids by the builder warps
+  // decode extras, 512 bytes after the barriers: the batch's adapter list derived from the ids
+  // by the builder warps
   uint8_t *extra = reinterpret_cast<uint8_t *>(bars) + 512;
-  volatile uint8_t *s_cmask = extra;                                        // [stages][4]
   volatile int32_t *s_nlg = reinterpret_cast<volatile int32_t *>(extra + 64);
   uint64_t *lg_bar = reinterpret_cast<uint64_t *>(extra + 72);              // builder -> TMA, MMA
   int32_t *s_lg = reinterpret_cast<int32_t *>(extra + 128);                 // [256] ids ascending
@@ -378,26 +377,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
             const uint32_t sr = ptx::smem_u32(smem + static_cast<size_t>(stage) * stage_bytes);
             const uint64_t da = ptx::umma_desc_k128(sr);
             const uint64_t db = ptx::umma_desc_k128(sr + r_bytes);
-            if (p.mode == kModePrefill) {
-              for (int k = 0; k < lora_ksteps; ++k) ptx::umma_bf16(tmem_d, da + 2 * k, db + 2 * k, idesc, 1u);
-            } else {
-              // decode: only the 32-token column blocks that hold tokens of this adapter; the
-              // builder wrote those blocks of the z operand and left a flag per block
-              const uint32_t idesc32 = ptx::umma_idesc_bf16(kTileM, 32);
-#pragma unroll
-              for (int w = 0; w < 4; ++w) {
-                const uint32_t flags = s_cmask[stage * 4 + w];
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                  if (flags & (1u << h)) {
-                    const uint32_t cb = static_cast<uint32_t>(h * 4 + w);  // tokens [32 cb, 32 cb + 32)
-                    const uint64_t dbc = ptx::umma_desc_k128(sr + r_bytes + cb * 4096u);
-                    for (int k = 0; k < lora_ksteps; ++k)
-                      ptx::umma_bf16(tmem_d + cb * 32u, da + 2 * k, dbc + 2 * k, idesc32, 1u);
-                  }
-                }
-              }
-            }
+            // the whole z operand is there (rows of tokens on other adapters are zero), so one
+            // MMA per 16 rank columns covers every token: an MMA costs about the same whatever
+            // its N, and the issuing thread is what bounds a LoRA K block
+            for (int k = 0; k < lora_ksteps; ++k) ptx::umma_bf16(tmem_d, da + 2 * k, db + 2 * k, idesc, 1u);
             ptx::umma_commit(&empty_bar[stage]);
             if (++stage == nstages) {
               stage = 0;
@@ -636,11 +619,11 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         gophase ^= 1u << stage;
         uint8_t *dst = smem + static_cast<size_t>(stage) * stage_bytes + region;
         // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8.
-        // Prefill: all 128 token rows are written.  Decode: warp w owns the 32-token column
-        // blocks w and 4 + w and writes a block only if one of its tokens uses this adapter.
+        // Every token row the MMAs read is written: z of the tokens on this adapter, zeros for
+        // the others (prefill: the tile's 128 rows; decode: rows btid and btid + 128 below BN).
         const bool m_lo = id_lo == a, m_hi = id_hi == a;
-        const bool w_lo = p.mode == kModePrefill || __any_sync(0xffffffffu, m_lo);
-        const bool w_hi = kMinBlocks == 1 && p.mode == kModeDecode && __any_sync(0xffffffffu, m_hi);
+        const bool w_lo = p.mode == kModePrefill || btid < p.BN;
+        const bool w_hi = kMinBlocks == 1 && p.mode == kModeDecode && btid + 128 < p.BN;
         if (w_lo) {
           uint8_t *drow = dst + btid * 128;
 #pragma unroll
@@ -657,7 +640,6 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
               *reinterpret_cast<uint4 *>(drow + ((c ^ (btid & 7)) << 4)) =
                   m_hi ? z_hi[c] : make_uint4(0u, 0u, 0u, 0u);
         }
-        if (lane == 0) s_cmask[stage * 4 + bwarp] = static_cast<uint8_t>((w_lo ? 1 : 0) | (w_hi ? 2 : 0));
         fence_proxy_async_smem();  // make the generic-proxy writes visible to the tensor core
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&zfull_bar[stage]);

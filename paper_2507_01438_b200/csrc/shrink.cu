@@ -167,7 +167,7 @@ __device__ __forceinline__ int block_scan_256(int v, int *wt /* smem[9] */, int 
   return res;
 }
 
-constexpr int kDsMaxDepth = 4;                      // ring stages per warp: 4, or 2 for small batches
+constexpr int kDsMaxDepth = 5;                      // ring stages per warp: up to 5, or 2 for small batches
 constexpr int kDsRowBytes = kShrinkStepElems * 2;   // 512: one row segment of one K step
 constexpr int kDsStageBytes = (8 + kDsTok) * kDsRowBytes;  // 8 rows of A, then up to 4 rows of x
 
@@ -176,15 +176,26 @@ constexpr int kDsStageBytes = (8 + kDsTok) * kDsRowBytes;  // 8 rows of A, then 
 // in flight with TMA copies (one box of 8 x 512 bytes of A and one 512-byte row of x per token)
 // into the warp's private ring; columns past h_in arrive as zeros.  `phase` holds one parity bit
 // per ring stage and lives across calls.  Returns false if a wait gave up.
+// The ring's bytes are those of kDsDepth stages with four x rows; with fewer x rows a stage is
+// shorter, and with one token five stages fit where four did: a third more bytes in flight for the
+// items that dominate a many-adapter batch (the stream is bound by latency times bytes in flight).
 template <int NT, int kDsDepth>
+struct RingShape {
+  static constexpr int kStage = (8 + NT) * kDsRowBytes;
+  static constexpr int kDepth = (kDsDepth * kDsStageBytes) / kStage > kDsMaxDepth ? kDsMaxDepth
+                                                                                  : (kDsDepth * kDsStageBytes) / kStage;
+};
+template <int NT, int kDsDepthCfg>
 __device__ __forceinline__ bool shrink_rows8(const CUtensorMap *tmap_a, const CUtensorMap *tmap_x,
                                              int32_t slot, int32_t row0, const int32_t (&tok)[kDsTok],
                                              int step0, int step1, uint8_t *ring, uint64_t *bars,
                                              uint32_t &phase, int lane, float (&acc)[8 * kDsTok]) {
+  constexpr int kDsDepth = RingShape<NT, kDsDepthCfg>::kDepth;
+  constexpr int kStage = RingShape<NT, kDsDepthCfg>::kStage;
   auto issue = [&](int step, int stage) {
     if (lane == 0 && step < step1) {
-      uint8_t *dst = ring + stage * kDsStageBytes;
-      ptx::mbar_arrive_expect_tx(&bars[stage], (8 + NT) * kDsRowBytes);
+      uint8_t *dst = ring + stage * kStage;
+      ptx::mbar_arrive_expect_tx_relaxed(&bars[stage], (8 + NT) * kDsRowBytes);
       ptx::tma_load_3d(dst, tmap_a, &bars[stage], step * kShrinkStepElems, row0, slot);
 #pragma unroll
       for (int q = 0; q < NT; ++q)
@@ -199,7 +210,7 @@ __device__ __forceinline__ bool shrink_rows8(const CUtensorMap *tmap_a, const CU
     issue(step + kDsDepth - 1, (stage + kDsDepth - 1) % kDsDepth);
     if (!ptx::mbar_wait(&bars[stage], (phase >> stage) & 1u)) return false;
     phase ^= 1u << stage;
-    const uint4 *src = reinterpret_cast<const uint4 *>(ring + stage * kDsStageBytes) + lane;
+    const uint4 *src = reinterpret_cast<const uint4 *>(ring + stage * kStage) + lane;
     float xf[NT][8];
 #pragma unroll
     for (int q = 0; q < NT; ++q) unpack8(src[(8 + q) * (kDsRowBytes / 16)], xf[q]);
@@ -240,7 +251,7 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                      int32_t target_items, uint32_t *status) {
   extern __shared__ uint8_t s_ring_raw[];  // [warp][stage][8 A rows + 4 x rows][512 bytes]
   __shared__ uint64_t s_bars[kShrinkThreads / 32][kDsMaxDepth];
-  __shared__ int32_t s_id[256];        // validated id of each token
+  __shared__ __align__(16) int32_t s_id[256];  // validated id of each token
   __shared__ int32_t s_grp[256];       // group (in order of first appearance) of a group's first token
   __shared__ int32_t s_gadapter[256];  // adapter of each group
   __shared__ int32_t s_gstart[257];    // token list boundaries
@@ -258,7 +269,7 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     ptx::prefetch_tensormap(&tmap_a);
     ptx::prefetch_tensormap(&tmap_x);
   }
-  if (lane < kDsDepth) {  // every warp sets up its own ring barriers
+  if (lane < kDsMaxDepth) {  // every warp sets up its own ring barriers
     ptx::mbar_init(&s_bars[warp][lane], 1);
     ptx::fence_barrier_init();
   }
@@ -273,17 +284,28 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       bad = true;
     }
   }
+  SlotRow myrow = {0, 0.f, 0, 0};
+  if (a >= 0) myrow = slots[a];  // in flight during the duplicate scan below
   s_id[tid] = a;
   s_cnt[tid] = 0;
   __syncthreads();
   int pos = 0, first = tid;
-  if (a >= 0) {
-    for (int u = 0; u < tid; ++u) {
-      if (s_id[u] == a) {
+  if (a >= 0) {  // earlier tokens on the same adapter, four ids per shared-memory load
+    auto see = [&](int id, int u) {
+      if (id == a) {
         if (pos == 0) first = u;
         ++pos;
       }
+    };
+    const int full = tid & ~3;
+    for (int u = 0; u < full; u += 4) {
+      const int4 w = *reinterpret_cast<const int4 *>(&s_id[u]);
+      see(w.x, u);
+      see(w.y, u + 1);
+      see(w.z, u + 2);
+      see(w.w, u + 3);
     }
+    for (int u = full; u < tid; ++u) see(s_id[u], u);
   }
   const bool leader = a >= 0 && pos == 0;
   int G;
@@ -291,6 +313,8 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   if (leader) {
     s_grp[tid] = g;
     s_gadapter[g] = a;
+    s_grank[g] = myrow.rank;
+    s_gscale[g] = myrow.scale;
   }
   __syncthreads();
   int mygrp = -1;
@@ -300,11 +324,6 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   }
   __syncthreads();
   int tot;
-  if (tid < G) {  // in flight during the prefix sums below
-    const SlotRow row = slots[s_gadapter[tid]];
-    s_grank[tid] = row.rank;
-    s_gscale[tid] = row.scale;
-  }
   const int n_mine = tid < G ? s_cnt[tid] : 0;
   const int gs = block_scan_256(n_mine, s_wt, tot);
   if (tid < G) s_gstart[tid] = gs;
@@ -407,6 +426,34 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   const int warps_total = (gridDim.x - 1) * (kShrinkThreads / 32);
   int32_t *ticket = group_counters + kDsTicket;
   int item = publisher ? n_items : blockIdx.x * (kShrinkThreads / 32) + warp;  // first round is static
+  // The warp that completes a (group, row group) adds the K chunks in order into the final plane;
+  // it never waits for the others.  (Run at the end of the item, with the ring drained: its
+  // release is a fence, and a fence behind copies in flight waits for them too - putting it off
+  // into the next item's ramp-up measured slower.)
+  int pend_gi = -1, pend_rg = 0, pend_gt0 = 0, pend_gend = 0;
+  auto finalize = [&]() {
+    if (pend_gi < 0) return;
+    const int arrivals = KS * ((pend_gend - pend_gt0 + kDsBlockTok - 1) / kDsBlockTok);
+    __syncwarp();  // the lanes' z stores happen before lane 0's release
+    int old = 0;
+    if (lane == 0) old = atomic_add_acq_rel(&group_counters[pend_gi * 8 + pend_rg], 1);
+    old = __shfl_sync(0xffffffffu, old, 0);
+    if (old == arrivals - 1) {
+      if (lane == 0) group_counters[pend_gi * 8 + pend_rg] = 0;  // ready for the next launch
+      for (int idx = lane; idx < (pend_gend - pend_gt0) * 8; idx += 32) {
+        const int tq = idx >> 3;
+        const size_t off = static_cast<size_t>(s_gtok[pend_gt0 + tq]) * R_pad + pend_rg * 8 + (idx & 7);
+        float part[kMaxZSplits];
+#pragma unroll
+        for (int sp = 0; sp < kMaxZSplits; ++sp) part[sp] = sp < KS ? __ldcg(zws + sp * zplane + off) : 0.f;
+        float sum = 0.f;
+#pragma unroll
+        for (int sp = 0; sp < kMaxZSplits; ++sp) sum += part[sp];
+        zws[kMaxZSplits * zplane + off] = sum;
+      }
+    }
+    pend_gi = -1;
+  };
   while (ok && item < n_items) {
     int next = 0;
     if (lane == 0) next = warps_total + atomicAdd(ticket, 1);
@@ -465,27 +512,11 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     }
     if (!ok) break;
     if (KS > 1) {
-      // The warp that completes (group, row group) adds the K chunks in order into the final plane;
-      // it never waits for the others.
-      const int arrivals = KS * ((g_end - gt0 + kDsBlockTok - 1) / kDsBlockTok);
-      __syncwarp();  // the lanes' z stores happen before lane 0's release
-      int old = 0;
-      if (lane == 0) old = atomic_add_acq_rel(&group_counters[gi * 8 + rg], 1);
-      old = __shfl_sync(0xffffffffu, old, 0);
-      if (old == arrivals - 1) {
-        if (lane == 0) group_counters[gi * 8 + rg] = 0;  // ready for the next launch
-        for (int idx = lane; idx < (g_end - gt0) * 8; idx += 32) {
-          const int tq = idx >> 3;
-          const size_t off = static_cast<size_t>(s_gtok[gt0 + tq]) * R_pad + rg * 8 + (idx & 7);
-          float part[kMaxZSplits];
-#pragma unroll
-          for (int sp = 0; sp < kMaxZSplits; ++sp) part[sp] = sp < KS ? __ldcg(zws + sp * zplane + off) : 0.f;
-          float sum = 0.f;
-#pragma unroll
-          for (int sp = 0; sp < kMaxZSplits; ++sp) sum += part[sp];
-          zws[kMaxZSplits * zplane + off] = sum;
-        }
-      }
+      pend_gi = gi;
+      pend_rg = rg;
+      pend_gt0 = gt0;
+      pend_gend = g_end;
+      finalize();
     }
   }
   // Every warp stops at its first ticket >= n_items, so exactly n_items - (first round) + warps
