@@ -136,6 +136,10 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_
 __device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
+__device__ __forceinline__ void st_cluster_f32x4(uint32_t addr, float a, float b, float c, float d) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
+               : "memory");
+}
 
 // z of token t as packed bf16 (eight 16-byte chunks; chunks at or past the rank stride are zero):
 // the partial planes are added in order, values at or past the true rank forced to zero.
@@ -661,7 +665,13 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     const uint32_t my_rank = cluster_cta_rank();
     const int cols_per = p.BN / p.splits;  // a power of two (BN and splits are)
     const int shift = 31 - __clz(cols_per);
-    const bool have_acc = epi && !*abort_flag;  // this CTA's accumulator is complete (tfull waited)
+    // Large batches: the builder warps (6..9, the same four lane quadrants) send every other
+    // 32-token block, and all ten warps sum.  The epilogue warps have waited for the accumulator;
+    // the barrier below passes that on to the others.
+    const bool wide = !p.expand_in_reduce;
+    const bool sender = epi || (wide && warp >= 6);
+    const int c_first = (wide && warp >= 6) ? 32 : 0, c_step = wide ? 64 : 32;
+    const bool have_acc = sender && !*abort_flag;  // this CTA's accumulator is complete (tfull waited)
     __syncwarp();
     cluster_sync_all();
     if (have_acc) {
@@ -669,21 +679,33 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
       const uint32_t local = ptx::smem_u32(smem) +
                              ((my_rank * cols_per) * kTileM + row_in_tile) * 4u;
-      for (int32_t c0 = 0; c0 < p.BN; c0 += 32) {
+      const uint32_t qpo = static_cast<uint32_t>(cols_per) >> 2;  // token quads per owner
+      for (int32_t c0 = c_first; c0 < p.BN; c0 += c_step) {
         float v[32];
         ptx::tmem_ld_32x32(taddr + c0, v);
+        if (p.expand_in_reduce) {  // buf[src][token][row]
 #pragma unroll
-        for (int jj = 0; jj < 32; ++jj) {
-          const int col = c0 + jj;
-          const uint32_t owner = static_cast<uint32_t>(col >> shift);
-          const uint32_t off = static_cast<uint32_t>(col & (cols_per - 1)) * kTileM * 4u;
-          st_cluster_f32(map_to_cta(local + off, owner), v[jj]);  // a warp writes 128 bytes in a row
+          for (int jj = 0; jj < 32; ++jj) {
+            const int col = c0 + jj;
+            const uint32_t owner = static_cast<uint32_t>(col >> shift);
+            const uint32_t off = static_cast<uint32_t>(col & (cols_per - 1)) * kTileM * 4u;
+            st_cluster_f32(map_to_cta(local + off, owner), v[jj]);  // a warp writes 128 bytes in a row
+          }
+        } else {  // buf[src][token quad][row][4 tokens]: 16-byte stores, a warp writes 512 bytes in a row
+#pragma unroll
+          for (int g4 = 0; g4 < 8; ++g4) {
+            const int col = c0 + g4 * 4;
+            const uint32_t owner = static_cast<uint32_t>(col >> shift);
+            const uint32_t quad_i = static_cast<uint32_t>(col & (cols_per - 1)) >> 2;
+            const uint32_t addr = ptx::smem_u32(smem) + ((my_rank * qpo + quad_i) * kTileM + row_in_tile) * 16u;
+            st_cluster_f32x4(map_to_cta(addr, owner), v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
+          }
         }
       }
     }
     __syncwarp();
     cluster_sync_all();
-    if (epi) {
+    if (epi || wide) {
       const float *buf = reinterpret_cast<const float *>(smem);
       const int n_units = cols_per * 32;  // unit = (token, 4 adjacent W rows)
       const int row0 = blockIdx.x / p.splits * kTileM;
@@ -702,11 +724,26 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         *reinterpret_cast<uint2 *>(p.y + static_cast<size_t>(t) * p.h_out + j) = o;
       };
       if (!p.expand_in_reduce) {
-        for (int u = etid; u < n_units; u += 128) {
-          const int cl = u >> 5, r4 = (u & 31) << 2;
-          const int t = static_cast<int>(my_rank) * cols_per + cl, j = row0 + r4;
-          if (t >= p.T || j >= p.h_out) continue;  // h_out is a multiple of 8: 4 rows are all in or out
-          store4(t, j, sum_partials(cl, r4));
+        // unit = (token quad, W row): the splits' partial sums are 16 bytes each, lanes take
+        // adjacent rows, so a warp writes 64 bytes in a row of y per token
+        const int qpo = cols_per >> 2;
+        const float4 *buf4 = reinterpret_cast<const float4 *>(smem);
+        ptx::pdl_wait_prior_grids();  // warps 0 and 1 have not waited yet; earlier kernels may read y
+        for (int u = threadIdx.x; u < qpo * kTileM; u += kGemmThreads) {
+          const int qd = u >> 7, r = u & (kTileM - 1);
+          const int t0 = static_cast<int>(my_rank) * cols_per + qd * 4, j = row0 + r;
+          if (t0 >= p.T || j >= p.h_out) continue;
+          float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int sp = 0; sp < p.splits; ++sp) {
+            const float4 w = buf4[(sp * qpo + qd) * kTileM + r];
+            a4.x += w.x; a4.y += w.y; a4.z += w.z; a4.w += w.w;
+          }
+          const float o[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            if (t0 + i < p.T)
+              p.y[static_cast<size_t>(t0 + i) * p.h_out + j] =
+                  static_cast<uint16_t>(ptx::pack_bf16x2(o[i], 0.f) & 0xFFFFu);
         }
       } else {
         // Small batches.  Everything that does not need z first: the base product's sums stay in
