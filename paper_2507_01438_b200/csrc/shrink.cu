@@ -188,7 +188,7 @@ struct RingShape {
 template <int NT, int kDsDepthCfg>
 __device__ __forceinline__ bool shrink_rows8(const CUtensorMap *tmap_a, const CUtensorMap *tmap_x,
                                              int32_t slot, int32_t row0, const int32_t (&tok)[kDsTok],
-                                             int step0, int step1, uint8_t *ring, uint64_t *bars,
+                                             int step0, int step1, int stride, uint8_t *ring, uint64_t *bars,
                                              uint32_t &phase, int lane, float (&acc)[8 * kDsTok]) {
   constexpr int kDsDepth = RingShape<NT, kDsDepthCfg>::kDepth;
   constexpr int kStage = RingShape<NT, kDsDepthCfg>::kStage;
@@ -203,11 +203,11 @@ __device__ __forceinline__ bool shrink_rows8(const CUtensorMap *tmap_a, const CU
     }
   };
 #pragma unroll
-  for (int d = 0; d < kDsDepth - 1; ++d) issue(step0 + d, d);
+  for (int d = 0; d < kDsDepth - 1; ++d) issue(step0 + d * stride, d);
   int stage = 0;
-  for (int step = step0; step < step1; ++step) {
+  for (int step = step0; step < step1; step += stride) {
     __syncwarp();  // every lane has finished reading the stage that is refilled next
-    issue(step + kDsDepth - 1, (stage + kDsDepth - 1) % kDsDepth);
+    issue(step + (kDsDepth - 1) * stride, (stage + kDsDepth - 1) % kDsDepth);
     if (!ptx::mbar_wait(&bars[stage], (phase >> stage) & 1u)) return false;
     phase ^= 1u << stage;
     const uint4 *src = reinterpret_cast<const uint4 *>(ring + stage * kStage) + lane;
@@ -460,9 +460,12 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     next = __shfl_sync(0xffffffffu, next, 0);
     const int cur = item;
     item = next;
-    const int rg = cur % n_rgn;
-    const int bc = cur / n_rgn;
-    const int bi = bc / KS, c = bc - bi * KS;
+    // consecutive items are the K chunks of one (token block, row group), and chunk c takes the K
+    // steps c, c + KS, c + 2 KS, ...: warps that run side by side fetch neighbouring 512-byte
+    // pieces of the same rows at about the same time
+    const int c = cur % KS;
+    const int br = cur / KS;
+    const int bi = br / n_rgn, rg = br - bi * n_rgn;
     const int gi = s_bgrp[bi];
     const int ad = s_gadapter[gi];
     const int rank = s_grank[gi];
@@ -475,7 +478,7 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     }
     const int n_rg = (rank + 7) >> 3;  // live groups of eight rows
     if (rg >= n_rg) continue;               // rows past the rank are zero padding: nothing to do
-    const int step0 = c * spc, step1 = min(n_ksteps, step0 + spc);
+    const int step0 = c, step1 = n_ksteps;
     const int q = lane & 3, r = rg * 8 + (lane >> 2);
     for (int tb = t0; ok && tb < t1; tb += kDsTok) {
       const int nt = min(kDsTok, t1 - tb);
@@ -485,10 +488,10 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       int32_t tok[kDsTok];
 #pragma unroll
       for (int qq = 0; qq < kDsTok; ++qq) tok[qq] = s_gtok[tb + min(qq, nt - 1)];
-      if (nt == 1) ok = shrink_rows8<1, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
-      else if (nt == 2) ok = shrink_rows8<2, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
-      else if (nt == 3) ok = shrink_rows8<3, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
-      else ok = shrink_rows8<4, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, ring, bars, phase, lane, acc);
+      if (nt == 1) ok = shrink_rows8<1, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
+      else if (nt == 2) ok = shrink_rows8<2, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
+      else if (nt == 3) ok = shrink_rows8<3, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
+      else ok = shrink_rows8<4, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       // lane L ends with the sum over lanes of value L (= row L / 4, token L % 4)

@@ -92,6 +92,8 @@ def test_ragged_ranks(max_rank, ranks, T):
     (64, 2048, 1024, 16, [16, 8, 3, 16, 12, 16]),   # same path at its largest token count
     (64, 1024, 2048, 64, [64, 64, 17]),             # too many B loads per owner: LoRA K blocks, 64 tokens
     (200, 1024, 1024, 32, [32, 8, 24, 16]),         # LoRA K blocks with both halves of the 256-token tile
+    (255, 1536, 1000, 64, [64, 8, 32, 16, 50]),     # 8 K splits of a 256-token tile, ragged last row tile and token quad
+    (97, 2048, 520, 32, [32, 5, 16]),               # 128-token tile through the wide cluster reduction
 ])
 def test_small_and_medium_decode_paths(T, h_in, h_out, max_rank, ranks):
     w = random_workload(T + h_out + max_rank, T, h_in, h_out, ranks=ranks, max_rank=max_rank)
