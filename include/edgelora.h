@@ -130,6 +130,20 @@ int edgelora_lora_linear_host(edgelora_pool_t *pool, const void *W_dev, const ui
                               const int32_t *adapter_id_host, int32_t T, uint16_t *y_host,
                               void *stream);
 
+/* The same, pipelined: returns as soon as the copies and the layer are enqueued.  x_host,
+ * adapter_id_host and y_host should be page-locked (otherwise the copies still complete but do
+ * not overlap) and must stay valid and untouched until edgelora_pool_host_sync returns.  The
+ * library keeps two sets of device mirrors and two copy streams: the copy-in of call i + 1 and
+ * the copy-out of call i - 1 run beside the layer of call i (which runs on `stream`).  Calls of
+ * one pool are issued from one thread.  (Serving loop of Section 3.4: a batch is formed while
+ * the previous one computes.) */
+int edgelora_lora_linear_host_async(edgelora_pool_t *pool, const void *W_dev, const uint16_t *x_host,
+                                    const int32_t *adapter_id_host, int32_t T, uint16_t *y_host,
+                                    void *stream);
+
+/* Blocks until every y_host of earlier edgelora_lora_linear_host_async calls is complete. */
+int edgelora_pool_host_sync(edgelora_pool_t *pool);
+
 /* Routing plan (Section 3.4 "u-batch" grouping; Section 4.3 "maps adapter IDs to sample
  * indices ... scattered back to their original positions").  A plan depends only on the
  * ids, so one plan can serve every linear site that sees the same batch. */

@@ -28,7 +28,8 @@ EXPORTS = (
     "edgelora_plan_build", "edgelora_plan_export", "edgelora_lora_linear_planned",
     "edgelora_pool_plan", "edgelora_pool_sync_status", "edgelora_pool_set_option",
     "edgelora_pool_last_launch", "edgelora_pool_kernel_times", "edgelora_pool_destroy",
-    "edgelora_strerror", "edgelora_plan_build_static",
+    "edgelora_strerror", "edgelora_plan_build_static", "edgelora_lora_linear_host_async",
+    "edgelora_pool_host_sync",
 )
 
 
@@ -65,6 +66,8 @@ def lib() -> ctypes.CDLL:
     L.edgelora_pool_wait_loads.argtypes = [vp]
     L.edgelora_lora_linear.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     L.edgelora_lora_linear_host.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+    L.edgelora_lora_linear_host_async.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+    L.edgelora_pool_host_sync.argtypes = [vp]
     L.edgelora_plan_create.argtypes = [i32, i32, cp(vp)]
     L.edgelora_plan_destroy.argtypes = [vp]
     L.edgelora_plan_build.argtypes = [vp, vp, i32, vp]
@@ -164,6 +167,20 @@ def edgelora_lora_linear_host(pool, W, x_host: np.ndarray, ids_host: np.ndarray,
     _check(lib().edgelora_lora_linear_host(pool, _dev_ptr(W, 2, "W"), x_host.ctypes.data,
                                            ids_host.ctypes.data, T, y_host.ctypes.data,
                                            _stream_ptr(stream)), "lora_linear_host")
+
+
+def edgelora_lora_linear_host_async(pool, W, x_host, ids_host, y_host, stream=None) -> None:
+    """Pipelined host-buffer call; the arguments are page-locked CPU tensors (torch, pin_memory) or
+    numpy arrays of uint16 / int32 / uint16 and must stay alive until ``edgelora_pool_host_sync``."""
+    def ptr(a):
+        return a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data
+    T = int(x_host.shape[0])
+    _check(lib().edgelora_lora_linear_host_async(pool, _dev_ptr(W, 2, "W"), ptr(x_host), ptr(ids_host), T,
+                                                 ptr(y_host), _stream_ptr(stream)), "lora_linear_host_async")
+
+
+def edgelora_pool_host_sync(pool) -> None:
+    _check(lib().edgelora_pool_host_sync(pool), "pool_host_sync")
 
 
 def edgelora_plan_create(max_tokens: int, n_slots: int) -> int:

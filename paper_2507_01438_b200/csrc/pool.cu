@@ -147,6 +147,12 @@ struct edgelora_pool {
   // host-buffer entry point
   uint16_t *hx = nullptr, *hy = nullptr, *dx = nullptr, *dy = nullptr;
   int32_t *hids = nullptr, *dids = nullptr;
+  // pipelined host-buffer path: two sets of device mirrors, two copy streams, events per set
+  uint16_t *pdx[2] = {nullptr, nullptr}, *pdy[2] = {nullptr, nullptr};
+  int32_t *pdids[2] = {nullptr, nullptr};
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+  uint64_t host_calls = 0;
 };
 
 namespace {
@@ -451,6 +457,16 @@ int edgelora_pool_destroy(edgelora_pool_t *p) {
   if (p->dx) cudaFree(p->dx);
   if (p->dy) cudaFree(p->dy);
   if (p->dids) cudaFree(p->dids);
+  for (int b = 0; b < 2; ++b) {
+    if (p->pdx[b]) cudaFree(p->pdx[b]);
+    if (p->pdy[b]) cudaFree(p->pdy[b]);
+    if (p->pdids[b]) cudaFree(p->pdids[b]);
+    if (p->ev_in[b]) cudaEventDestroy(p->ev_in[b]);
+    if (p->ev_done[b]) cudaEventDestroy(p->ev_done[b]);
+    if (p->ev_out[b]) cudaEventDestroy(p->ev_out[b]);
+  }
+  if (p->h2d_stream) cudaStreamDestroy(p->h2d_stream);
+  if (p->d2h_stream) cudaStreamDestroy(p->d2h_stream);
   cudaGetLastError();
   delete p;
   return EDGELORA_OK;
@@ -886,6 +902,56 @@ int edgelora_lora_linear_host(edgelora_pool_t *p, const void *W_dev, const uint1
   CUDA_TRY(cudaMemcpyAsync(p->hy, p->dy, yb, cudaMemcpyDeviceToHost, s));
   CUDA_TRY(cudaStreamSynchronize(s));
   memcpy(y_host, p->hy, yb);
+  return EDGELORA_OK;
+}
+
+int edgelora_lora_linear_host_async(edgelora_pool_t *p, const void *W_dev, const uint16_t *x_host,
+                                    const int32_t *adapter_id_host, int32_t T, uint16_t *y_host,
+                                    void *stream) {
+  if (!p || T < 0) return EDGELORA_ERR_INVALID_ARG;
+  if (T == 0) return EDGELORA_OK;
+  if (!x_host || !adapter_id_host || !y_host) return EDGELORA_ERR_INVALID_ARG;
+  if (T > p->cfg.max_tokens) return EDGELORA_ERR_TOO_MANY_TOKENS;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t mt = p->cfg.max_tokens;
+  if (!p->h2d_stream) {  // first use
+    CUDA_TRY(cudaStreamCreateWithFlags(&p->h2d_stream, cudaStreamNonBlocking));
+    CUDA_TRY(cudaStreamCreateWithFlags(&p->d2h_stream, cudaStreamNonBlocking));
+    for (int b = 0; b < 2; ++b) {
+      CUDA_TRY(cudaMalloc(&p->pdx[b], mt * p->cfg.h_in * 2));
+      CUDA_TRY(cudaMalloc(&p->pdy[b], mt * p->cfg.h_out * 2));
+      CUDA_TRY(cudaMalloc(&p->pdids[b], mt * 4));
+      CUDA_TRY(cudaEventCreateWithFlags(&p->ev_in[b], cudaEventDisableTiming));
+      CUDA_TRY(cudaEventCreateWithFlags(&p->ev_done[b], cudaEventDisableTiming));
+      CUDA_TRY(cudaEventCreateWithFlags(&p->ev_out[b], cudaEventDisableTiming));
+    }
+  }
+  const int b = static_cast<int>(p->host_calls & 1);
+  const bool reused = p->host_calls >= 2;  // the set was used two calls ago
+  ++p->host_calls;
+  const size_t xb = static_cast<size_t>(T) * p->cfg.h_in * 2, yb = static_cast<size_t>(T) * p->cfg.h_out * 2;
+  // inputs: after the layer that last read this set of mirrors
+  if (reused) CUDA_TRY(cudaStreamWaitEvent(p->h2d_stream, p->ev_done[b], 0));
+  CUDA_TRY(cudaMemcpyAsync(p->pdx[b], x_host, xb, cudaMemcpyHostToDevice, p->h2d_stream));
+  CUDA_TRY(cudaMemcpyAsync(p->pdids[b], adapter_id_host, static_cast<size_t>(T) * 4, cudaMemcpyHostToDevice,
+                           p->h2d_stream));
+  CUDA_TRY(cudaEventRecord(p->ev_in[b], p->h2d_stream));
+  // layer: after its inputs, and after the copy-out that last read this set's y
+  CUDA_TRY(cudaStreamWaitEvent(s, p->ev_in[b], 0));
+  if (reused) CUDA_TRY(cudaStreamWaitEvent(s, p->ev_out[b], 0));
+  int rc = lora_linear_impl(p, p->plan, p->pdids[b], W_dev, p->pdx[b], T, p->pdy[b], s);
+  if (rc != EDGELORA_OK) return rc;
+  CUDA_TRY(cudaEventRecord(p->ev_done[b], s));
+  // result
+  CUDA_TRY(cudaStreamWaitEvent(p->d2h_stream, p->ev_done[b], 0));
+  CUDA_TRY(cudaMemcpyAsync(y_host, p->pdy[b], yb, cudaMemcpyDeviceToHost, p->d2h_stream));
+  CUDA_TRY(cudaEventRecord(p->ev_out[b], p->d2h_stream));
+  return EDGELORA_OK;
+}
+
+int edgelora_pool_host_sync(edgelora_pool_t *p) {
+  if (!p) return EDGELORA_ERR_INVALID_ARG;
+  if (p->d2h_stream) CUDA_TRY(cudaStreamSynchronize(p->d2h_stream));
   return EDGELORA_OK;
 }
 

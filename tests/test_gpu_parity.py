@@ -277,6 +277,37 @@ def test_host_buffer_entry_point():
         pool.close()
 
 
+def test_pipelined_host_buffer_entry_point():
+    # five calls in flight over two sets of device mirrors: every y must match its own inputs
+    import torch
+    base = random_workload(900, 40, 256, 384, ranks=[8, 16, 4, 12], max_rank=16)
+    pool = make_pool(base, 128)
+    try:
+        W = to_dev_bf16(base.W)
+        rng = np.random.Generator(np.random.PCG64(901))
+        batches = []
+        for i in range(5):
+            T = 40 + 17 * i
+            x = wl.normal_bf16(rng, (T, base.h_in), 1.0)
+            ids = rng.integers(-1, 4, size=T).astype(np.int32)
+            batches.append(wl.Workload(f"pipelined{i}", base.h_in, base.h_out, base.n_slots, base.max_rank,
+                                       base.W, x, ids, base.adapters))
+        pin = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a).view(dt)).pin_memory()
+        xs = [pin(b.x, np.int16) for b in batches]
+        ids = [pin(b.ids, np.int32) for b in batches]
+        ys = [torch.zeros((b.T, b.h_out), dtype=torch.int16).pin_memory() for b in batches]
+        for x, i, y in zip(xs, ids, ys):
+            B.edgelora_lora_linear_host_async(pool.handle, W, x, i, y)
+        B.edgelora_pool_host_sync(pool.handle)
+        assert pool.status() == (0, 0)
+        for b, y in zip(batches, ys):
+            got = wl.bf16_bits_to_f32(y.numpy().view(np.uint16))
+            assert_parity(got, oracle_of(b), f"pipelined T={b.T}")
+            assert np.array_equal(got, run_gpu(b, pool=pool))
+    finally:
+        pool.close()
+
+
 def test_profiling_option_reports_every_kernel():
     w = random_workload(41, 300, 256, 256, ranks=[16, 16], max_rank=16, id_mode="runs", run_len=64)
     pool = make_pool(w, 512)
