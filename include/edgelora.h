@@ -47,7 +47,8 @@ typedef enum {
   EDGELORA_ERR_BAD_ADAPTER_ID = -6,
   EDGELORA_ERR_SLOT_EMPTY = -7,
   EDGELORA_ERR_TIMEOUT = -8,
-  EDGELORA_ERR_TOO_MANY_TOKENS = -9
+  EDGELORA_ERR_TOO_MANY_TOKENS = -9,
+  EDGELORA_ERR_CACHE_FULL = -10
 } edgelora_status;
 
 /* Bits of the device status word returned by edgelora_pool_sync_status(). */
@@ -217,6 +218,36 @@ int edgelora_pool_kernel_times(edgelora_pool_t *pool, double ms_out[5], int64_t 
 
 /* Releases everything the pool owns (never the caller's arena).  Synchronises first. */
 int edgelora_pool_destroy(edgelora_pool_t *pool);
+
+/* ---- Adapter memory manager (host side; Section 3.3 "adapter memory manager", Section 4.2:
+ * recency list + set of resident adapters + stack of free blocks).  Decides which block of a
+ * pool an adapter lives in; moves no bytes (the caller passes the block to
+ * edgelora_pool_load_slot on a miss, which copies on the pool's side stream beside the layer
+ * calls).  Keys are the caller's adapter ids (>= 0); blocks are slot indices 0 .. n_blocks-1.
+ * Host memory only, no CUDA call; one thread at a time per cache. */
+typedef struct edgelora_cache edgelora_cache_t;
+#define EDGELORA_CACHE_LRU 0 /* evict the least recently used adapter (Section 4.2)              */
+#define EDGELORA_CACHE_LFU 1 /* evict the least frequently used one (Section 3.3), ties by recency;
+                                a use count restarts when an adapter returns after an eviction  */
+
+int edgelora_cache_create(int32_t n_blocks, int32_t policy, edgelora_cache_t **cache_out);
+int edgelora_cache_destroy(edgelora_cache_t *cache);
+
+/* The block of `key`.  Resident: *hit_out = 1, recency and use count updated.  Not resident:
+ * *hit_out = 0 and *slot_out is the block to load it into: the lowest free block while any is
+ * free, otherwise the victim's, whose key goes to *evicted_key_out (-1 if nothing was evicted).
+ * pin != 0 marks the adapter as held by a running request until edgelora_cache_release: held
+ * adapters are never victims; EDGELORA_ERR_CACHE_FULL when every block is held.  hit_out and
+ * evicted_key_out may be NULL. */
+int edgelora_cache_acquire(edgelora_cache_t *cache, int64_t key, int32_t pin, int32_t *slot_out,
+                           int32_t *hit_out, int64_t *evicted_key_out);
+/* Drops one hold on `key` (EDGELORA_ERR_INVALID_ARG if it has none). */
+int edgelora_cache_release(edgelora_cache_t *cache, int64_t key);
+/* Block of `key` or -1, without touching recency or counts. */
+int edgelora_cache_lookup(const edgelora_cache_t *cache, int64_t key, int32_t *slot_out);
+/* Counters since creation; any pointer may be NULL. */
+int edgelora_cache_stats(const edgelora_cache_t *cache, int64_t *hits, int64_t *misses,
+                         int64_t *evictions, int32_t *resident);
 
 const char *edgelora_strerror(int code);
 

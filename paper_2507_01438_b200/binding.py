@@ -29,7 +29,8 @@ EXPORTS = (
     "edgelora_pool_plan", "edgelora_pool_sync_status", "edgelora_pool_set_option",
     "edgelora_pool_last_launch", "edgelora_pool_kernel_times", "edgelora_pool_destroy",
     "edgelora_strerror", "edgelora_plan_build_static", "edgelora_lora_linear_host_async",
-    "edgelora_pool_host_sync",
+    "edgelora_pool_host_sync", "edgelora_cache_create", "edgelora_cache_destroy", "edgelora_cache_acquire",
+    "edgelora_cache_release", "edgelora_cache_lookup", "edgelora_cache_stats",
 )
 
 
@@ -68,6 +69,13 @@ def lib() -> ctypes.CDLL:
     L.edgelora_lora_linear_host.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     L.edgelora_lora_linear_host_async.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     L.edgelora_pool_host_sync.argtypes = [vp]
+    i64 = ctypes.c_int64
+    L.edgelora_cache_create.argtypes = [i32, i32, cp(vp)]
+    L.edgelora_cache_destroy.argtypes = [vp]
+    L.edgelora_cache_acquire.argtypes = [vp, i64, i32, cp(i32), cp(i32), cp(i64)]
+    L.edgelora_cache_release.argtypes = [vp, i64]
+    L.edgelora_cache_lookup.argtypes = [vp, i64, cp(i32)]
+    L.edgelora_cache_stats.argtypes = [vp, cp(i64), cp(i64), cp(i64), cp(i32)]
     L.edgelora_plan_create.argtypes = [i32, i32, cp(vp)]
     L.edgelora_plan_destroy.argtypes = [vp]
     L.edgelora_plan_build.argtypes = [vp, vp, i32, vp]
@@ -268,6 +276,45 @@ def edgelora_pool_kernel_times(pool, reset: bool = True) -> dict:
 
 def edgelora_pool_destroy(pool) -> None:
     _check(lib().edgelora_pool_destroy(pool), "pool_destroy")
+
+
+CACHE_LRU, CACHE_LFU = 0, 1
+ERR_CACHE_FULL = -10
+
+
+def edgelora_cache_create(n_blocks: int, policy: int = CACHE_LRU) -> int:
+    out = ctypes.c_void_p()
+    _check(lib().edgelora_cache_create(n_blocks, policy, ctypes.byref(out)), "cache_create")
+    return out.value
+
+
+def edgelora_cache_destroy(cache) -> None:
+    _check(lib().edgelora_cache_destroy(cache), "cache_destroy")
+
+
+def edgelora_cache_acquire(cache, key: int, pin: bool = False):
+    """Returns (block, hit, evicted key or -1)."""
+    slot, hit, ev = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int64()
+    _check(lib().edgelora_cache_acquire(cache, key, 1 if pin else 0, ctypes.byref(slot), ctypes.byref(hit),
+                                        ctypes.byref(ev)), "cache_acquire")
+    return slot.value, bool(hit.value), ev.value
+
+
+def edgelora_cache_release(cache, key: int) -> None:
+    _check(lib().edgelora_cache_release(cache, key), "cache_release")
+
+
+def edgelora_cache_lookup(cache, key: int) -> int:
+    slot = ctypes.c_int32()
+    _check(lib().edgelora_cache_lookup(cache, key, ctypes.byref(slot)), "cache_lookup")
+    return slot.value
+
+
+def edgelora_cache_stats(cache) -> dict:
+    h, m, e, r = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int32()
+    _check(lib().edgelora_cache_stats(cache, ctypes.byref(h), ctypes.byref(m), ctypes.byref(e), ctypes.byref(r)),
+           "cache_stats")
+    return {"hits": h.value, "misses": m.value, "evictions": e.value, "resident": r.value}
 
 
 class Pool:

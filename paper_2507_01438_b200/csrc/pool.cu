@@ -270,6 +270,7 @@ const char *edgelora_strerror(int code) {
     case EDGELORA_ERR_SLOT_EMPTY: return "an adapter id named an empty slot (token computed base-only)";
     case EDGELORA_ERR_TIMEOUT: return "a bounded in-kernel wait gave up";
     case EDGELORA_ERR_TOO_MANY_TOKENS: return "T exceeds max_tokens (or max_tokens exceeds 32768)";
+    case EDGELORA_ERR_CACHE_FULL: return "every block of the adapter cache is held by a running request";
     default: return "unknown error";
   }
 }
