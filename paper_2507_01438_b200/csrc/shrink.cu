@@ -38,16 +38,20 @@ bgmv_shrink_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ 
   ptx::pdl_launch_dependents();
   ptx::pdl_wait_prior_grids();  // the plan comes from the previous kernel
 
-  const int g = blockIdx.x / R_pad;
-  const int i = blockIdx.x % R_pad;
-  if (g >= pv.counts[0]) return;
+  // Work items (group, rank row) are strided over a grid sized for the machine, not for the worst
+  // case of groups: most batches have far fewer groups than slots, and CTAs that only find out
+  // that they have nothing to do cost more than the items themselves.
+  const int n_work = pv.counts[0] * R_pad;
+  for (int wi = blockIdx.x; wi < n_work; wi += gridDim.x) {
+  const int g = wi / R_pad;
+  const int i = wi % R_pad;
   const int a = pv.group_adapter[g];
-  if (a < 0) return;
+  if (a < 0) continue;
   const SlotRow row = slots[a];
   const int g0 = pv.gs_short[g], g1 = pv.gs_short[g + 1];
   if (row.rank <= 0) {
     if (threadIdx.x == 0 && i == 0) atomicOr(status, EDGELORA_STATUS_SLOT_EMPTY);
-    return;
+    continue;
   }
   const bool live_row = i < row.rank;
   const uint4 *Arow =
@@ -98,6 +102,7 @@ bgmv_shrink_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ 
       for (int sp = 1; sp < zsplits; ++sp) zws[sp * zsplit_stride + off] = 0.f;
     }
   }
+  }
 }
 
 void launch_bgmv_shrink(const uint16_t *x, const uint16_t *A_pool, const SlotRow *slots,
@@ -105,7 +110,15 @@ void launch_bgmv_shrink(const uint16_t *x, const uint16_t *A_pool, const SlotRow
                         int32_t n_slots, int32_t zsplits, int32_t max_tokens, uint32_t *status,
                         bool pdl, cudaStream_t stream) {
   const int max_groups = (T < n_slots + 1) ? T : n_slots + 1;
-  launch_ex(bgmv_shrink_kernel, dim3(max_groups * R_pad), dim3(kBgmvThreads), 0, stream, pdl, 1, x,
+  static int sms = 0;  // same on every device of a node
+  if (sms == 0) {
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    sms = n > 0 ? n : 148;
+  }
+  const int grid = max_groups * R_pad < sms * 8 ? max_groups * R_pad : sms * 8;
+  launch_ex(bgmv_shrink_kernel, dim3(grid), dim3(kBgmvThreads), 0, stream, pdl, 1, x,
             A_pool, slots, pv, zws, T, h_in, R_pad, zsplits, max_tokens, status);
 }
 
