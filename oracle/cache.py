@@ -79,3 +79,21 @@ class AdapterCache:
 
     def resident(self) -> int:
         return len(self.slot)
+
+
+def select_adapter(cache: AdapterCache, scores, k: int, pin: bool = False):
+    """Cache-aware adapter selection (paper Algorithm 1, second half; Section 3.2): of the k
+    adapters with the highest router scores, taken in descending order of score, the first one
+    that is resident is used; if none is, the one with the highest score is loaded.  Scores are
+    compared as given (float32); equal scores rank by adapter index.
+    Returns (adapter, block, hit, evicted key or -1)."""
+    import numpy as np
+    s = np.asarray(scores, dtype=np.float32)
+    order = sorted(range(len(s)), key=lambda j: (-float(s[j]), j))
+    top = order[:max(1, min(k, len(order)))]
+    for a in top:
+        if cache.lookup(a) >= 0:
+            block, hit, evicted = cache.acquire(a, pin)
+            return a, block, hit, evicted
+    block, hit, evicted = cache.acquire(top[0], pin)
+    return top[0], block, hit, evicted

@@ -98,3 +98,63 @@ def test_invariants_on_a_power_law_trace(policy):
     assert c.hits + c.misses == len(trace) and c.evictions == c.misses - 16
     # a popular head makes the cache useful: far more hits than a uniform trace would give
     assert c.hits / len(trace) > 0.4
+
+
+# ---------------------------------------------------------------- cache-aware selection (Algorithm 1)
+from oracle.cache import select_adapter
+
+
+def brute_force_choice(resident, scores, k):
+    # every adapter ranked by hand; the answer is the best-scored resident one inside the top k,
+    # else the best-scored overall
+    ranked = []
+    remaining = list(range(len(scores)))
+    while remaining:
+        best = remaining[0]
+        for j in remaining:
+            if scores[j] > scores[best]:
+                best = j
+        ranked.append(best)
+        remaining.remove(best)
+    inside = [a for a in ranked[:k] if a in resident]
+    return inside[0] if inside else ranked[0]
+
+
+def test_selection_with_k_one_is_the_argmax():
+    rng = np.random.Generator(np.random.PCG64(2))
+    c = AdapterCache(4)
+    for _ in range(50):
+        s = rng.random(20).astype(np.float32)
+        a, _, _, _ = select_adapter(c, s, 1)
+        assert a == int(np.argmax(s))
+
+
+def test_selection_prefers_a_resident_adapter_inside_the_top_k_only():
+    c = AdapterCache(2)
+    c.acquire(5)
+    c.acquire(9)
+    s = np.zeros(12, dtype=np.float32)
+    s[[3, 5, 9, 7]] = [0.9, 0.8, 0.7, 0.6]
+    assert select_adapter(c, s, 1)[:3] == (3, 0, False)      # k = 1: top-1 loaded although 5 and 9 are resident
+    c2 = AdapterCache(2)
+    c2.acquire(5)
+    c2.acquire(9)
+    assert select_adapter(c2, s, 2)[:3] == (5, 0, True)       # 5 is the best resident one inside the top 2
+    s[5] = 0.0
+    assert select_adapter(c2, s, 2)[:3] == (9, 1, True)       # top 2 is now {3, 9}, and 9 is resident
+    s[9] = 0.0
+    assert select_adapter(c2, s, 2)[:3] == (3, 0, False)      # top 2 = {3, 7}: none resident, 3 is loaded over 5
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 8])
+def test_selection_against_brute_force(k):
+    rng = np.random.Generator(np.random.PCG64(30 + k))
+    c = AdapterCache(5)
+    for _ in range(300):
+        s = rng.random(24).astype(np.float32)
+        if rng.random() < 0.3:
+            s[rng.integers(0, 24, size=4)] = s[0]           # ties
+        expect = brute_force_choice(set(c.slot), s.tolist(), k)
+        was_resident = c.lookup(expect) >= 0
+        a, block, hit, evicted = select_adapter(c, s, k)
+        assert a == expect and hit == was_resident and c.lookup(a) == block
