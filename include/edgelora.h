@@ -241,6 +241,14 @@ int edgelora_cache_destroy(edgelora_cache_t *cache);
  * evicted_key_out may be NULL. */
 int edgelora_cache_acquire(edgelora_cache_t *cache, int64_t key, int32_t pin, int32_t *slot_out,
                            int32_t *hit_out, int64_t *evicted_key_out);
+/* Cache-aware adapter selection (Algorithm 1 of the paper, Section 3.2): scores[j] is the
+ * router's confidence for adapter j (host array, n entries, key = index).  Of the k best-scored
+ * adapters, in descending order of score (equal scores: lower index first; scores are finite), the
+ * first resident one is chosen; if none of them is resident the best-scored one is chosen and
+ * admitted.  The choice goes to *key_out; the rest is edgelora_cache_acquire of that key. */
+int edgelora_cache_select(edgelora_cache_t *cache, const float *scores, int32_t n, int32_t k,
+                          int32_t pin, int64_t *key_out, int32_t *slot_out, int32_t *hit_out,
+                          int64_t *evicted_key_out);
 /* Drops one hold on `key` (EDGELORA_ERR_INVALID_ARG if it has none). */
 int edgelora_cache_release(edgelora_cache_t *cache, int64_t key);
 /* Block of `key` or -1, without touching recency or counts. */

@@ -30,7 +30,7 @@ EXPORTS = (
     "edgelora_pool_last_launch", "edgelora_pool_kernel_times", "edgelora_pool_destroy",
     "edgelora_strerror", "edgelora_plan_build_static", "edgelora_lora_linear_host_async",
     "edgelora_pool_host_sync", "edgelora_cache_create", "edgelora_cache_destroy", "edgelora_cache_acquire",
-    "edgelora_cache_release", "edgelora_cache_lookup", "edgelora_cache_stats",
+    "edgelora_cache_release", "edgelora_cache_lookup", "edgelora_cache_stats", "edgelora_cache_select",
 )
 
 
@@ -74,6 +74,7 @@ def lib() -> ctypes.CDLL:
     L.edgelora_cache_destroy.argtypes = [vp]
     L.edgelora_cache_acquire.argtypes = [vp, i64, i32, cp(i32), cp(i32), cp(i64)]
     L.edgelora_cache_release.argtypes = [vp, i64]
+    L.edgelora_cache_select.argtypes = [vp, vp, i32, i32, i32, cp(i64), cp(i32), cp(i32), cp(i64)]
     L.edgelora_cache_lookup.argtypes = [vp, i64, cp(i32)]
     L.edgelora_cache_stats.argtypes = [vp, cp(i64), cp(i64), cp(i64), cp(i32)]
     L.edgelora_plan_create.argtypes = [i32, i32, cp(vp)]
@@ -298,6 +299,16 @@ def edgelora_cache_acquire(cache, key: int, pin: bool = False):
     _check(lib().edgelora_cache_acquire(cache, key, 1 if pin else 0, ctypes.byref(slot), ctypes.byref(hit),
                                         ctypes.byref(ev)), "cache_acquire")
     return slot.value, bool(hit.value), ev.value
+
+
+def edgelora_cache_select(cache, scores: np.ndarray, k: int, pin: bool = False):
+    """Returns (adapter, block, hit, evicted key or -1); scores is a float32 numpy array."""
+    assert scores.dtype == np.float32 and scores.flags.c_contiguous
+    key, slot, hit, ev = ctypes.c_int64(), ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int64()
+    _check(lib().edgelora_cache_select(cache, scores.ctypes.data, int(scores.shape[0]), k, 1 if pin else 0,
+                                       ctypes.byref(key), ctypes.byref(slot), ctypes.byref(hit), ctypes.byref(ev)),
+           "cache_select")
+    return key.value, slot.value, bool(hit.value), ev.value
 
 
 def edgelora_cache_release(cache, key: int) -> None:

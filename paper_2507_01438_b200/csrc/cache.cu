@@ -121,6 +121,37 @@ int edgelora_cache_acquire(edgelora_cache_t *c, int64_t key, int32_t pin, int32_
   return EDGELORA_OK;
 }
 
+// Paper Algorithm 1, second half (Section 3.2): of the k adapters with the highest router scores,
+// in descending order of score (equal scores: lower index first), the first resident one is
+// used; if none is resident the best-scored one is admitted (and has to be loaded).
+int edgelora_cache_select(edgelora_cache_t *c, const float *scores, int32_t n, int32_t k, int32_t pin,
+                          int64_t *key_out, int32_t *slot_out, int32_t *hit_out, int64_t *evicted_key_out) {
+  if (!c || !scores || n < 1 || k < 1 || !key_out || !slot_out) return EDGELORA_ERR_INVALID_ARG;
+  if (k > n) k = n;
+  // k passes of selection: k is a handful (the paper's settings use 3), n up to thousands
+  std::vector<int32_t> top;
+  std::vector<uint8_t> taken(static_cast<size_t>(n), 0);
+  top.reserve(k);
+  for (int32_t r = 0; r < k; ++r) {
+    int32_t best = -1;
+    for (int32_t j = 0; j < n; ++j) {
+      if (taken[j]) continue;
+      if (best < 0 || scores[j] > scores[best]) best = j;
+    }
+    taken[best] = 1;
+    top.push_back(best);
+  }
+  int64_t chosen = top[0];
+  for (int32_t t : top) {
+    if (c->where.find(t) != c->where.end()) {
+      chosen = t;
+      break;
+    }
+  }
+  *key_out = chosen;
+  return edgelora_cache_acquire(c, chosen, pin, slot_out, hit_out, evicted_key_out);
+}
+
 int edgelora_cache_release(edgelora_cache_t *c, int64_t key) {
   if (!c) return EDGELORA_ERR_INVALID_ARG;
   auto it = c->where.find(key);

@@ -87,3 +87,23 @@ def test_argument_errors():
             B.edgelora_cache_acquire(c, -3)
     finally:
         B.edgelora_cache_destroy(c)
+
+
+@pytest.mark.parametrize("k", [1, 3, 8, 500])
+@pytest.mark.parametrize("policy", [B.CACHE_LRU, B.CACHE_LFU])
+def test_cache_aware_selection_matches_the_oracle(policy, k):
+    # router scores favour a few adapters per request (a sparse sigmoid output), with exact ties
+    from oracle.cache import select_adapter
+    rng = np.random.Generator(np.random.PCG64(50 + k))
+    n = 300
+    ref = AdapterCache(16, policy)
+    c = B.edgelora_cache_create(16, policy)
+    try:
+        for step in range(800):
+            s = (rng.random(n) * 0.05).astype(np.float32)
+            hot = rng.choice(n, size=6, replace=False, p=None)
+            s[hot] = rng.choice(np.array([0.5, 0.7, 0.9, 0.9], dtype=np.float32), size=6)
+            assert B.edgelora_cache_select(c, s, k) == select_adapter(ref, s, k), f"step {step}"
+        assert B.edgelora_cache_stats(c)["hits"] == ref.hits
+    finally:
+        B.edgelora_cache_destroy(c)
