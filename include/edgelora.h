@@ -257,6 +257,16 @@ int edgelora_cache_lookup(const edgelora_cache_t *cache, int64_t key, int32_t *s
 int edgelora_cache_stats(const edgelora_cache_t *cache, int64_t *hits, int64_t *misses,
                          int64_t *evictions, int32_t *resident);
 
+/* Scoring head of the adapter router (Section 3.2: a score s_j in [0, 1] per adapter j for a
+ * prompt): scores_dev[b][j] = sigmoid(sum_k Wr_dev[j][k] * h_dev[b][k] + bias_dev[j]).
+ * Wr_dev [n][hidden] and h_dev [B][hidden] are bfloat16, row-major, 16-byte aligned device memory;
+ * bias_dev [n] float32 or NULL; scores_dev [B][n] float32.  hidden is a multiple of 8, at most
+ * 8192.  fp32 accumulation.  Enqueued on `stream`, asynchronous, no allocation; B == 0 is a
+ * no-op.  The backbone pass that produces h and the training of the router are not part of this
+ * library; the scores feed edgelora_cache_select after a copy to the host. */
+int edgelora_router_scores(const void *Wr_dev, const float *bias_dev, const void *h_dev, int32_t B,
+                           int32_t n, int32_t hidden, float *scores_dev, void *stream);
+
 const char *edgelora_strerror(int code);
 
 #ifdef __cplusplus

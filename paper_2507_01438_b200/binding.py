@@ -31,6 +31,7 @@ EXPORTS = (
     "edgelora_strerror", "edgelora_plan_build_static", "edgelora_lora_linear_host_async",
     "edgelora_pool_host_sync", "edgelora_cache_create", "edgelora_cache_destroy", "edgelora_cache_acquire",
     "edgelora_cache_release", "edgelora_cache_lookup", "edgelora_cache_stats", "edgelora_cache_select",
+    "edgelora_router_scores",
 )
 
 
@@ -74,6 +75,7 @@ def lib() -> ctypes.CDLL:
     L.edgelora_cache_destroy.argtypes = [vp]
     L.edgelora_cache_acquire.argtypes = [vp, i64, i32, cp(i32), cp(i32), cp(i64)]
     L.edgelora_cache_release.argtypes = [vp, i64]
+    L.edgelora_router_scores.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
     L.edgelora_cache_select.argtypes = [vp, vp, i32, i32, i32, cp(i64), cp(i32), cp(i32), cp(i64)]
     L.edgelora_cache_lookup.argtypes = [vp, i64, cp(i32)]
     L.edgelora_cache_stats.argtypes = [vp, cp(i64), cp(i64), cp(i64), cp(i32)]
@@ -309,6 +311,19 @@ def edgelora_cache_select(cache, scores: np.ndarray, k: int, pin: bool = False):
                                        ctypes.byref(key), ctypes.byref(slot), ctypes.byref(hit), ctypes.byref(ev)),
            "cache_select")
     return key.value, slot.value, bool(hit.value), ev.value
+
+
+def edgelora_router_scores(Wr, bias, h, scores=None, stream=None):
+    """Wr [n, hidden], h [B, hidden] bf16 device tensors, bias [n] float32 device tensor or None."""
+    import torch
+    n, hidden = int(Wr.shape[0]), int(Wr.shape[1])
+    Bn = int(h.shape[0])
+    if scores is None:
+        scores = torch.empty((Bn, n), dtype=torch.float32, device=Wr.device)
+    _check(lib().edgelora_router_scores(_dev_ptr(Wr, 2, "Wr"), bias.data_ptr() if bias is not None else None,
+                                        _dev_ptr(h, 2, "h") if Bn else None, Bn, n, hidden, scores.data_ptr(),
+                                        _stream_ptr(stream)), "router_scores")
+    return scores
 
 
 def edgelora_cache_release(cache, key: int) -> None:
