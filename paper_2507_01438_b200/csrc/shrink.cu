@@ -2,9 +2,9 @@
 // (paper Section 2.1 for A: r x h_in; Section 4.3: tokens that share an adapter are handled as one
 // sub-batch so the adapter is fetched once).
 //
-// One CTA per (group, rank row i): it streams row i of A_a once from HBM with 128-bit loads and
-// dots it against the x rows of up to eight tokens of the group at a time; partial sums are
-// reduced with warp shuffles and a small shared-memory stage.  It walks the plan's "short" token
+// One work item per (group, rank row i), strided over the CTAs: a CTA streams row i of A_a once
+// from HBM with 128-bit loads and dots it against the x rows of up to eight tokens of the group at
+// a time; partial sums are reduced with warp shuffles and a small shared-memory stage.  It walks the plan's "short" token
 // lists: in large batches tokens that belong to long runs are left to the segment shrink.
 #include "internal.cuh"
 #include "launch.cuh"
