@@ -261,7 +261,7 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                      const int32_t *__restrict__ ids, const SlotRow *__restrict__ slots,
                      PlanView pv, float *__restrict__ zws, int32_t *__restrict__ group_counters,
                      int32_t T, int32_t h_in, int32_t R_pad, int32_t n_slots, int32_t max_tokens,
-                     int32_t target_items, uint32_t *status) {
+                     int32_t target_items, int32_t late_ticket, uint32_t *status) {
   extern __shared__ uint8_t s_ring_raw[];  // [warp][stage][8 A rows + 4 x rows][512 bytes]
   __shared__ uint64_t s_bars[kShrinkThreads / 32][kDsMaxDepth];
   __shared__ __align__(16) int32_t s_id[256];  // validated id of each token
@@ -467,12 +467,27 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     }
     pend_gi = -1;
   };
+  // When this launch may start under the kernels of the call before it (late_ticket), another
+  // instance of this kernel can still be running, and the counter is theirs until this warp's
+  // dependency wait has returned: the draw then comes after the wait, at the end of the item.
+  const bool use_tickets = n_items > warps_total;  // otherwise the static first round is everything
+  auto draw = [&]() {
+    if (!use_tickets) return n_items;
+    if (!waited) {
+      ptx::pdl_wait_prior_grids();
+      waited = true;
+    }
+    int n = 0;
+    if (lane == 0) n = warps_total + atomicAdd(ticket, 1);
+    return __shfl_sync(0xffffffffu, n, 0);
+  };
   while (ok && item < n_items) {
     int next = 0;
-    if (lane == 0) next = warps_total + atomicAdd(ticket, 1);
-    next = __shfl_sync(0xffffffffu, next, 0);
+    if (!late_ticket) {
+      if (lane == 0 && use_tickets) next = warps_total + atomicAdd(ticket, 1);
+      next = use_tickets ? __shfl_sync(0xffffffffu, next, 0) : n_items;
+    }
     const int cur = item;
-    item = next;
     // consecutive items are the K chunks of one (token block, row group), and chunk c takes the K
     // steps c, c + KS, c + 2 KS, ...: warps that run side by side fetch neighbouring 512-byte
     // pieces of the same rows at about the same time
@@ -487,10 +502,14 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     const int t0 = s_btok[bi], t1 = min(t0 + kDsBlockTok, g_end);
     if (rank <= 0) {
       if (lane == 0 && c == 0 && rg == 0 && t0 == gt0) atomicOr(status, EDGELORA_STATUS_SLOT_EMPTY);
+      item = late_ticket ? draw() : next;
       continue;
     }
     const int n_rg = (rank + 7) >> 3;  // live groups of eight rows
-    if (rg >= n_rg) continue;               // rows past the rank are zero padding: nothing to do
+    if (rg >= n_rg) {  // rows past the rank are zero padding: nothing to do
+      item = late_ticket ? draw() : next;
+      continue;
+    }
     const int step0 = c, step1 = n_ksteps;
     const int q = lane & 3, r = rg * 8 + (lane >> 2);
     for (int tb = t0; ok && tb < t1; tb += kDsTok) {
@@ -527,6 +546,7 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             scale * acc[0];
     }
     if (!ok) break;
+    item = late_ticket ? draw() : next;
     if (KS > 1) {
       pend_gi = gi;
       pend_rg = rg;
@@ -537,7 +557,7 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   }
   // Every warp stops at its first ticket >= n_items, so exactly n_items - (first round) + warps
   // draws happen; the one that drew the last ticket resets the counter for the next launch.
-  if (lane == 0 && ok && !publisher) {
+  if (lane == 0 && ok && !publisher && use_tickets) {
     const int first_round = min(n_items, warps_total);
     const int last_ticket = warps_total + (n_items - first_round) + first_round - 1;
     if (item == last_ticket) *ticket = 0;
@@ -551,6 +571,7 @@ cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &t
                                  int32_t R_pad, int32_t n_slots, int32_t max_tokens,
                                  int32_t target_items, int32_t grid, uint32_t *status, bool pdl,
                                  cudaStream_t stream) {
+  const int32_t late_ticket = pdl ? 1 : 0;  // pdl here = this launch may start under the call before it
   static bool configured = false;  // per process; the attribute is per function and device-wide
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(decode_shrink_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -564,10 +585,10 @@ cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &t
   if (T <= 64)
     return launch_ex(decode_shrink_kernel<2>, dim3(grid), dim3(kShrinkThreads), ds_ring_bytes(2), stream, pdl, 1,
                      tmap_a, tmap_x, ids, slots, pv, zws, group_counters, T, h_in, R_pad, n_slots,
-                     max_tokens, target_items, status);
+                     max_tokens, target_items, late_ticket, status);
   return launch_ex(decode_shrink_kernel<4>, dim3(grid), dim3(kShrinkThreads), ds_ring_bytes(4), stream, pdl, 1,
                    tmap_a, tmap_x, ids, slots, pv, zws, group_counters, T, h_in, R_pad, n_slots,
-                   max_tokens, target_items, status);
+                   max_tokens, target_items, late_ticket, status);
 }
 
 }  // namespace edgelora

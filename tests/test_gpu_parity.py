@@ -308,6 +308,52 @@ def test_pipelined_host_buffer_entry_point():
         pool.close()
 
 
+@pytest.mark.parametrize("pdl", [1, 2])
+@pytest.mark.parametrize("T,h_in,h_out,max_rank", [(32, 4096, 4096, 16), (200, 1024, 1024, 32)])
+def test_cuda_graph_replay_in_the_benchmarks_launch_configuration(pdl, T, h_in, h_out, max_rank):
+    # bench.py replays a CUDA graph of consecutive calls, with programmatic dependent launch inside
+    # a call (1) or also across calls (2: the next call's shrink starts under this call's base
+    # product).  Three different batches through one pool, captured twice over, replayed three times.
+    import torch
+    base = random_workload(500 + T, T, h_in, h_out, ranks=[max_rank, 8, max_rank, 4, 16, 8], max_rank=max_rank)
+    rng = np.random.Generator(np.random.PCG64(600 + T))
+    batches = []
+    for i in range(3):
+        x = wl.normal_bf16(rng, (T, h_in), 1.0)
+        ids = rng.integers(-1, 6, size=T).astype(np.int32)
+        batches.append(wl.Workload(f"graph{i}", h_in, h_out, base.n_slots, max_rank, base.W, x, ids, base.adapters))
+    pool = make_pool(base)
+    try:
+        B.edgelora_pool_set_option(pool.handle, B.OPT_PDL, pdl)
+        W = to_dev_bf16(base.W)
+        xs = [to_dev_bf16(b.x) for b in batches]
+        ids = [torch.from_numpy(b.ids).cuda() for b in batches]
+        ys = [torch.zeros((T, h_out), dtype=torch.bfloat16, device="cuda") for _ in batches]
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            for i in range(3):
+                B.edgelora_lora_linear(pool.handle, W, xs[i], ids[i], ys[i], stream)
+        stream.synchronize()
+        eager = [from_dev_bf16(y) for y in ys]
+        for y in ys:
+            y.zero_()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(6):
+                B.edgelora_lora_linear(pool.handle, W, xs[i % 3], ids[i % 3], ys[i % 3], stream)
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                graph.replay()
+        stream.synchronize()
+        assert pool.status() == (0, 0)
+        for b, y, e in zip(batches, ys, eager):
+            got = from_dev_bf16(y)
+            assert_parity(got, oracle_of(b), f"graph replay pdl={pdl} T={T}")
+            assert np.array_equal(got, e)
+    finally:
+        pool.close()
+
+
 def test_profiling_option_reports_every_kernel():
     w = random_workload(41, 300, 256, 256, ranks=[16, 16], max_rank=16, id_mode="runs", run_len=64)
     pool = make_pool(w, 512)
