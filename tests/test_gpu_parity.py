@@ -309,7 +309,7 @@ def test_pipelined_host_buffer_entry_point():
 
 
 @pytest.mark.parametrize("pdl", [1, 2])
-@pytest.mark.parametrize("T,h_in,h_out,max_rank", [(32, 4096, 4096, 16), (200, 1024, 1024, 32), (400, 512, 640, 16)])
+@pytest.mark.parametrize("T,h_in,h_out,max_rank", [(32, 4096, 4096, 16), (200, 1024, 1024, 32), (256, 2048, 512, 64), (400, 512, 640, 16)])
 def test_cuda_graph_replay_in_the_benchmarks_launch_configuration(pdl, T, h_in, h_out, max_rank):
     # bench.py replays a CUDA graph of consecutive calls, with programmatic dependent launch inside
     # a call (1) or also across calls (2: the next call's shrink starts under this call's base
