@@ -331,6 +331,23 @@ def main():
     ms = max_over_ranks(ms, world, "cuda")
     value = aggregate_tokens_per_s(w.T, args.steps, world, ms * 1e-3)
 
+    # ---- spread over 20 windows of the same steps (one event at every window boundary)
+    n_win = 20
+    win_steps = per_graph if graph is not None else max(1, args.steps // (n_win * 5))
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_win + 1)]
+    barrier()
+    t_start = time.time()
+    evs[0].record(stream)
+    for i in range(n_win):
+        run_steps(win_steps)
+        evs[i + 1].record(stream)
+    barrier()
+    windows.append((t_start, time.time()))
+    per_step = sorted(evs[i].elapsed_time(evs[i + 1]) / win_steps for i in range(n_win))
+    iterations = {"windows": n_win, "steps_per_window": int(win_steps),
+                  "ms_per_step_median": 0.5 * (per_step[n_win // 2 - 1] + per_step[n_win // 2]),
+                  "ms_per_step_best": per_step[0], "ms_per_step_worst": per_step[-1]}
+
     dependent = None
     if pdl_mode == 2:   # same steps with the library's default launch mode, plain stream launches
         for p_ in pools:
@@ -451,6 +468,7 @@ def main():
         "kernels_per_step": info["launches"],
         "roofline": roof,
         "step_roofline_frac": step_frac,
+        "iterations": iterations,
         "kernel_ms_profiled": {k: v for k, v in kt.items() if v["launches"]},
     }
     if dependent is not None:
