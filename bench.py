@@ -468,7 +468,8 @@ def main():
         peak = pk["hbm_gbs"]
         roof = {"bound": "hbm", "kernel": "lora_gemm_kernel (decode mode)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "traffic": ncu_traffic(args.workload),
-                "algorithmic_bytes": gemm_bytes, "kernel_us": gemm_us, "peak_source": pk["_source"] + ", burst copy"}
+                "algorithmic_bytes": gemm_bytes, "kernel_us": gemm_us, "peak_source": pk["_source"] + ", burst copy",
+                "frac_of_nominal": achieved / 7700.0, "nominal": "7.7 TB/s HBM3e (HGX B200)"}
         step_frac = (ws_bytes / (ms * 1e-3 / args.steps) / 1e9) / peak
     else:
         gemm_flops = 2.0 * w.T * w.h_in * w.h_out + 2.0 * sum(w.adapters[int(a)].rank for a in w.ids if a >= 0) * w.h_out
@@ -476,7 +477,8 @@ def main():
         peak = pk["bf16_tflops"]
         roof = {"bound": "tensor", "kernel": "lora_gemm_kernel (prefill mode)", "achieved": achieved, "peak": peak,
                 "unit": "TFLOP/s", "frac": achieved / peak, "traffic": ncu_traffic(args.workload),
-                "algorithmic_flops": gemm_flops, "kernel_us": gemm_us, "peak_source": pk["_source"] + ", burst"}
+                "algorithmic_flops": gemm_flops, "kernel_us": gemm_us, "peak_source": pk["_source"] + ", burst",
+                "frac_of_nominal": achieved / 2250.0, "nominal": "2.25 PFLOP/s dense bf16"}
         step_frac = (w.algorithmic_flops() / (ms * 1e-3 / args.steps) / 1e12) / peak
 
     if rank == 0:
