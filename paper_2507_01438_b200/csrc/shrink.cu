@@ -31,7 +31,7 @@ __global__ void __launch_bounds__(kBgmvThreads)
 bgmv_shrink_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ A_pool,
                    const SlotRow *__restrict__ slots, PlanView pv, float *__restrict__ zws,
                    int32_t T, int32_t h_in, int32_t R_pad, int32_t zsplits, int32_t max_tokens,
-                   uint32_t *status) {
+                   int32_t max_groups, uint32_t *status) {
   __shared__ float red[kBgmvThreads / 32][kBgmvTok];
   __shared__ int32_t tok[kBgmvTok];
 
@@ -41,14 +41,22 @@ bgmv_shrink_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ 
   // Work items (group, rank row) are strided over a grid sized for the machine, not for the worst
   // case of groups: most batches have far fewer groups than slots, and CTAs that only find out
   // that they have nothing to do cost more than the items themselves.
-  const int n_work = pv.counts[0] * R_pad;
-  for (int wi = blockIdx.x; wi < n_work; wi += gridDim.x) {
+  // The plan arrays are cold by the time they are read here (a step streams gigabytes between
+  // two uses), so an item is a chain of dependent DRAM round trips; loads that do not depend on
+  // each other are issued together: {group count, the group's adapter and token range} (g is
+  // below the host's bound on groups, so these reads stay inside the arrays whatever the count
+  // turns out to be), then {slot row, first tokens}, then the rows themselves.
+  for (int wi = blockIdx.x; wi / R_pad < max_groups; wi += gridDim.x) {
   const int g = wi / R_pad;
   const int i = wi % R_pad;
+  const int n_groups = pv.counts[0];
   const int a = pv.group_adapter[g];
-  if (a < 0) continue;
-  const SlotRow row = slots[a];
   const int g0 = pv.gs_short[g], g1 = pv.gs_short[g + 1];
+  if (g >= n_groups) break;
+  if (a < 0) continue;
+  int32_t first_tok = 0;
+  if (static_cast<int>(threadIdx.x) < min(kBgmvTok, g1 - g0)) first_tok = pv.perm_short[g0 + threadIdx.x];
+  const SlotRow row = slots[a];
   if (row.rank <= 0) {
     if (threadIdx.x == 0 && i == 0) atomicOr(status, EDGELORA_STATUS_SLOT_EMPTY);
     continue;
@@ -63,7 +71,7 @@ bgmv_shrink_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ 
   for (int base = g0; base < g1; base += kBgmvTok) {
     const int n_tok = min(kBgmvTok, g1 - base);
     __syncthreads();
-    if (threadIdx.x < n_tok) tok[threadIdx.x] = pv.perm_short[base + threadIdx.x];
+    if (threadIdx.x < n_tok) tok[threadIdx.x] = base == g0 ? first_tok : pv.perm_short[base + threadIdx.x];
     __syncthreads();
 
     if (!live_row) {  // padding rows of the block: z is defined as zero there
@@ -73,18 +81,22 @@ bgmv_shrink_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ 
     }
 
     float acc[kBgmvTok];
+    const uint4 *xrow[kBgmvTok];
 #pragma unroll
-    for (int q = 0; q < kBgmvTok; ++q) acc[q] = 0.f;
+    for (int q = 0; q < kBgmvTok; ++q) {
+      acc[q] = 0.f;
+      xrow[q] = reinterpret_cast<const uint4 *>(x + static_cast<size_t>(tok[min(q, n_tok - 1)]) * h_in);
+    }
+    // every load of a K step is issued before the first product: with the loads inside the
+    // per-token branches a step cost one memory round trip per token (4 us per token on a
+    // 14336-wide row)
     for (int k = threadIdx.x; k < n8; k += kBgmvThreads) {
       const uint4 av = __ldg(Arow + k);
+      uint4 xv[kBgmvTok];
 #pragma unroll
-      for (int q = 0; q < kBgmvTok; ++q) {
-        if (q < n_tok) {
-          const uint4 xv =
-              __ldg(reinterpret_cast<const uint4 *>(x + static_cast<size_t>(tok[q]) * h_in) + k);
-          acc[q] += dot8(av, xv);
-        }
-      }
+      for (int q = 0; q < kBgmvTok; ++q) xv[q] = q < n_tok ? __ldg(xrow[q] + k) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int q = 0; q < kBgmvTok; ++q) acc[q] += dot8(av, xv[q]);
     }
 #pragma unroll
     for (int q = 0; q < kBgmvTok; ++q) {
@@ -119,7 +131,7 @@ void launch_bgmv_shrink(const uint16_t *x, const uint16_t *A_pool, const SlotRow
   }
   const int grid = max_groups * R_pad < sms * 8 ? max_groups * R_pad : sms * 8;
   launch_ex(bgmv_shrink_kernel, dim3(grid), dim3(kBgmvThreads), 0, stream, pdl, 1, x,
-            A_pool, slots, pv, zws, T, h_in, R_pad, zsplits, max_tokens, status);
+            A_pool, slots, pv, zws, T, h_in, R_pad, zsplits, max_tokens, max_groups, status);
 }
 
 }  // namespace edgelora
