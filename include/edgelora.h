@@ -86,6 +86,9 @@ typedef struct {
                                     call before it (independent sites / batches)                  */
 #define EDGELORA_OPT_DECODE_SPLITS 4 /* tuning: K splits per W row tile in decode, 0 = automatic  */
 #define EDGELORA_OPT_SHRINK_ITEMS 5  /* tuning: work items the decode shrink aims for, 0 = auto   */
+#define EDGELORA_OPT_WAIT_CYCLES 6   /* limit of every bounded in-kernel wait of the layer, in units
+                                        of 1024 SM clock cycles; 0 = default (about two seconds).
+                                        A wait that runs out raises EDGELORA_STATUS_TIMEOUT           */
 
 /* Bytes of device memory the slot blocks need for this geometry (what arena_bytes must
  * be at least).  Host-only arithmetic. */
@@ -101,8 +104,15 @@ int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool
  * `slot`, asynchronously: the data is first copied into pinned staging (so the caller may
  * free A_host / B_host on return), then moved with cudaMemcpyAsync on the pool's side
  * stream.  The copy waits for the last edgelora_lora_linear call issued before it, and
- * later edgelora_lora_linear calls wait for the copy, so a call never sees a half-written
- * block; the caller must not reload a slot that ids of a still-queued call refer to.
+ * later edgelora_lora_linear calls (on any stream) wait for the copy, so a call never sees a
+ * half-written block; the caller must not reload a slot that ids of a still-queued call refer
+ * to.  When several streams run calls of one pool, the copy waits only for the most recent
+ * call: order the others yourself.
+ * CUDA graphs: a call issued while its stream is being captured records neither of these
+ * waits (an event wait inside a graph would name a load that is long gone at replay).  The
+ * owner of a graph therefore calls edgelora_pool_wait_loads before capturing and before any
+ * replay that follows a load, and synchronises the replays' stream before reloading a slot
+ * their ids use.
  * rank must be in [1, max_rank]; scale is s_a. */
 int edgelora_pool_load_slot(edgelora_pool_t *pool, int32_t slot, int32_t rank, float scale,
                             const uint16_t *A_host, const uint16_t *B_host);
@@ -120,7 +130,8 @@ int edgelora_pool_wait_loads(edgelora_pool_t *pool);
  * routing plan -> shrink (z = s_a A_a x) -> base product W x on the tensor cores with
  * the expand B_a z accumulated into the same tile (z rounded to bfloat16 for it) -> y written
  * once.  Asynchronous; no host synchronisation, no
- * allocation.  T == 0 is a no-op.  x_dev / y_dev must not alias. */
+ * allocation.  T == 0 is a no-op.  x_dev / y_dev must not alias.  Calls of one pool share its
+ * workspaces: they must not overlap on the GPU (one stream, or ordered by events). */
 int edgelora_lora_linear(edgelora_pool_t *pool, const void *W_dev, const void *x_dev,
                          const int32_t *adapter_id_dev, int32_t T, void *y_dev, void *stream);
 
@@ -167,6 +178,11 @@ int edgelora_lora_linear_planned(edgelora_pool_t *pool, edgelora_plan_t *plan, c
                                  const void *x_dev, int32_t T, void *y_dev, void *stream);
 /* The pool's own plan object (the one edgelora_lora_linear builds each call). */
 int edgelora_pool_plan(edgelora_pool_t *pool, edgelora_plan_t **plan_out);
+/* Status word of a plan built with edgelora_plan_build (an id outside [-1, n_slots) raises
+ * EDGELORA_STATUS_BAD_ADAPTER_ID there, not in the pools that later use the plan): synchronises
+ * `stream`, returns the bits in *bits_out (may be NULL), clears them; return value as for
+ * edgelora_pool_sync_status. */
+int edgelora_plan_sync_status(edgelora_plan_t *plan, void *stream, uint32_t *bits_out);
 
 /* No counterpart in the paper: a routing-plan builder for callers that cannot allocate.
  *
@@ -202,6 +218,14 @@ int edgelora_plan_build_static(const int32_t *adapter_id_dev, int32_t T, int32_t
 int edgelora_pool_sync_status(edgelora_pool_t *pool, uint32_t *bits_out);
 
 int edgelora_pool_set_option(edgelora_pool_t *pool, int32_t option, int32_t value);
+
+/* Self-test of the time-out path.  Enqueues on `stream` a one-thread kernel that waits, with the
+ * pool's wait limit, on a shared-memory barrier nothing arrives at; the wait runs out, the kernel
+ * raises EDGELORA_STATUS_TIMEOUT in the pool's status word and returns.  Nothing else is touched
+ * and the context stays usable: edgelora_pool_sync_status then reports EDGELORA_ERR_TIMEOUT once.
+ * Only with EDGELORA_OPT_WAIT_CYCLES lowered to at most 16384 (16 M cycles); otherwise
+ * EDGELORA_ERR_INVALID_ARG and nothing is launched. */
+int edgelora_pool_selftest_wait(edgelora_pool_t *pool, void *stream);
 
 /* Launch bookkeeping for measurement.  info_out[0] = kernels launched by the last
  * edgelora_lora_linear call, [1] = regime used (1 decode, 2 prefill), [2] = grid of the

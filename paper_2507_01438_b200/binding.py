@@ -18,8 +18,8 @@ OK = 0
 ERR_INVALID_ARG, ERR_BAD_SLOT, ERR_RANK_TOO_LARGE, ERR_ARENA_TOO_SMALL = -1, -2, -3, -4
 ERR_CUDA, ERR_BAD_ADAPTER_ID, ERR_SLOT_EMPTY, ERR_TIMEOUT, ERR_TOO_MANY_TOKENS = -5, -6, -7, -8, -9
 STATUS_BAD_ADAPTER_ID, STATUS_SLOT_EMPTY, STATUS_TIMEOUT = 0x1, 0x2, 0x4
-OPT_REGIME, OPT_PROFILE, OPT_PDL, OPT_DECODE_SPLITS, OPT_SHRINK_ITEMS = 1, 2, 3, 4, 5
-KERNEL_NAMES = ("plan", "shrink_bgmv", "shrink_sgmv", "base_gemm", "decode_combine")
+OPT_REGIME, OPT_PROFILE, OPT_PDL, OPT_DECODE_SPLITS, OPT_SHRINK_ITEMS, OPT_WAIT_CYCLES = 1, 2, 3, 4, 5, 6
+KERNEL_NAMES = ("plan", "shrink_bgmv", "shrink_sgmv", "base_gemm")
 
 EXPORTS = (
     "edgelora_pool_bytes_required", "edgelora_pool_create", "edgelora_pool_load_slot",
@@ -31,7 +31,7 @@ EXPORTS = (
     "edgelora_strerror", "edgelora_plan_build_static", "edgelora_lora_linear_host_async",
     "edgelora_pool_host_sync", "edgelora_cache_create", "edgelora_cache_destroy", "edgelora_cache_acquire",
     "edgelora_cache_release", "edgelora_cache_lookup", "edgelora_cache_stats", "edgelora_cache_select",
-    "edgelora_router_scores",
+    "edgelora_router_scores", "edgelora_plan_sync_status", "edgelora_pool_selftest_wait",
 )
 
 
@@ -86,6 +86,8 @@ def lib() -> ctypes.CDLL:
     L.edgelora_lora_linear_planned.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     L.edgelora_plan_build_static.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.edgelora_pool_plan.argtypes = [vp, cp(vp)]
+    L.edgelora_plan_sync_status.argtypes = [vp, vp, cp(ctypes.c_uint32)]
+    L.edgelora_pool_selftest_wait.argtypes = [vp, vp]
     L.edgelora_pool_sync_status.argtypes = [vp, cp(ctypes.c_uint32)]
     L.edgelora_pool_set_option.argtypes = [vp, i32, i32]
     L.edgelora_pool_last_launch.argtypes = [vp, vp]
@@ -255,6 +257,20 @@ def edgelora_pool_sync_status(pool):
     if rc == ERR_CUDA or rc == ERR_INVALID_ARG:
         raise EdgeLoraError(rc, "pool_sync_status")
     return rc, bits.value
+
+
+def edgelora_plan_sync_status(plan, stream=None):
+    """Returns (return code, status bits) of a plan built with edgelora_plan_build; clears the bits."""
+    bits = ctypes.c_uint32(0)
+    rc = lib().edgelora_plan_sync_status(plan, _stream_ptr(stream), ctypes.byref(bits))
+    if rc == ERR_CUDA or rc == ERR_INVALID_ARG:
+        raise EdgeLoraError(rc, "plan_sync_status")
+    return rc, bits.value
+
+
+def edgelora_pool_selftest_wait(pool, stream=None) -> int:
+    """Returns the C return code (INVALID_ARG unless the pool's wait limit was lowered first)."""
+    return lib().edgelora_pool_selftest_wait(pool, _stream_ptr(stream))
 
 
 def edgelora_pool_set_option(pool, option: int, value: int) -> None:

@@ -210,6 +210,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   uint32_t *s_key = reinterpret_cast<uint32_t *>(extra + 2432);             // [256] sort keys
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wl = p.wait_cycles;  // limit of every bounded wait below
   // LoRA K blocks: prefill always; decode unless the batch is small enough for the expand to be
   // added by the owners of the cluster reduction (then z is needed only at the very end and the
   // whole main loop overlaps the shrink kernel)
@@ -258,7 +259,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
         const TileCoord tc = tile_coord(p, tile);
         for (int32_t kb = tc.kb0; kb < tc.kb1; ++kb) {
-          if (!ptx::mbar_wait(&empty_bar[stage], phase ^ 1) || *abort_flag) {
+          if (!ptx::mbar_wait(&empty_bar[stage], phase ^ 1, wl) || *abort_flag) {
             ok = false;
             break;
           }
@@ -277,7 +278,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         if (!ok || !has_lora) continue;
         if (!waited) {
           if (p.mode == kModeDecode) {  // the builder warps derive the adapter list from the ids
-            if (!ptx::mbar_wait(lg_bar, 0)) {
+            if (!ptx::mbar_wait(lg_bar, 0, wl)) {
               ok = false;
               break;
             }
@@ -290,7 +291,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
           const int32_t a = ll.list[e];
           if (p.mode != kModeDecode && p.slots[a].rank <= 0) continue;
-          if (!ptx::mbar_wait(&empty_bar[stage], phase ^ 1) || *abort_flag) {
+          if (!ptx::mbar_wait(&empty_bar[stage], phase ^ 1, wl) || *abort_flag) {
             ok = false;
             break;
           }
@@ -328,14 +329,14 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         const TileCoord tc = tile_coord(p, tile);
         const uint32_t acc = (p.n_acc == 2) ? (it & 1) : 0;
         const uint32_t use = (p.n_acc == 2) ? (it >> 1) : it;
-        if (!ptx::mbar_wait(&tempty_bar[acc], (use & 1) ^ 1) || *abort_flag) {
+        if (!ptx::mbar_wait(&tempty_bar[acc], (use & 1) ^ 1, wl) || *abort_flag) {
           ok = false;
           break;
         }
         ptx::tc_fence_after_sync();
         const uint32_t tmem_d = tmem_base + acc * static_cast<uint32_t>(p.BN);
         for (int32_t kb = tc.kb0; kb < tc.kb1; ++kb) {
-          if (!ptx::mbar_wait(&full_bar[stage], phase) || *abort_flag) {
+          if (!ptx::mbar_wait(&full_bar[stage], phase, wl) || *abort_flag) {
             ok = false;
             break;
           }
@@ -358,7 +359,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         if (has_lora) {
           if (!waited) {
             if (p.mode == kModeDecode) {
-              if (!ptx::mbar_wait(lg_bar, 0)) {
+              if (!ptx::mbar_wait(lg_bar, 0, wl)) {
                 ok = false;
                 break;
               }
@@ -371,8 +372,8 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
           for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
             const int32_t a = ll.list[e];
             if (p.mode != kModeDecode && p.slots[a].rank <= 0) continue;
-            if (!ptx::mbar_wait(&full_bar[stage], phase) ||
-                !ptx::mbar_wait(&zfull_bar[stage], (zphase >> stage) & 1u) || *abort_flag) {
+            if (!ptx::mbar_wait(&full_bar[stage], phase, wl) ||
+                !ptx::mbar_wait(&zfull_bar[stage], (zphase >> stage) & 1u, wl) || *abort_flag) {
               ok = false;
               break;
             }
@@ -445,7 +446,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       float scale = 0.f;
       if (p.mode == kModeSgmv) scale = p.slots[tc.slot].scale;
 
-      const bool got = ptx::mbar_wait(&tfull_bar[acc], use & 1) && !*abort_flag;
+      const bool got = ptx::mbar_wait(&tfull_bar[acc], use & 1, wl) && !*abort_flag;
       if (!got) {
         ok = false;
         *abort_flag = 1;
@@ -616,7 +617,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         if (p.mode != kModeDecode && p.slots[a].rank <= 0) continue;
         const uint32_t stage = count % nstages;
         ++count;
-        if (!ptx::mbar_wait(&zgo_bar[stage], (gophase >> stage) & 1u) || *abort_flag) {
+        if (!ptx::mbar_wait(&zgo_bar[stage], (gophase >> stage) & 1u, wl) || *abort_flag) {
           ok = false;
           break;
         }

@@ -69,6 +69,7 @@ struct GemmParams {
   int32_t expand_in_reduce;  // decode, small batches: B_a z is added by the owners of the cluster
                              // reduction on the CUDA cores instead of by LoRA K blocks
   int32_t max_tokens;  // row stride of the z / plan workspaces
+  long long wait_cycles;  // limit of the bounded in-kernel waits, in SM clock cycles
   const int32_t *ids_valid;
   const int32_t *ids;       // decode: the caller's ids (validated again inside the kernel)
   int32_t n_slots;
@@ -84,18 +85,20 @@ struct GemmParams {
   uint32_t *status;
 };
 
-// kernels (defined in plan.cu, shrink.cu, gemm.cu, combine.cu)
+// kernels (defined in plan.cu, shrink.cu, gemm.cu)
 void launch_plan(const int32_t *ids, int32_t T, int32_t n_slots, const PlanView &pv, bool pdl,
                  cudaStream_t stream);
 void launch_bgmv_shrink(const uint16_t *x, const uint16_t *A_pool, const SlotRow *slots,
                         const PlanView &pv, float *zws, int32_t T, int32_t h_in, int32_t R_pad,
-                        int32_t n_slots, int32_t zsplits, int32_t max_tokens, uint32_t *status,
-                        bool pdl, cudaStream_t stream);
+                        int32_t n_slots, int32_t zsplits, int32_t max_tokens, int32_t sms,
+                        uint32_t *status, bool pdl, cudaStream_t stream);
 void init_plan_kernel();
 cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
                         const CUtensorMap &tmap_b, const GemmParams &p, int32_t grid,
                         size_t smem_bytes, bool pdl, cudaStream_t stream);
 cudaError_t gemm_set_smem_limit(size_t smem_bytes);
+cudaError_t shrink_set_smem_limit();
+cudaError_t launch_wait_selftest(uint32_t *status, long long wait_cycles, cudaStream_t stream);
 cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &tmap_x,
                                  const int32_t *ids, const SlotRow *slots, const PlanView &pv,
                                  float *zws, int32_t *group_counters, int32_t T, int32_t h_in,

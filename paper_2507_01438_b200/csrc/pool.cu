@@ -10,9 +10,11 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "internal.cuh"
+#include "ptx.cuh"
 
 using namespace edgelora;
 
@@ -127,7 +129,8 @@ struct edgelora_pool {
   int next_staging = 0;
   cudaStream_t side = nullptr;
   cudaEvent_t load_ev = nullptr, use_ev = nullptr;
-  uint64_t load_seq = 0, load_seq_waited = 0;
+  uint64_t load_seq = 0;
+  std::vector<std::pair<cudaStream_t, uint64_t>> load_waited;  // per stream: last load it waited for
   bool use_recorded = false;
   edgelora_plan *plan = nullptr;
   float *zws = nullptr;
@@ -137,6 +140,7 @@ struct edgelora_pool {
   std::vector<TmapEntry> tmaps;
   size_t tmap_next = 0;
   int opt_regime = 0, opt_profile = 0, opt_pdl = 1;
+  long long wait_cycles = ptx::kWaitLimitCycles;
   int64_t last_info[8] = {0};
   int64_t total_launches = 0;
   // profiling
@@ -157,24 +161,25 @@ struct edgelora_pool {
 
 namespace {
 
-int get_tmap(edgelora_pool *p, const CUtensorMap **out, const void *base, uint64_t d0, uint64_t d1,
+// The descriptor is copied out: a later miss of the same call may reuse the cache entry it came
+// from (the cache is a ring), and the launch takes its descriptors by value anyway.
+int get_tmap(edgelora_pool *p, CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1,
              uint64_t d2, uint32_t box_rows, uint32_t box_cols = kBlockK) {
   TmapKey key{base, d0, d1, d2, box_rows, box_cols};
   for (auto &e : p->tmaps)
     if (e.key == key) {
-      *out = &e.map;
+      *out = e.map;
       return EDGELORA_OK;
     }
   TmapEntry e;
   e.key = key;
   int rc = encode_tmap(&e.map, base, d0, d1, d2, box_rows, box_cols);
   if (rc != EDGELORA_OK) return rc;
+  *out = e.map;
   if (p->tmaps.size() < static_cast<size_t>(kTmapCache)) {
     p->tmaps.push_back(e);
-    *out = &p->tmaps.back().map;
   } else {
     p->tmaps[p->tmap_next] = e;
-    *out = &p->tmaps[p->tmap_next].map;
     p->tmap_next = (p->tmap_next + 1) % kTmapCache;
   }
   return EDGELORA_OK;
@@ -422,6 +427,7 @@ int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool
   POOL_TRY(cudaMalloc(&p->group_counters, sizeof(int32_t) * (kDecodeMaxT * 8 + 32)));
   POOL_TRY(cudaMemset(p->group_counters, 0, sizeof(int32_t) * (kDecodeMaxT * 8 + 32)));
   POOL_TRY(gemm_set_smem_limit(kSmemBudget));
+  POOL_TRY(shrink_set_smem_limit());
   rc = edgelora_plan_create(p->cfg.max_tokens, cfg->n_slots, &p->plan);
   if (rc != EDGELORA_OK) {
     edgelora_pool_destroy(p);
@@ -568,6 +574,10 @@ int edgelora_pool_set_option(edgelora_pool_t *p, int32_t option, int32_t value) 
       if (value < 0 || value > kMaxDecodeSplits) return EDGELORA_ERR_INVALID_ARG;
       p->opt_decode_splits = value;
       return EDGELORA_OK;
+    case EDGELORA_OPT_WAIT_CYCLES:
+      if (value < 0) return EDGELORA_ERR_INVALID_ARG;
+      p->wait_cycles = value == 0 ? ptx::kWaitLimitCycles : static_cast<long long>(value) * 1024;
+      return EDGELORA_OK;
     case EDGELORA_OPT_SHRINK_ITEMS:
       if (value < 0) return EDGELORA_ERR_INVALID_ARG;
       p->opt_shrink_items = value;
@@ -623,6 +633,28 @@ int edgelora_pool_sync_status(edgelora_pool_t *p, uint32_t *bits_out) {
   return EDGELORA_OK;
 }
 
+int edgelora_plan_sync_status(edgelora_plan_t *plan, void *stream, uint32_t *bits_out) {
+  if (!plan) return EDGELORA_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  CUDA_TRY(cudaStreamSynchronize(s));
+  uint32_t bits = 0;
+  CUDA_TRY(cudaMemcpy(&bits, plan->pv.status, 4, cudaMemcpyDeviceToHost));
+  CUDA_TRY(cudaMemset(plan->pv.status, 0, 4));
+  if (bits_out) *bits_out = bits;
+  if (bits & EDGELORA_STATUS_TIMEOUT) return EDGELORA_ERR_TIMEOUT;
+  if (bits & EDGELORA_STATUS_BAD_ADAPTER_ID) return EDGELORA_ERR_BAD_ADAPTER_ID;
+  if (bits & EDGELORA_STATUS_SLOT_EMPTY) return EDGELORA_ERR_SLOT_EMPTY;
+  return EDGELORA_OK;
+}
+
+int edgelora_pool_selftest_wait(edgelora_pool_t *p, void *stream) {
+  if (!p) return EDGELORA_ERR_INVALID_ARG;
+  // only with a lowered limit: at the default the kernel would spin for seconds
+  if (p->wait_cycles > (1LL << 24)) return EDGELORA_ERR_INVALID_ARG;
+  CUDA_TRY(launch_wait_selftest(p->status_dev, p->wait_cycles, static_cast<cudaStream_t>(stream)));
+  return EDGELORA_OK;
+}
+
 // The layer.  Decode regime (T <= 256): routing + shrink in one kernel, then the base product with
 // the expand and the split-K reduction fused in.  Prefill regime: plan, gather shrink for short
 // runs, segment shrink for long runs, base product with the expand fused in.
@@ -645,9 +677,21 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
   const uint16_t *x = static_cast<const uint16_t *>(x_dev);
   int launches = 0;
 
-  if (p->load_seq != p->load_seq_waited && !capturing) {
-    CUDA_TRY(cudaStreamWaitEvent(stream, p->load_ev, 0));
-    p->load_seq_waited = p->load_seq;
+  // Order this call behind every load issued so far, once per stream and load (a wait node
+  // between two calls of one stream would also keep them from overlapping).  A captured call
+  // records no such wait: see the header for what a graph's owner has to do instead.
+  if (p->load_seq != 0 && !capturing) {
+    auto it = std::find_if(p->load_waited.begin(), p->load_waited.end(),
+                           [&](const std::pair<cudaStream_t, uint64_t> &e) { return e.first == stream; });
+    if (it == p->load_waited.end()) {
+      if (p->load_waited.size() >= 64) p->load_waited.clear();  // streams come and go: start over
+      p->load_waited.emplace_back(stream, 0);
+      it = p->load_waited.end() - 1;
+    }
+    if (it->second != p->load_seq) {
+      CUDA_TRY(cudaStreamWaitEvent(stream, p->load_ev, 0));
+      it->second = p->load_seq;
+    }
   }
 
   int regime = (T <= kDecodeMaxT) ? 1 : 2;
@@ -675,6 +719,7 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
   g.mt_count = plan->pv.mt_count;
   g.mt_list = plan->pv.mt_list;
   g.status = p->status_dev;
+  g.wait_cycles = p->wait_cycles;
 
   auto smem_for = [](int stages, int BN) {
     // alignment slack + operand ring + barriers (512) + decode extras (3456, rounded up)
@@ -706,12 +751,12 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
       const int max_chunks = target == 1 ? 1 : std::max(1, std::min(kMaxZSplits, n_ksteps / 4));
       const int max_items = std::min(T, p->cfg.n_slots) * (R / 8) * max_chunks;
       const int grid = std::max(1, std::min(p->sms - 1, (max_items + 7) / 8)) + 1;  // + the publishing CTA
-      const CUtensorMap *ma, *mx;
+      CUtensorMap ma, mx;
       int rc = get_tmap(p, &ma, p->A_pool, h_in, R, p->cfg.n_slots, 8, kShrinkStepElems);
       if (rc) return rc;
       rc = get_tmap(p, &mx, x, h_in, T, 0, 1, kShrinkStepElems);
       if (rc) return rc;
-      CUDA_TRY(launch_decode_shrink(*ma, *mx, ids_in, p->slots_dev, plan->pv, p->zws, p->group_counters,
+      CUDA_TRY(launch_decode_shrink(ma, mx, ids_in, p->slots_dev, plan->pv, p->zws, p->group_counters,
                                     T, h_in, R, p->cfg.n_slots, p->cfg.max_tokens, target, grid,
                                     p->status_dev, pdl_first, stream));
       ++launches;
@@ -759,7 +804,7 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
       ++g.stages;
     g.n_acc = 1;
     g.tmem_cols = pow2_cols(N);
-    const CUtensorMap *mr, *mc, *mb;
+    CUtensorMap mr, mc, mb;
     int rc = get_tmap(p, &mr, W_dev, h_in, h_out, 0, kTileM);
     if (rc) return rc;
     rc = get_tmap(p, &mc, x, h_in, T, 0, N);
@@ -772,7 +817,7 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
       // With one CTA per SM the base product cannot start beside the shrink (both fill an SM's
       // shared memory), and an early launch then only costs: measured 178 vs 122 us per step on
       // the 14336 -> 4096, T = 256 workload.
-      CUDA_TRY(launch_gemm(*mr, *mc, *mb, g, grid, smem_for(g.stages, N), pdl && ctas_per_sm == 2, stream));
+      CUDA_TRY(launch_gemm(mr, mc, mb, g, grid, smem_for(g.stages, N), pdl && ctas_per_sm == 2, stream));
       ++launches;
     }
     p->last_info[2] = grid;
@@ -799,11 +844,11 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     {
       ProfScope ps(p, 1, stream);
       launch_bgmv_shrink(x, p->A_pool, p->slots_dev, plan->pv, p->zws, T, h_in, R, p->cfg.n_slots,
-                         zsplits, p->cfg.max_tokens, p->status_dev, ids_dev ? pdl : pdl_first, stream);
+                         zsplits, p->cfg.max_tokens, p->sms, p->status_dev, ids_dev ? pdl : pdl_first, stream);
       CUDA_TRY(cudaGetLastError());
       ++launches;
     }
-    const CUtensorMap *mx;
+    CUtensorMap mx;
     int rc = get_tmap(p, &mx, x, h_in, T, 0, kTileM);
     if (rc) return rc;
     if (sgmv) {
@@ -815,12 +860,12 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
       s.stages = stages_for(R, s.kb_per, kSmemBudget);
       s.n_acc = 2;
       s.tmem_cols = pow2_cols(2 * R);
-      const CUtensorMap *mc;
+      CUtensorMap mc;
       rc = get_tmap(p, &mc, p->A_pool, h_in, R, p->cfg.n_slots, R);
       if (rc) return rc;
       const int grid = std::max(1, std::min(p->sms, plan->pv.max_sgmv_tiles * zsplits));
       ProfScope ps(p, 2, stream);
-      CUDA_TRY(launch_gemm(*mx, *mc, *mc, s, grid, smem_for(s.stages, R), pdl, stream));
+      CUDA_TRY(launch_gemm(mx, mc, mc, s, grid, smem_for(s.stages, R), pdl, stream));
       ++launches;
     }
     const int n_mtiles = (T + kTileM - 1) / kTileM;
@@ -836,14 +881,14 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     g.stages = stages_for(BN, kb_total, kSmemBudget);
     g.n_acc = 2;
     g.tmem_cols = pow2_cols(2 * BN);
-    const CUtensorMap *mc, *mb;
+    CUtensorMap mc, mb;
     rc = get_tmap(p, &mc, W_dev, h_in, h_out, 0, BN);
     if (rc) return rc;
     rc = get_tmap(p, &mb, p->B_pool, R, h_out, p->cfg.n_slots, BN);
     if (rc) return rc;
     const int grid = std::min(p->sms, g.n_mtiles * g.n_ntiles);
     ProfScope ps(p, 3, stream);
-    CUDA_TRY(launch_gemm(*mx, *mc, *mb, g, grid, smem_for(g.stages, BN), pdl, stream));
+    CUDA_TRY(launch_gemm(mx, mc, mb, g, grid, smem_for(g.stages, BN), pdl, stream));
     ++launches;
     p->last_info[2] = grid;
     p->last_info[3] = 1;

@@ -55,13 +55,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: about two seconds of SM clock, far above any legitimate wait in this library.
+// Bounded wait.  The default limit is about two seconds of SM clock, far above any legitimate
+// wait in this library; a pool can lower it (EDGELORA_OPT_WAIT_CYCLES).
 constexpr long long kWaitLimitCycles = 4000000000LL;
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity,
+                                          long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitLimitCycles) return false;
+    if (clock64() - t0 > limit_cycles) return false;
   }
   return true;
 }

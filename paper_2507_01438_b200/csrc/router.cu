@@ -10,6 +10,7 @@
 #include "ptx.cuh"
 
 #include <algorithm>
+#include <mutex>
 
 namespace edgelora {
 
@@ -92,20 +93,26 @@ extern "C" int edgelora_router_scores(const void *Wr_dev, const float *bias_dev,
   if (B < 0 || n < 1 || hidden < 8 || (hidden & 7) || hidden > 8192) return EDGELORA_ERR_INVALID_ARG;
   if (B == 0) return EDGELORA_OK;
   if (!Wr_dev || !h_dev || !scores_dev) return EDGELORA_ERR_INVALID_ARG;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(router_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kRouterReq * 8192 * 2) != cudaSuccess) {
-      cudaGetLastError();
-      return EDGELORA_ERR_CUDA;
-    }
-    configured = true;
-  }
+  // the shared-memory limit is an attribute of (function, device): kept per device
+  static std::mutex mu;
+  static int sms_of[64] = {0};  // 0 = this device is not configured yet
   int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
     cudaGetLastError();
     return EDGELORA_ERR_CUDA;
+  }
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (sms_of[dev] == 0) {
+      if (cudaFuncSetAttribute(router_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               kRouterReq * 8192 * 2) != cudaSuccess ||
+          cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+        cudaGetLastError();
+        return EDGELORA_ERR_CUDA;
+      }
+      sms_of[dev] = sms;
+    }
+    sms = sms_of[dev];
   }
   const int warps = kRouterThreads / 32;
   const int grid = std::max(1, std::min((n + warps - 1) / warps, sms * 4));

@@ -119,16 +119,9 @@ bgmv_shrink_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ 
 
 void launch_bgmv_shrink(const uint16_t *x, const uint16_t *A_pool, const SlotRow *slots,
                         const PlanView &pv, float *zws, int32_t T, int32_t h_in, int32_t R_pad,
-                        int32_t n_slots, int32_t zsplits, int32_t max_tokens, uint32_t *status,
-                        bool pdl, cudaStream_t stream) {
+                        int32_t n_slots, int32_t zsplits, int32_t max_tokens, int32_t sms,
+                        uint32_t *status, bool pdl, cudaStream_t stream) {
   const int max_groups = (T < n_slots + 1) ? T : n_slots + 1;
-  static int sms = 0;  // same on every device of a node
-  if (sms == 0) {
-    int dev = 0, n = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    sms = n > 0 ? n : 148;
-  }
   const int grid = max_groups * R_pad < sms * 8 ? max_groups * R_pad : sms * 8;
   launch_ex(bgmv_shrink_kernel, dim3(grid), dim3(kBgmvThreads), 0, stream, pdl, 1, x,
             A_pool, slots, pv, zws, T, h_in, R_pad, zsplits, max_tokens, max_groups, status);
@@ -577,6 +570,16 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   if (!ok && lane == 0) atomicOr(status, EDGELORA_STATUS_TIMEOUT);
 }
 
+// The shared-memory limit is an attribute of (function, device): set for the current device, by
+// edgelora_pool_create, so that every device a pool lives on is configured.
+cudaError_t shrink_set_smem_limit() {
+  cudaError_t e = cudaFuncSetAttribute(decode_shrink_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(ds_ring_bytes(4)));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(decode_shrink_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(ds_ring_bytes(2)));
+}
+
 cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &tmap_x,
                                  const int32_t *ids, const SlotRow *slots, const PlanView &pv,
                                  float *zws, int32_t *group_counters, int32_t T, int32_t h_in,
@@ -584,16 +587,6 @@ cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &t
                                  int32_t target_items, int32_t grid, uint32_t *status, bool pdl,
                                  cudaStream_t stream) {
   const int32_t late_ticket = pdl ? 1 : 0;  // pdl here = this launch may start under the call before it
-  static bool configured = false;  // per process; the attribute is per function and device-wide
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(decode_shrink_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(ds_ring_bytes(4)));
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(decode_shrink_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(ds_ring_bytes(2)));
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
   if (T <= 64)
     return launch_ex(decode_shrink_kernel<2>, dim3(grid), dim3(kShrinkThreads), ds_ring_bytes(2), stream, pdl, 1,
                      tmap_a, tmap_x, ids, slots, pv, zws, group_counters, T, h_in, R_pad, n_slots,

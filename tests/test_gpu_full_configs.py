@@ -1,9 +1,11 @@
 """The task's full-size workloads (gate/up prefill, many-tenant down_proj, the 224-site projection set)
-run in the launch configuration the benchmark uses.  The oracle is too slow for every element at
-these sizes, so each check has two parts:
-  - sampled token rows, full width, element by element (rows chosen to cover every run boundary,
-    every base-only class and the most and least popular adapters), and
-  - for ALL tokens, the projection p[t] = sum_j v[j] y[t][j] against the oracle's projection form.
+run in the launch configuration the benchmark uses.
+
+gate/up prefill and the many-tenant down_proj are compared with the oracle on EVERY element (the
+oracle needs seconds to a minute for them).  The projection set is 224 sites: there every row of
+the first 128-token tile (the 64 decode tokens and the first tokens of the first long run) plus the
+boundary rows of the long runs are compared element by element on the sampled sites.  The
+projection p[t] = sum_j v[j] y[t][j] over all tokens stays as an extra check, not the carrier.
 """
 import numpy as np
 import pytest
@@ -53,8 +55,7 @@ def test_gate_up_prefill_full_size():
     w = wl.gate_up_prefill()
     assert (w.T, w.h_in, w.h_out) == (4096, 4096, 14336)
     y = run_gpu(w)
-    rows = boundary_rows(w.ids, 16, 3)
-    assert_parity(y[rows], oracle_of(w, rows), "gate_up_prefill sampled rows")
+    assert_parity(y, oracle_of(w), "gate_up_prefill, all 4096 x 14336 elements")
     projection_check(w, y, 3)
 
 
@@ -62,15 +63,7 @@ def test_down_proj_many_tenant_full_size():
     w = wl.down_proj_many_tenant(only_used=False)       # all 1000 slots resident (2.36 GB)
     assert (w.T, w.h_in, w.h_out, len(w.adapters)) == (256, 14336, 4096, 1000)
     y = run_gpu(w)
-    # rows: every base-only token class, the most popular adapter's tokens, singletons, random
-    vals, counts = np.unique(w.ids[w.ids >= 0], return_counts=True)
-    rows = set(np.where(w.ids == -1)[0][:4].tolist())
-    rows.update(np.where(w.ids == vals[np.argmax(counts)])[0][:4].tolist())
-    for a in vals[counts == 1][:6]:
-        rows.update(np.where(w.ids == a)[0].tolist())
-    rows.update(boundary_rows(w.ids, 8, 4).tolist()[:24])
-    rows = np.array(sorted(rows))
-    assert_parity(y[rows], oracle_of(w, rows), "down_proj sampled rows")
+    assert_parity(y, oracle_of(w), "down_proj many-tenant, all 256 x 4096 elements")
     projection_check(w, y, 4)
 
 
@@ -85,8 +78,10 @@ def test_full_projection_set_sampled_sites():
     import torch
     batch = wl.full_set_batch()
     assert batch.ids.shape[0] == 2112
+    # the whole first token tile (64 decode tokens + the head of the first run), run boundaries, a
+    # few random rows
     rows = boundary_rows(batch.ids, 4, 5)
-    rows = np.array(sorted(set(rows.tolist()[:10] + [63, 64, 1087, 1088, 2111])))
+    rows = np.array(sorted(set(range(128)) | set(rows.tolist()[:10]) | {1087, 1088, 2111}))
     ids_dev = torch.from_numpy(batch.ids).cuda()
     plan = B.edgelora_plan_create(2112, batch.n_slots)
     xs = {4096: to_dev_bf16(batch.x4096), 14336: to_dev_bf16(batch.x14336)}

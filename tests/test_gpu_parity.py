@@ -363,7 +363,7 @@ def test_profiling_option_reports_every_kernel():
         t = B.edgelora_pool_kernel_times(pool.handle)
         assert t["plan"]["launches"] == 1 and t["shrink_bgmv"]["launches"] == 1
         assert t["shrink_sgmv"]["launches"] == 1 and t["base_gemm"]["launches"] == 1
-        assert t["decode_combine"]["launches"] == 0 and t["base_gemm"]["ms"] > 0
+        assert t["base_gemm"]["ms"] > 0
         info = B.edgelora_pool_last_launch(pool.handle)
         assert info["launches"] == 4 and info["regime"] == "prefill"
     finally:

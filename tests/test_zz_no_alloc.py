@@ -14,6 +14,7 @@ through every other test.
 import numpy as np
 import pytest
 
+import oracle
 from paper_2507_01438_b200 import binding as B
 
 pytestmark = pytest.mark.gpu
@@ -66,6 +67,49 @@ def test_static_plan_matches_allocating_plan_twice_in_a_row():
             assert np.array_equal(want[k], got[k]), k
         assert info[3] == 0
         assert bool(info[2] & B.STATUS_BAD_ADAPTER_ID) == bad
+        check_against_oracle(got, ids, 97)
+
+
+def check_against_oracle(got, ids, n_slots):
+    """The plan as the paper's grouping defines it (Section 3.4), from the CPU oracle."""
+    valid = np.where((ids < -1) | (ids >= n_slots), -1, ids).astype(np.int32)
+    seg_start, seg_adapter = oracle.segments(valid)
+    perm, group_start, group_adapter = oracle.groups(valid, n_slots)
+    assert np.array_equal(got["ids_valid"], valid)
+    assert np.array_equal(got["seg_start"], seg_start) and np.array_equal(got["seg_adapter"], seg_adapter)
+    assert np.array_equal(got["perm"], perm)
+    assert np.array_equal(got["group_start"], group_start) and np.array_equal(got["group_adapter"], group_adapter)
+
+
+def test_static_plan_at_its_size_limit():
+    # T = the limit, once with alternating ids (as many runs as tokens: every fixed array is full)
+    # and once as a single run; the second call must not allocate device memory.
+    import torch
+    T = B.PLAN_STATIC_MAX_TOKENS
+    alternating = (np.arange(T) % 2).astype(np.int32) * 5
+    one_run = np.full(T, 3, dtype=np.int32)
+    want, got, info = build_both(alternating, 8)
+    assert info[1] == T and info[0] == 2
+    for k in KEYS:
+        assert np.array_equal(want[k], got[k]), k
+    check_against_oracle(got, alternating, 8)
+
+    ids = torch.from_numpy(one_run).cuda()
+    out = {k: torch.full((T + 1,), -7, dtype=torch.int32, device="cuda") for k in KEYS}
+    info_t = torch.full((4,), -7, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    rc = B.edgelora_plan_build_static(ids, 8, out["ids_valid"], out["perm"], out["group_start"],
+                                      out["group_adapter"], out["seg_start"], out["seg_adapter"], info_t)
+    assert rc == B.OK
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before, "the non-allocating entry point took device memory"
+    info = info_t.cpu().numpy()
+    assert info.tolist() == [1, 1, 0, 0]
+    got = {"ids_valid": out["ids_valid"][:T], "perm": out["perm"][:T], "group_start": out["group_start"][:2],
+           "group_adapter": out["group_adapter"][:1], "seg_start": out["seg_start"][:2],
+           "seg_adapter": out["seg_adapter"][:1]}
+    check_against_oracle({k: v.cpu().numpy() for k, v in got.items()}, one_run, 8)
 
 
 def test_static_plan_rejects_oversize_and_handles_empty():
