@@ -86,6 +86,11 @@ typedef struct {
                                     call before it (independent sites / batches)                  */
 #define EDGELORA_OPT_DECODE_SPLITS 4 /* tuning: K splits per W row tile in decode, 0 = automatic  */
 #define EDGELORA_OPT_SHRINK_ITEMS 5  /* tuning: work items the decode shrink aims for, 0 = auto   */
+#define EDGELORA_OPT_GATHER_SPLITS 7 /* tuning: K splits of the tensor-core gather shrink in decode, 0 = chosen
+                                        on the device from the number of adapters the batch touches  */
+#define EDGELORA_OPT_GATHER_MIN_T 8  /* tuning: decode batches above this many tokens (default 64) use the
+                                        routing kernel + tensor-core gather shrink; smaller ones the
+                                        single shrink kernel with the routing inside                 */
 #define EDGELORA_OPT_WAIT_CYCLES 6   /* limit of every bounded in-kernel wait of the layer, in units
                                         of 1024 SM clock cycles; 0 = default (about two seconds).
                                         A wait that runs out raises EDGELORA_STATUS_TIMEOUT           */
@@ -184,6 +189,35 @@ int edgelora_pool_plan(edgelora_pool_t *pool, edgelora_plan_t **plan_out);
  * edgelora_pool_sync_status. */
 int edgelora_plan_sync_status(edgelora_plan_t *plan, void *stream, uint32_t *bits_out);
 
+/* ---- A set of linear sites over one batch (Section 3.4: every LoRA-augmented layer of the model
+ * sees the same mixed batch; Section 4.3: the id -> sample mapping is worked out once).  Site i is
+ * (pools[i], W_dev[i]) and reads input number input_of_site[i] (sites with the same input width
+ * may share an input, e.g. q/k/v/o/gate/up of a decoder layer); all pools have the same n_slots
+ * and max_tokens >= the set's.  A run builds ONE routing plan from the ids and evaluates the sites
+ * in order; the sites are independent given their inputs, so in batches above 256 tokens the
+ * shrink of site i + 1 is issued with the kernels of site i and only the first site's shrink stands
+ * alone.  The set borrows the pools and W (the caller keeps them alive) and owns its plan and the
+ * device mirrors of the host-buffer call.  One thread at a time per set; runs of one set (and of
+ * its pools) must not overlap on the GPU. */
+typedef struct edgelora_siteset edgelora_siteset_t;
+int edgelora_siteset_create(int32_t n_sites, edgelora_pool_t *const *pools, const void *const *W_dev,
+                            const int32_t *input_of_site, int32_t n_inputs, int32_t max_tokens,
+                            edgelora_siteset_t **set_out);
+int edgelora_siteset_destroy(edgelora_siteset_t *set);
+/* x_dev [n_inputs] device pointers ([T][width of that input] bf16), adapter_id_dev [T],
+ * y_dev [n_sites] device pointers ([T][h_out of that site]); asynchronous on `stream`. */
+int edgelora_siteset_run(edgelora_siteset_t *set, const void *const *x_dev, const int32_t *adapter_id_dev,
+                         int32_t T, void *const *y_dev, void *stream);
+/* The same with HOST buffers (page-locked for full copy speed): copies the inputs and the ids to
+ * the device, runs the set, copies back y of every site whose y_host entry is not NULL (the others
+ * stay on the device and are overwritten by the next site of the same width) and synchronises
+ * `stream` before returning.  Allocates its device mirrors on first use. */
+int edgelora_siteset_run_host(edgelora_siteset_t *set, const uint16_t *const *x_host,
+                              const int32_t *adapter_id_host, int32_t T, uint16_t *const *y_host,
+                              void *stream);
+/* The set's plan object (for edgelora_plan_export / edgelora_plan_sync_status). */
+int edgelora_siteset_plan(edgelora_siteset_t *set, edgelora_plan_t **plan_out);
+
 /* No counterpart in the paper: a routing-plan builder for callers that cannot allocate.
  *
  * Some hosts of this library may not call cudaMalloc on the path where they need a plan: a
@@ -235,8 +269,8 @@ int edgelora_pool_last_launch(edgelora_pool_t *pool, int64_t info_out[8]);
 
 /* With EDGELORA_OPT_PROFILE on: accumulated device time per kernel since the last reset,
  * from CUDA events on the launching stream (synchronises them).  ms_out / launches_out:
- * [0] plan, [1] shrink (gather-by-token), [2] shrink (segment), [3] base product
- * (expand and combine included), [4] unused.  reset != 0 clears the accumulators afterwards. */
+ * [0] plan, [1] shrink of small decode batches (routing inside), [2] shrink on the tensor cores
+ * (segment and gather tiles), [3] base product (expand and combine included), [4] unused.  reset != 0 clears the accumulators afterwards. */
 int edgelora_pool_kernel_times(edgelora_pool_t *pool, double ms_out[5], int64_t launches_out[5],
                                int32_t reset);
 

@@ -19,7 +19,8 @@ ERR_INVALID_ARG, ERR_BAD_SLOT, ERR_RANK_TOO_LARGE, ERR_ARENA_TOO_SMALL = -1, -2,
 ERR_CUDA, ERR_BAD_ADAPTER_ID, ERR_SLOT_EMPTY, ERR_TIMEOUT, ERR_TOO_MANY_TOKENS = -5, -6, -7, -8, -9
 STATUS_BAD_ADAPTER_ID, STATUS_SLOT_EMPTY, STATUS_TIMEOUT = 0x1, 0x2, 0x4
 OPT_REGIME, OPT_PROFILE, OPT_PDL, OPT_DECODE_SPLITS, OPT_SHRINK_ITEMS, OPT_WAIT_CYCLES = 1, 2, 3, 4, 5, 6
-KERNEL_NAMES = ("plan", "shrink_bgmv", "shrink_sgmv", "base_gemm")
+OPT_GATHER_SPLITS, OPT_GATHER_MIN_T = 7, 8
+KERNEL_NAMES = ("plan", "shrink_small_decode", "shrink_tiles", "base_gemm")
 
 EXPORTS = (
     "edgelora_pool_bytes_required", "edgelora_pool_create", "edgelora_pool_load_slot",
@@ -32,6 +33,8 @@ EXPORTS = (
     "edgelora_pool_host_sync", "edgelora_cache_create", "edgelora_cache_destroy", "edgelora_cache_acquire",
     "edgelora_cache_release", "edgelora_cache_lookup", "edgelora_cache_stats", "edgelora_cache_select",
     "edgelora_router_scores", "edgelora_plan_sync_status", "edgelora_pool_selftest_wait",
+    "edgelora_siteset_create", "edgelora_siteset_destroy", "edgelora_siteset_run",
+    "edgelora_siteset_run_host", "edgelora_siteset_plan",
 )
 
 
@@ -86,6 +89,11 @@ def lib() -> ctypes.CDLL:
     L.edgelora_lora_linear_planned.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     L.edgelora_plan_build_static.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.edgelora_pool_plan.argtypes = [vp, cp(vp)]
+    L.edgelora_siteset_create.argtypes = [i32, cp(vp), cp(vp), cp(i32), i32, i32, cp(vp)]
+    L.edgelora_siteset_destroy.argtypes = [vp]
+    L.edgelora_siteset_run.argtypes = [vp, cp(vp), vp, i32, cp(vp), vp]
+    L.edgelora_siteset_run_host.argtypes = [vp, cp(vp), vp, i32, cp(vp), vp]
+    L.edgelora_siteset_plan.argtypes = [vp, cp(vp)]
     L.edgelora_plan_sync_status.argtypes = [vp, vp, cp(ctypes.c_uint32)]
     L.edgelora_pool_selftest_wait.argtypes = [vp, vp]
     L.edgelora_pool_sync_status.argtypes = [vp, cp(ctypes.c_uint32)]
@@ -242,6 +250,49 @@ def edgelora_plan_build_static(adapter_id, n_slots: int, ids_valid, perm, group_
                                             ptr(group_start), ptr(group_adapter), ptr(seg_start),
                                             ptr(seg_adapter), _dev_ptr(info, 4, "info"),
                                             _stream_ptr(stream))
+
+
+def _ptr_array(ptrs):
+    return (ctypes.c_void_p * len(ptrs))(*[ctypes.c_void_p(p) if p else None for p in ptrs])
+
+
+def edgelora_siteset_create(pools, Ws, input_of_site, n_inputs: int, max_tokens: int) -> int:
+    """pools: pool handles, Ws: bf16 CUDA tensors [h_out, h_in] (kept alive by the caller)."""
+    n = len(pools)
+    idx = (ctypes.c_int32 * n)(*[int(i) for i in input_of_site])
+    out = ctypes.c_void_p()
+    _check(lib().edgelora_siteset_create(n, _ptr_array(list(pools)), _ptr_array([_dev_ptr(W, 2, "W") for W in Ws]),
+                                         idx, n_inputs, max_tokens, ctypes.byref(out)), "siteset_create")
+    return out.value
+
+
+def edgelora_siteset_destroy(s) -> None:
+    _check(lib().edgelora_siteset_destroy(s), "siteset_destroy")
+
+
+def edgelora_siteset_run(s, xs, adapter_id, ys, stream=None) -> None:
+    """xs: one bf16 CUDA tensor per input, ys: one per site, adapter_id: int32 CUDA tensor [T]."""
+    T = int(adapter_id.shape[0])
+    _check(lib().edgelora_siteset_run(s, _ptr_array([_dev_ptr(x, 2, "x") for x in xs]),
+                                      _dev_ptr(adapter_id, 4, "ids") if T else None, T,
+                                      _ptr_array([_dev_ptr(y, 2, "y") for y in ys]), _stream_ptr(stream)),
+           "siteset_run")
+
+
+def edgelora_siteset_run_host(s, xs_host, ids_host, ys_host, stream=None) -> None:
+    """Host buffers (pinned torch CPU tensors or numpy arrays); ys_host entries may be None."""
+    def ptr(a):
+        return None if a is None else (a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data)
+    T = int(ids_host.shape[0])
+    _check(lib().edgelora_siteset_run_host(s, _ptr_array([ptr(x) for x in xs_host]), ptr(ids_host), T,
+                                           _ptr_array([ptr(y) for y in ys_host]), _stream_ptr(stream)),
+           "siteset_run_host")
+
+
+def edgelora_siteset_plan(s) -> int:
+    out = ctypes.c_void_p()
+    _check(lib().edgelora_siteset_plan(s, ctypes.byref(out)), "siteset_plan")
+    return out.value
 
 
 def edgelora_pool_plan(pool) -> int:

@@ -39,18 +39,53 @@ struct TileCoord {
   int32_t split;
   int32_t nrows;   // sgmv: tokens of the tile that belong to the run
   int32_t mtile;   // prefill: token tile; decode: W row tile
+  // gather tiles of a shrink job: R = the A blocks of `ng` consecutive LoRA groups stacked (R_pad rows
+  // each), C = the rows of x of those groups' tokens, fetched one by one
+  int32_t kind;    // 0 regular, 1 gather
+  int32_t g0, ng;  // first group (index into the plan's group arrays) and number of groups
+  int32_t tok0, ntok;  // the groups' tokens: perm_short[tok0 .. tok0 + ntok)
+  int32_t gtile;   // index of the gather tile (its arrival counter)
 };
+
+// K splits of the gather tiles when the host leaves the choice to the device (it does not know
+// how many adapters a batch touches): the split count up to 8 whose (tile, split) items fill whole
+// waves of the grid best, each split keeping at least four K blocks.
+__device__ __forceinline__ int32_t gather_splits(const GemmParams &p, int32_t n_gt, int32_t grid) {
+  if (p.splits > 0) return p.splits;
+  int32_t best = 1;
+  float best_eff = 0.f;
+  for (int32_t sp = 1; sp <= 8 && p.kb_total / sp >= 4; ++sp) {
+    if ((sp - 1) * ((p.kb_total + sp - 1) / sp) >= p.kb_total) continue;  // every split needs a K block
+    const int32_t items = n_gt * sp, waves = (items + grid - 1) / grid;
+    const float eff = waves > 0 ? static_cast<float>(items) / static_cast<float>(waves * grid) : 0.f;
+    if (eff > best_eff + 0.02f) {
+      best_eff = eff;
+      best = sp;
+    }
+  }
+  return best;
+}
+// LoRA groups (ids >= 0) of the batch per gather tile, and the number of gather tiles.
+__device__ __forceinline__ int32_t gather_tiles(const GemmParams &p) {
+  if (!p.gather) return 0;
+  const int32_t per = kTileM / p.R_pad;
+  return (p.counts[4] + per - 1) / per;
+}
 
 __device__ __forceinline__ int32_t total_tiles(const GemmParams &p) {
   if (p.mode == kModePrefill) return p.n_mtiles * p.n_ntiles;
   if (p.mode == kModeDecode) return p.n_mtiles * p.splits;
-  return p.counts[2] * p.splits;
+  const int32_t n_gt = gather_tiles(p);
+  return p.counts[2] * max(p.splits, 1) + n_gt * gather_splits(p, n_gt, gridDim.x);
 }
 
 __device__ __forceinline__ TileCoord tile_coord(const GemmParams &p, int32_t tile) {
   TileCoord c;
   c.slot = 0;
   c.nrows = kTileM;
+  c.kind = 0;
+  c.g0 = c.ng = c.tok0 = c.ntok = c.gtile = 0;
+  int32_t kb_per = p.kb_per;
   if (p.mode == kModePrefill) {
     const int m = tile % p.n_mtiles, n = tile / p.n_mtiles;
     c.row_r = m * kTileM;
@@ -65,17 +100,40 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams &p, int32_t til
     c.mtile = m;
   } else {
     const int n_t = p.counts[2];
-    const int st = tile % n_t;
-    c.split = tile / n_t;
-    c.row_r = p.sgmv_tiles[4 * st + 0];
-    c.nrows = p.sgmv_tiles[4 * st + 1];
-    c.slot = p.sgmv_tiles[4 * st + 2];
+    const int n_seg_items = n_t * max(p.splits, 1);
     c.row_c = 0;
     c.mtile = 0;
+    if (tile < n_seg_items) {
+      const int st = tile % n_t;
+      c.split = tile / n_t;
+      c.row_r = p.sgmv_tiles[4 * st + 0];
+      c.nrows = p.sgmv_tiles[4 * st + 1];
+      c.slot = p.sgmv_tiles[4 * st + 2];
+    } else {
+      const int n_gt = gather_tiles(p);
+      const int gsp = gather_splits(p, n_gt, gridDim.x);
+      const int g = tile - n_seg_items;
+      const int per = kTileM / p.R_pad;
+      const int n_groups = p.counts[0], n_lg = p.counts[4];
+      c.kind = 1;
+      c.gtile = g % n_gt;
+      c.split = g / n_gt;
+      c.g0 = (n_groups - n_lg) + c.gtile * per;  // the group of id -1, when there is one, comes first
+      c.ng = min(per, n_groups - c.g0);
+      c.tok0 = p.gs_short[c.g0];
+      c.ntok = p.gs_short[c.g0 + c.ng] - c.tok0;
+      c.row_r = 0;
+      kb_per = (p.kb_total + gsp - 1) / gsp;
+    }
   }
-  c.kb0 = c.split * p.kb_per;
-  c.kb1 = min(p.kb_total, c.kb0 + p.kb_per);
+  c.kb0 = c.split * kb_per;
+  c.kb1 = min(p.kb_total, c.kb0 + kb_per);
+  if (c.kb1 < c.kb0) c.kb1 = c.kb0;
   return c;
+}
+// Passes over a tile: a gather tile with more tokens than one pass holds takes several.
+__device__ __forceinline__ int32_t tile_passes(const GemmParams &p, const TileCoord &c) {
+  return c.kind == 1 ? (c.ntok + p.gN - 1) / p.gN : 1;
 }
 
 // decode: first W row of the tile this CTA works on
@@ -183,13 +241,21 @@ __device__ __forceinline__ void load_z_packed(const GemmParams &p, int32_t t, in
 template <int kMinBlocks>
 __global__ void __launch_bounds__(kGemmThreads, kMinBlocks)
 lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_constant__ CUtensorMap tmap_c,
-                 const __grid_constant__ CUtensorMap tmap_b, const GemmParams p) {
+                 const __grid_constant__ CUtensorMap tmap_b, const GemmParams p,
+                 const __grid_constant__ CUtensorMap tmap_r2, const __grid_constant__ CUtensorMap tmap_c2,
+                 const __grid_constant__ CUtensorMap tmap_g2, const GemmParams p2) {
   extern __shared__ uint8_t smem_raw[];
   // tiles need 1024-byte alignment for the 128-byte swizzle
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t r_bytes = kTileM * kBlockK * 2;              // 16 KB
   const uint32_t c_bytes = static_cast<uint32_t>(p.BN) * kBlockK * 2;
-  const uint32_t stage_bytes = r_bytes + c_bytes;
+  // the ring is laid out for the first job: its C region holds ring_rows rows
+  const uint32_t stage_bytes = r_bytes + static_cast<uint32_t>(p.ring_rows) * kBlockK * 2;
+  // Second job (optional): the segment shrink of ANOTHER linear site as extra tiles of this
+  // persistent grid, after the first job's tiles.  Its tile list comes from a plan on the device, so
+  // the host passes an upper bound (p2.n_mtiles) and every role stops at the true count, which it
+  // reads after the dependency wait.  Its N tile is never wider than the first job's.
+  const bool has2 = p2.mode == kModeSgmv;
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + static_cast<size_t>(p.stages) * stage_bytes);
   uint64_t *full_bar = bars;                      // [stages]  TMA -> MMA
   uint64_t *empty_bar = bars + kMaxStages;        // [stages]  MMA -> TMA
@@ -208,6 +274,8 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   int32_t *s_vid = reinterpret_cast<int32_t *>(extra + 1152);               // [256] validated ids
   uint8_t *s_head = extra + 2176;                                           // [256]
   uint32_t *s_key = reinterpret_cast<uint32_t *>(extra + 2432);             // [256] sort keys
+  volatile int32_t *s_last = reinterpret_cast<volatile int32_t *>(extra + 80);  // gather tiles: last arriver
+  uint64_t *ep_bar = reinterpret_cast<uint64_t *>(extra + 88);              // rendezvous of the epilogue warps
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wl = p.wait_cycles;  // limit of every bounded wait below
@@ -220,6 +288,12 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     ptx::prefetch_tensormap(&tmap_r);
     ptx::prefetch_tensormap(&tmap_c);
     if (has_lora) ptx::prefetch_tensormap(&tmap_b);
+    if (has2) {
+      ptx::prefetch_tensormap(&tmap_r2);
+      ptx::prefetch_tensormap(&tmap_c2);
+      if (p2.gather) ptx::prefetch_tensormap(&tmap_g2);
+    }
+    if (p.mode == kModeSgmv && p.gather) ptx::prefetch_tensormap(&tmap_b);
     for (int s = 0; s < p.stages; ++s) {
       ptx::mbar_init(&full_bar[s], 1);
       ptx::mbar_init(&empty_bar[s], 1);
@@ -231,6 +305,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       ptx::mbar_init(&tempty_bar[i], 4);  // one arrival per epilogue warp
     }
     ptx::mbar_init(lg_bar, 1);
+    ptx::mbar_init(ep_bar, 4);  // one arrival per epilogue warp
     *abort_flag = 0;
     *s_nlg = 0;
     ptx::fence_barrier_init();
@@ -248,37 +323,110 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   ptx::pdl_launch_dependents();
 
   if (p.mode == kModeSgmv) ptx::pdl_wait_prior_grids();  // tile list comes from the plan kernel
-  const int32_t n_tiles = total_tiles(p);
+  const int32_t n_tiles0 = total_tiles(p);
+  const int32_t n_tiles = n_tiles0 + (has2 ? p2.n_mtiles : 0);
   const uint32_t nstages = static_cast<uint32_t>(p.stages);
+  // Every role walks the same tile sequence: tiles below n_tiles0 belong to the first job; for the
+  // others the true count of the second job is read once (after griddepcontrol.wait: the plan may
+  // come from a kernel this one was allowed to start under) and the walk ends at it.
+  int32_t n2_true = -1;
+  auto second_job_tile = [&](int32_t tile) -> int32_t {  // local tile index, or -1 = stop
+    if (n2_true < 0) {
+      ptx::pdl_wait_prior_grids();
+      n2_true = total_tiles(p2);
+    }
+    const int32_t local = tile - n_tiles0;
+    return local < n2_true ? local : -1;
+  };
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // The whole warp walks the loop (state stays uniform); lane 0 waits and issues the tile loads,
+    // and for gather tiles every lane issues its share of the one-row loads.
+    {
       uint32_t stage = 0, phase = 0;
       bool ok = true, waited = p.mode == kModeSgmv;
+      auto wait_empty = [&]() {  // lane 0 polls, the warp learns the result
+        int got = 1;
+        if (lane == 0) got = (ptx::mbar_wait(&empty_bar[stage], phase ^ 1, wl) && !*abort_flag) ? 1 : 0;
+        return __shfl_sync(0xffffffffu, got, 0) != 0;
+      };
+      auto advance = [&]() {
+        if (++stage == nstages) {
+          stage = 0;
+          phase ^= 1;
+        }
+      };
       for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
-        const TileCoord tc = tile_coord(p, tile);
+        const bool second = tile >= n_tiles0;
+        int32_t local = tile;
+        if (second && (local = second_job_tile(tile)) < 0) break;
+        const GemmParams &jp = second ? p2 : p;
+        const CUtensorMap *mr = second ? &tmap_r2 : &tmap_r, *mc = second ? &tmap_c2 : &tmap_c;
+        const TileCoord tc = tile_coord(jp, local);
+        if (tc.kind == 1) {
+          // gather tile: lane i fetches the A block of the tile's i-th group (rows [i R_pad, ...) of
+          // the R tile), lane l the x rows of tokens l, l + 32, ... of the pass
+          const CUtensorMap *mg = second ? &tmap_g2 : &tmap_b;
+          int32_t my_slot = -1;
+          if (lane < tc.ng) {
+            const int32_t a = jp.group_adapter[tc.g0 + lane];
+            if (a >= 0 && jp.slots[a].rank > 0) my_slot = a;
+          }
+          const uint32_t n_live = __popc(__ballot_sync(0xffffffffu, my_slot >= 0));
+          const uint32_t a_bytes = static_cast<uint32_t>(jp.R_pad) * kBlockK * 2;
+          for (int32_t t0 = 0; ok && t0 < tc.ntok; t0 += jp.gN) {
+            const int32_t n = min(jp.gN, tc.ntok - t0);
+            int32_t tok[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const int c = q * 32 + lane;
+              tok[q] = c < n ? jp.perm_short[tc.tok0 + t0 + c] : -1;
+            }
+            const uint32_t tx = n_live * a_bytes + static_cast<uint32_t>(n) * kBlockK * 2;
+            for (int32_t kb = tc.kb0; kb < tc.kb1; ++kb) {
+              if (!wait_empty()) {
+                ok = false;
+                break;
+              }
+              uint8_t *sr = smem + static_cast<size_t>(stage) * stage_bytes;
+              if (lane == 0) ptx::mbar_arrive_expect_tx(&full_bar[stage], tx);
+              __syncwarp();
+              if (my_slot >= 0)
+                ptx::tma_load_3d(sr + static_cast<size_t>(lane) * a_bytes, mc, &full_bar[stage], kb * kBlockK, 0, my_slot);
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                if (tok[q] >= 0)
+                  ptx::tma_load_2d(sr + r_bytes + static_cast<size_t>(q * 32 + lane) * (kBlockK * 2), mg,
+                                   &full_bar[stage], kb * kBlockK, tok[q]);
+              advance();
+            }
+          }
+          continue;
+        }
+        const uint32_t tx_bytes = r_bytes + static_cast<uint32_t>(jp.BN) * kBlockK * 2;
         for (int32_t kb = tc.kb0; kb < tc.kb1; ++kb) {
-          if (!ptx::mbar_wait(&empty_bar[stage], phase ^ 1, wl) || *abort_flag) {
+          if (!wait_empty()) {
             ok = false;
             break;
           }
-          uint8_t *sr = smem + static_cast<size_t>(stage) * stage_bytes;
-          ptx::mbar_arrive_expect_tx(&full_bar[stage], stage_bytes);
-          ptx::tma_load_2d(sr, &tmap_r, &full_bar[stage], kb * kBlockK, tc.row_r);
-          if (p.mode == kModeSgmv)
-            ptx::tma_load_3d(sr + r_bytes, &tmap_c, &full_bar[stage], kb * kBlockK, 0, tc.slot);
-          else
-            ptx::tma_load_2d(sr + r_bytes, &tmap_c, &full_bar[stage], kb * kBlockK, tc.row_c);
-          if (++stage == nstages) {
-            stage = 0;
-            phase ^= 1;
+          if (lane == 0) {
+            uint8_t *sr = smem + static_cast<size_t>(stage) * stage_bytes;
+            ptx::mbar_arrive_expect_tx(&full_bar[stage], tx_bytes);
+            ptx::tma_load_2d(sr, mr, &full_bar[stage], kb * kBlockK, tc.row_r);
+            if (jp.mode == kModeSgmv)
+              ptx::tma_load_3d(sr + r_bytes, mc, &full_bar[stage], kb * kBlockK, 0, tc.slot);
+            else
+              ptx::tma_load_2d(sr + r_bytes, mc, &full_bar[stage], kb * kBlockK, tc.row_c);
           }
+          advance();
         }
-        if (!ok || !has_lora) continue;
+        if (!ok || !has_lora || second) continue;
         if (!waited) {
           if (p.mode == kModeDecode) {  // the builder warps derive the adapter list from the ids
-            if (!ptx::mbar_wait(lg_bar, 0, wl)) {
+            int got = 1;
+            if (lane == 0) got = ptx::mbar_wait(lg_bar, 0, wl) ? 1 : 0;
+            if (!__shfl_sync(0xffffffffu, got, 0)) {
               ok = false;
               break;
             }
@@ -291,28 +439,27 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
           const int32_t a = ll.list[e];
           if (p.mode != kModeDecode && p.slots[a].rank <= 0) continue;
-          if (!ptx::mbar_wait(&empty_bar[stage], phase ^ 1, wl) || *abort_flag) {
+          if (!wait_empty()) {
             ok = false;
             break;
           }
-          // The stage is free: let the builder write its half (it follows this warp, never the
-          // stage barriers directly, so it cannot run ahead of the ring).
-          ptx::mbar_arrive(&zgo_bar[stage]);
-          uint8_t *sr = smem + static_cast<size_t>(stage) * stage_bytes;
-          if (p.mode == kModePrefill) {  // C operand: rows [row_c, row_c + BN) of B_a
-            ptx::mbar_arrive_expect_tx(&full_bar[stage], c_bytes);
-            ptx::tma_load_3d(sr + r_bytes, &tmap_b, &full_bar[stage], 0, tc.row_c, a);
-          } else {                       // R operand: rows [row_r, row_r + 128) of B_a
-            ptx::mbar_arrive_expect_tx(&full_bar[stage], r_bytes);
-            ptx::tma_load_3d(sr, &tmap_b, &full_bar[stage], 0, tc.row_r, a);
+          if (lane == 0) {
+            // The stage is free: let the builder write its half (it follows this warp, never the
+            // stage barriers directly, so it cannot run ahead of the ring).
+            ptx::mbar_arrive(&zgo_bar[stage]);
+            uint8_t *sr = smem + static_cast<size_t>(stage) * stage_bytes;
+            if (p.mode == kModePrefill) {  // C operand: rows [row_c, row_c + BN) of B_a
+              ptx::mbar_arrive_expect_tx(&full_bar[stage], c_bytes);
+              ptx::tma_load_3d(sr + r_bytes, &tmap_b, &full_bar[stage], 0, tc.row_c, a);
+            } else {                       // R operand: rows [row_r, row_r + 128) of B_a
+              ptx::mbar_arrive_expect_tx(&full_bar[stage], r_bytes);
+              ptx::tma_load_3d(sr, &tmap_b, &full_bar[stage], 0, tc.row_r, a);
+            }
           }
-          if (++stage == nstages) {
-            stage = 0;
-            phase ^= 1;
-          }
+          advance();
         }
       }
-      if (!ok) {
+      if (!ok && lane == 0) {
         *abort_flag = 1;
         atomicOr(p.status, EDGELORA_STATUS_TIMEOUT);
       }
@@ -320,43 +467,61 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = ptx::umma_idesc_bf16(kTileM, static_cast<uint32_t>(p.BN));
       const int lora_ksteps = p.R_pad / kUmmaK;
       uint32_t stage = 0, phase = 0, zphase = 0;  // zphase: one parity bit per stage
       bool ok = true, waited = p.mode == kModeSgmv;
       int32_t it = 0;
-      for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++it) {
-        const TileCoord tc = tile_coord(p, tile);
-        const uint32_t acc = (p.n_acc == 2) ? (it & 1) : 0;
-        const uint32_t use = (p.n_acc == 2) ? (it >> 1) : it;
-        if (!ptx::mbar_wait(&tempty_bar[acc], (use & 1) ^ 1, wl) || *abort_flag) {
-          ok = false;
-          break;
-        }
-        ptx::tc_fence_after_sync();
-        const uint32_t tmem_d = tmem_base + acc * static_cast<uint32_t>(p.BN);
-        for (int32_t kb = tc.kb0; kb < tc.kb1; ++kb) {
-          if (!ptx::mbar_wait(&full_bar[stage], phase, wl) || *abort_flag) {
+      for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+        const bool second = tile >= n_tiles0;
+        int32_t local = tile;
+        if (second && (local = second_job_tile(tile)) < 0) break;
+        const GemmParams &jp = second ? p2 : p;
+        const TileCoord tc = tile_coord(jp, local);
+        const int32_t n_pass = tile_passes(jp, tc);
+        uint32_t acc = 0, tmem_d = tmem_base;
+        for (int32_t pass = 0; ok && pass < n_pass; ++pass, ++it) {
+          // UMMA N: the job's N tile, or for a gather pass its token count rounded up to 16
+          const uint32_t n_cols = tc.kind == 1
+                                      ? static_cast<uint32_t>((min(jp.gN, tc.ntok - pass * jp.gN) + 15) & ~15)
+                                      : static_cast<uint32_t>(jp.BN);
+          const uint32_t idesc = ptx::umma_idesc_bf16(kTileM, n_cols);
+          acc = (p.n_acc == 2) ? (it & 1) : 0;
+          const uint32_t use = (p.n_acc == 2) ? (it >> 1) : it;
+          if (!ptx::mbar_wait(&tempty_bar[acc], (use & 1) ^ 1, wl) || *abort_flag) {
             ok = false;
             break;
           }
           ptx::tc_fence_after_sync();
-          const uint32_t sr = ptx::smem_u32(smem + static_cast<size_t>(stage) * stage_bytes);
-          const uint64_t da = ptx::umma_desc_k128(sr);
-          const uint64_t db = ptx::umma_desc_k128(sr + r_bytes);
+          tmem_d = tmem_base + acc * static_cast<uint32_t>(p.acc_cols);
+          for (int32_t kb = tc.kb0; kb < tc.kb1; ++kb) {
+            if (!ptx::mbar_wait(&full_bar[stage], phase, wl) || *abort_flag) {
+              ok = false;
+              break;
+            }
+            ptx::tc_fence_after_sync();
+            const uint32_t sr = ptx::smem_u32(smem + static_cast<size_t>(stage) * stage_bytes);
+            const uint64_t da = ptx::umma_desc_k128(sr);
+            const uint64_t db = ptx::umma_desc_k128(sr + r_bytes);
 #pragma unroll
-          for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-            // advancing 16 bf16 along K inside the swizzled row = 32 bytes = 2 descriptor units
-            ptx::umma_bf16(tmem_d, da + 2 * k, db + 2 * k, idesc, (kb > tc.kb0 || k > 0) ? 1u : 0u);
+            for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+              // advancing 16 bf16 along K inside the swizzled row = 32 bytes = 2 descriptor units
+              ptx::umma_bf16(tmem_d, da + 2 * k, db + 2 * k, idesc, (kb > tc.kb0 || k > 0) ? 1u : 0u);
+            }
+            ptx::umma_commit(&empty_bar[stage]);  // frees the smem stage once these MMAs are done
+            if (++stage == nstages) {
+              stage = 0;
+              phase ^= 1;
+            }
           }
-          ptx::umma_commit(&empty_bar[stage]);  // frees the smem stage once these MMAs are done
-          if (++stage == nstages) {
-            stage = 0;
-            phase ^= 1;
-          }
+          if (!ok) break;
+          // a gather pass is complete here; other tiles go on with their LoRA K blocks below
+          if (tc.kind == 1) ptx::umma_commit(&tfull_bar[acc]);
         }
         if (!ok) break;
-        if (has_lora) {
+        if (tc.kind == 1) continue;
+        const uint32_t idesc = ptx::umma_idesc_bf16(kTileM, static_cast<uint32_t>(jp.BN));
+        if (!ok) break;
+        if (has_lora && !second) {
           if (!waited) {
             if (p.mode == kModeDecode) {
               if (!ptx::mbar_wait(lg_bar, 0, wl)) {
@@ -438,13 +603,135 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     if (!(clustered && p.expand_in_reduce)) ptx::pdl_wait_prior_grids();
     bool ok = true;
     int32_t it = 0;
-    for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++it) {
-      const TileCoord tc = tile_coord(p, tile);
+    uint32_t ep_phase = 0;
+    for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+      const bool second = tile >= n_tiles0;
+      int32_t local = tile;
+      if (second && (local = second_job_tile(tile)) < 0) break;
+      const GemmParams &jp = second ? p2 : p;
+      const TileCoord tc = tile_coord(jp, local);
+      if (tc.kind == 1) {
+        // ---- gather tile: accumulator row m = (group m / R_pad of the tile, rank row m % R_pad),
+        // column c = token perm_short[tok0 + pass * gN + c].  This thread writes z of its rank row
+        // for the tokens of its group, scaled by s_a, into the partial plane of the tile's K split.
+        const int32_t gi = row_in_tile / jp.R_pad, r = row_in_tile % jp.R_pad;
+        int32_t c_lo = 0, c_hi = 0;  // this row's tokens, as positions inside the tile's token list
+        float scale = 0.f;
+        bool live = false;
+        if (gi < tc.ng) {
+          const int32_t a = jp.group_adapter[tc.g0 + gi];
+          const SlotRow row = jp.slots[a];
+          live = row.rank > 0;
+          scale = row.scale;
+          c_lo = jp.gs_short[tc.g0 + gi] - tc.tok0;
+          c_hi = jp.gs_short[tc.g0 + gi + 1] - tc.tok0;
+          if (!live && r == 0 && tc.split == 0 && c_hi > c_lo) atomicOr(jp.status, EDGELORA_STATUS_SLOT_EMPTY);
+        }
+        const size_t plane = static_cast<size_t>(jp.max_tokens) * jp.R_pad;
+        float *zsplit = jp.zws_out + static_cast<size_t>(tc.split) * plane;
+        const int32_t n_pass = tile_passes(jp, tc);
+        for (int32_t pass = 0; ok && pass < n_pass; ++pass, ++it) {
+          const uint32_t acc = (p.n_acc == 2) ? (it & 1) : 0;
+          const uint32_t use = (p.n_acc == 2) ? (it >> 1) : it;
+          if (!(ptx::mbar_wait(&tfull_bar[acc], use & 1, wl) && !*abort_flag)) {
+            ok = false;
+            *abort_flag = 1;
+            break;
+          }
+          ptx::tc_fence_after_sync();
+          const int32_t t0 = pass * jp.gN, n = min(jp.gN, tc.ntok - t0);
+          int32_t tok[8];  // lane l keeps the tokens of columns l, l + 32, ...
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int c = q * 32 + lane;
+            tok[q] = c < n ? jp.perm_short[tc.tok0 + t0 + c] : 0;
+          }
+          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
+                                 acc * static_cast<uint32_t>(p.acc_cols);
+          const int32_t n16 = (n + 15) & ~15;
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int32_t c0 = q * 32;
+            if (c0 < n16) {  // uniform over the warp
+              float v[32];
+              if (n16 - c0 >= 32) {
+                ptx::tmem_ld_32x32(taddr + c0, v);
+              } else {
+                float h[16];
+                ptx::tmem_ld_32x16(taddr + c0, h);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                  v[i] = h[i];
+                  v[i + 16] = 0.f;
+                }
+              }
+#pragma unroll
+              for (int jj = 0; jj < 32; ++jj) {
+                const int32_t t = __shfl_sync(0xffffffffu, tok[q], jj);
+                const int32_t c = t0 + c0 + jj;  // position inside the tile's token list
+                if (live && c >= c_lo && c < c_hi && c0 + jj < n)
+                  zsplit[static_cast<size_t>(t) * jp.R_pad + r] = scale * v[jj];
+              }
+            }
+          }
+          ptx::tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&tempty_bar[acc]);
+        }
+        if (!ok) break;
+        if (jp.finalize) {
+          // Whichever K split of this tile arrives last adds the splits, in order, into the final
+          // plane (the one the base-product kernel reads); nobody waits for another CTA.  The four
+          // epilogue warps meet on a barrier with a bounded wait, like every wait of this kernel.
+          auto ep_sync = [&]() {
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ep_bar);
+            const bool met = ptx::mbar_wait(ep_bar, ep_phase, wl);
+            ep_phase ^= 1u;
+            __syncwarp();
+            return met;
+          };
+          const int32_t n_gt = gather_tiles(jp);
+          const int32_t gsp = gather_splits(jp, n_gt, gridDim.x);
+          __threadfence();                 // this thread's z stores, before the arrival below
+          if (!ep_sync()) {
+            ok = false;
+            break;
+          }
+          if (threadIdx.x == 64) {
+            const int32_t old = atomicAdd(&jp.tile_counters[tc.gtile], 1);
+            *s_last = (old == gsp - 1) ? 1 : 0;
+            if (old == gsp - 1) jp.tile_counters[tc.gtile] = 0;  // ready for the next launch
+          }
+          if (!ep_sync()) {
+            ok = false;
+            break;
+          }
+          if (*s_last) {
+            __threadfence();
+            if (live) {
+              float *zfinal = jp.zws_out + static_cast<size_t>(kMaxZSplits) * plane;
+              for (int32_t c = c_lo; c < c_hi; ++c) {
+                const size_t off = static_cast<size_t>(jp.perm_short[tc.tok0 + c]) * jp.R_pad + r;
+                float sum = 0.f;
+                for (int32_t sp = 0; sp < gsp; ++sp) sum += __ldcg(jp.zws_out + sp * plane + off);
+                zfinal[off] = sum;
+              }
+            }
+          }
+          if (!ep_sync()) {                // s_last is reused by the next tile
+            ok = false;
+            break;
+          }
+        }
+        continue;
+      }
       const uint32_t acc = (p.n_acc == 2) ? (it & 1) : 0;
       const uint32_t use = (p.n_acc == 2) ? (it >> 1) : it;
+      ++it;
       const int32_t row = tc.row_r + row_in_tile;
       float scale = 0.f;
-      if (p.mode == kModeSgmv) scale = p.slots[tc.slot].scale;
+      if (jp.mode == kModeSgmv) scale = jp.slots[tc.slot].scale;
 
       const bool got = ptx::mbar_wait(&tfull_bar[acc], use & 1, wl) && !*abort_flag;
       if (!got) {
@@ -455,10 +742,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       if (clustered) break;  // the accumulator is read after the cluster barrier below
       ptx::tc_fence_after_sync();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
-                             acc * static_cast<uint32_t>(p.BN);
-      for (int32_t c0 = 0; got && c0 < p.BN; c0 += 32) {
+                             acc * static_cast<uint32_t>(p.acc_cols);  // accumulators are spaced for the first job
+      for (int32_t c0 = 0; got && c0 < jp.BN; c0 += 32) {
         float v[32];
-        if (p.BN - c0 >= 32) {
+        if (jp.BN - c0 >= 32) {
           ptx::tmem_ld_32x32(taddr + c0, v);
         } else {  // sgmv with a rank stride of 16: only 16 columns exist
           float h[16];
@@ -469,14 +756,14 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
             v[i + 16] = 0.f;
           }
         }
-        if (p.mode == kModePrefill) {
+        if (jp.mode == kModePrefill) {
           // row = token, columns = output features row_c + c0 + [0, 32)
-          if (row < p.T) {
-            uint16_t *yrow = p.y + static_cast<size_t>(row) * p.h_out;
+          if (row < jp.T) {
+            uint16_t *yrow = jp.y + static_cast<size_t>(row) * jp.h_out;
 #pragma unroll
             for (int q = 0; q < 32; q += 8) {
               const int j = tc.row_c + c0 + q;
-              if (j < p.h_out) {  // h_out is a multiple of 8: a group of 8 is all in or all out
+              if (j < jp.h_out) {  // h_out is a multiple of 8: a group of 8 is all in or all out
                 uint4 o;
                 o.x = ptx::pack_bf16x2(v[q + 0], v[q + 1]);
                 o.y = ptx::pack_bf16x2(v[q + 2], v[q + 3]);
@@ -486,22 +773,22 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
               }
             }
           }
-        } else if (p.mode == kModeDecode) {
+        } else if (jp.mode == kModeDecode) {
           // single K split: row = W row j, columns = tokens c0 + [0, 32), straight to y
-          if (row < p.h_out) {
+          if (row < jp.h_out) {
 #pragma unroll
             for (int jj = 0; jj < 32; ++jj) {
               const int t = c0 + jj;
-              if (t < p.T)
-                p.y[static_cast<size_t>(t) * p.h_out + row] =
+              if (t < jp.T)
+                jp.y[static_cast<size_t>(t) * jp.h_out + row] =
                     static_cast<uint16_t>(ptx::pack_bf16x2(v[jj], 0.f) & 0xFFFFu);
             }
           }
         } else {
           // sgmv: row = token of the run, columns = rank index; z partial = scale * acc
           if (row_in_tile < tc.nrows) {
-            float *zrow = p.zws_out + (static_cast<size_t>(tc.split) * p.max_tokens + row) * p.R_pad + c0;
-            const int nc = min(32, p.BN - c0);
+            float *zrow = jp.zws_out + (static_cast<size_t>(tc.split) * jp.max_tokens + row) * jp.R_pad + c0;
+            const int nc = min(32, jp.BN - c0);
             for (int q = 0; q < nc; q += 4)
               *reinterpret_cast<float4 *>(zrow + q) =
                   make_float4(scale * v[q], scale * v[q + 1], scale * v[q + 2], scale * v[q + 3]);
@@ -589,6 +876,13 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       if (btid == 0) ptx::mbar_arrive(lg_bar);
     }
     for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+      if (tile >= n_tiles0) {  // a tile of the second job: no LoRA blocks, only the ring moves on
+        const int32_t local = second_job_tile(tile);
+        if (local < 0) break;
+        const TileCoord t2 = tile_coord(p2, local);
+        count += static_cast<uint32_t>((t2.kb1 - t2.kb0) * tile_passes(p2, t2));
+        continue;
+      }
       const TileCoord tc = tile_coord(p, tile);
       count += static_cast<uint32_t>(tc.kb1 - tc.kb0);
       if (!waited) {  // z (and in prefill the tile lists) come from the kernels before this one
@@ -820,6 +1114,13 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   }
 }
 
+// A GemmParams that stands for "no second job".
+static GemmParams no_job() {
+  GemmParams none{};
+  none.mode = -1;
+  return none;
+}
+
 cudaError_t gemm_set_smem_limit(size_t smem_bytes) {
   cudaError_t e = cudaFuncSetAttribute(lora_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem_bytes));
@@ -831,12 +1132,23 @@ cudaError_t gemm_set_smem_limit(size_t smem_bytes) {
 cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
                         const CUtensorMap &tmap_b, const GemmParams &p, int32_t grid,
                         size_t smem_bytes, bool pdl, cudaStream_t stream) {
+  return launch_gemm2(tmap_row, tmap_col, tmap_b, p, tmap_row, tmap_col, tmap_b, no_job(), grid, smem_bytes,
+                      pdl, stream);
+}
+
+// With a second job: p2.mode == kModeSgmv (a shrink job: segment tiles and, with p2.gather, gather
+// tiles; tmap_g2 is then the one-row map of its x), p2.n_mtiles = upper bound on its tiles,
+// p2.BN and p2.gN <= p.ring_rows and p.acc_cols, and p is a prefill-mode job.
+cudaError_t launch_gemm2(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
+                         const CUtensorMap &tmap_b, const GemmParams &p, const CUtensorMap &tmap_row2,
+                         const CUtensorMap &tmap_col2, const CUtensorMap &tmap_g2, const GemmParams &p2,
+                         int32_t grid, size_t smem_bytes, bool pdl, cudaStream_t stream) {
   const int cluster = (p.mode == kModeDecode && p.splits > 1) ? p.splits : 1;
-  if (smem_bytes * 2 <= 225 * 1024 && p.BN <= 128)  // two CTAs fit an SM: registers within half the file
+  if (smem_bytes * 2 <= 225 * 1024 && p.BN <= 128 && p.acc_cols <= 128)  // two CTAs fit an SM
     return launch_ex(lora_gemm_kernel<2>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster,
-                     tmap_row, tmap_col, tmap_b, p);
+                     tmap_row, tmap_col, tmap_b, p, tmap_row2, tmap_col2, tmap_g2, p2);
   return launch_ex(lora_gemm_kernel<1>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster,
-                   tmap_row, tmap_col, tmap_b, p);
+                   tmap_row, tmap_col, tmap_b, p, tmap_row2, tmap_col2, tmap_g2, p2);
 }
 
 }  // namespace edgelora

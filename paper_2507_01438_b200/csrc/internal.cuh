@@ -58,7 +58,9 @@ struct GemmParams {
   int32_t BN;          // UMMA N = rows of the column-operand tile (multiple of 16, <= 256)
   int32_t stages;      // TMA pipeline depth
   int32_t n_acc;       // TMEM accumulator buffers (1 or 2)
-  int32_t tmem_cols;   // power of two >= n_acc * BN, >= 32
+  int32_t tmem_cols;   // power of two >= n_acc * acc_cols, >= 32
+  int32_t ring_rows;   // rows of the C region of a ring stage (>= BN; wider when gather passes need it)
+  int32_t acc_cols;    // TMEM columns between the accumulators (>= BN, >= gN)
   int32_t kb_total;    // K blocks of 64 covering h_in
   int32_t kb_per;      // K blocks per split
   int32_t splits;
@@ -70,6 +72,14 @@ struct GemmParams {
                              // reduction on the CUDA cores instead of by LoRA K blocks
   int32_t max_tokens;  // row stride of the z / plan workspaces
   long long wait_cycles;  // limit of the bounded in-kernel waits, in SM clock cycles
+  // shrink jobs (mode sgmv): gather tiles for the tokens the segment tiles do not cover
+  int32_t gather;      // 1: the job also has gather tiles (stacked A rows x gathered token rows)
+  int32_t finalize;    // 1: whoever completes a gather tile last adds its K splits into the final z plane
+  int32_t gN;          // most token rows of one gather pass (multiple of 16, <= rows of the ring's C region)
+  const int32_t *perm_short;     // plan: tokens ordered by (id, token), short runs only
+  const int32_t *gs_short;       // plan: group boundaries inside perm_short
+  const int32_t *group_adapter;  // plan: adapter of each group (-1 first when present)
+  int32_t *tile_counters;        // [>= gather tiles] arrivals per gather tile, zero between launches
   const int32_t *ids_valid;
   const int32_t *ids;       // decode: the caller's ids (validated again inside the kernel)
   int32_t n_slots;
@@ -88,14 +98,14 @@ struct GemmParams {
 // kernels (defined in plan.cu, shrink.cu, gemm.cu)
 void launch_plan(const int32_t *ids, int32_t T, int32_t n_slots, const PlanView &pv, bool pdl,
                  cudaStream_t stream);
-void launch_bgmv_shrink(const uint16_t *x, const uint16_t *A_pool, const SlotRow *slots,
-                        const PlanView &pv, float *zws, int32_t T, int32_t h_in, int32_t R_pad,
-                        int32_t n_slots, int32_t zsplits, int32_t max_tokens, int32_t sms,
-                        uint32_t *status, bool pdl, cudaStream_t stream);
 void init_plan_kernel();
 cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
                         const CUtensorMap &tmap_b, const GemmParams &p, int32_t grid,
                         size_t smem_bytes, bool pdl, cudaStream_t stream);
+cudaError_t launch_gemm2(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
+                         const CUtensorMap &tmap_b, const GemmParams &p, const CUtensorMap &tmap_row2,
+                         const CUtensorMap &tmap_col2, const CUtensorMap &tmap_g2, const GemmParams &p2,
+                         int32_t grid, size_t smem_bytes, bool pdl, cudaStream_t stream);
 cudaError_t gemm_set_smem_limit(size_t smem_bytes);
 cudaError_t shrink_set_smem_limit();
 cudaError_t launch_wait_selftest(uint32_t *status, long long wait_cycles, cudaStream_t stream);

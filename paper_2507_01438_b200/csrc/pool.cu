@@ -13,14 +13,20 @@
 #include <utility>
 #include <vector>
 
-#include "internal.cuh"
-#include "ptx.cuh"
+#include "pool.h"
 
 using namespace edgelora;
 
+namespace edgelora {
+thread_local char g_last_error[256] = "";
+void set_last_cuda_error(cudaError_t e, const char *what) {
+  snprintf(g_last_error, sizeof g_last_error, "%s: %s", what, cudaGetErrorString(e));
+  if (getenv("EDGELORA_LOG")) fprintf(stderr, "[edgelora] CUDA error: %s\n", g_last_error);
+}
+}  // namespace edgelora
+
 namespace {
 
-constexpr int kStagingBuffers = 4;
 constexpr int kTmapCache = 32;
 constexpr int kProfEvents = 8192;
 constexpr size_t kSmemBudget = 220 * 1024;
@@ -34,12 +40,6 @@ constexpr int kMaxDecodeSplits = 8;  // K splits of a row tile form one (portabl
       return EDGELORA_ERR_CUDA;                          \
     }                                                    \
   } while (0)
-
-thread_local char g_last_error[256] = "";
-void set_last_cuda_error(cudaError_t e, const char *what) {
-  snprintf(g_last_error, sizeof g_last_error, "%s: %s", what, cudaGetErrorString(e));
-  if (getenv("EDGELORA_LOG")) fprintf(stderr, "[edgelora] CUDA error: %s\n", g_last_error);
-}
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 inline int pad_rank(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : 64); }
@@ -60,19 +60,6 @@ EncodeTiledFn get_encode_fn() {
   }
   return fn;
 }
-
-struct TmapKey {
-  const void *base;
-  uint64_t d0, d1, d2;
-  uint32_t b1, b0;  // box rows, box columns (64 => 128-byte swizzle, otherwise no swizzle)
-  bool operator==(const TmapKey &o) const {
-    return base == o.base && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && b1 == o.b1 && b0 == o.b0;
-  }
-};
-struct TmapEntry {
-  TmapKey key;
-  CUtensorMap map;
-};
 
 // bf16 row-major [d2][d1][d0] (d2 == 0 => 2D), box = {box_cols, box_rows, 1}; out-of-range
 // elements read as zero.  box_cols == 64: the 128-byte-swizzled operand tiles of the GEMM;
@@ -97,67 +84,7 @@ int encode_tmap(CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1, ui
   return EDGELORA_OK;
 }
 
-struct StagingBuf {
-  uint8_t *host = nullptr;  // pinned: [A padded][B padded][SlotRow]
-  cudaEvent_t done = nullptr;
-  bool in_flight = false;
-};
-
-struct ProfRec {
-  int kernel;
-  cudaEvent_t start, stop;
-};
-
 }  // namespace
-
-struct edgelora_plan {
-  int32_t max_tokens = 0, n_slots = 0, last_T = 0;
-  void *block = nullptr;
-  PlanView pv{};
-};
-
-struct edgelora_pool {
-  edgelora_pool_config cfg{};
-  int R_pad = 0, device = 0, sms = 0;
-  bool owns_arena = false;
-  uint8_t *arena = nullptr;
-  uint16_t *A_pool = nullptr, *B_pool = nullptr;
-  size_t a_block = 0, b_block = 0;  // elements per slot
-  SlotRow *slots_dev = nullptr;
-  std::vector<SlotRow> slots_host;
-  StagingBuf staging[kStagingBuffers];
-  int next_staging = 0;
-  cudaStream_t side = nullptr;
-  cudaEvent_t load_ev = nullptr, use_ev = nullptr;
-  uint64_t load_seq = 0;
-  std::vector<std::pair<cudaStream_t, uint64_t>> load_waited;  // per stream: last load it waited for
-  bool use_recorded = false;
-  edgelora_plan *plan = nullptr;
-  float *zws = nullptr;
-  int32_t *group_counters = nullptr;
-  int opt_decode_splits = 0, opt_shrink_items = 0;
-  uint32_t *status_dev = nullptr;
-  std::vector<TmapEntry> tmaps;
-  size_t tmap_next = 0;
-  int opt_regime = 0, opt_profile = 0, opt_pdl = 1;
-  long long wait_cycles = ptx::kWaitLimitCycles;
-  int64_t last_info[8] = {0};
-  int64_t total_launches = 0;
-  // profiling
-  std::vector<ProfRec> prof;
-  size_t prof_used = 0;
-  double prof_ms[5] = {0};
-  int64_t prof_n[5] = {0};
-  // host-buffer entry point
-  uint16_t *hx = nullptr, *hy = nullptr, *dx = nullptr, *dy = nullptr;
-  int32_t *hids = nullptr, *dids = nullptr;
-  // pipelined host-buffer path: two sets of device mirrors, two copy streams, events per set
-  uint16_t *pdx[2] = {nullptr, nullptr}, *pdy[2] = {nullptr, nullptr};
-  int32_t *pdids[2] = {nullptr, nullptr};
-  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
-  cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
-  uint64_t host_calls = 0;
-};
 
 namespace {
 
@@ -582,6 +509,14 @@ int edgelora_pool_set_option(edgelora_pool_t *p, int32_t option, int32_t value) 
       if (value < 0) return EDGELORA_ERR_INVALID_ARG;
       p->opt_shrink_items = value;
       return EDGELORA_OK;
+    case EDGELORA_OPT_GATHER_SPLITS:
+      if (value < 0 || value > 8) return EDGELORA_ERR_INVALID_ARG;
+      p->opt_gather_splits = value;
+      return EDGELORA_OK;
+    case EDGELORA_OPT_GATHER_MIN_T:
+      if (value < 0 || value > kDecodeMaxT) return EDGELORA_ERR_INVALID_ARG;
+      p->opt_gather_min_t = value;
+      return EDGELORA_OK;
     default:
       return EDGELORA_ERR_INVALID_ARG;
   }
@@ -658,9 +593,12 @@ int edgelora_pool_selftest_wait(edgelora_pool_t *p, void *stream) {
 // The layer.  Decode regime (T <= 256): routing + shrink in one kernel, then the base product with
 // the expand and the split-K reduction fused in.  Prefill regime: plan, gather shrink for short
 // runs, segment shrink for long runs, base product with the expand fused in.
-static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_dev,
-                            const void *W_dev, const void *x_dev, int32_t T, void *y_dev,
-                            cudaStream_t stream) {
+}  // extern "C"
+
+namespace edgelora {
+int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_dev, const void *W_dev,
+                     const void *x_dev, int32_t T, void *y_dev, cudaStream_t stream, bool skip_shrink,
+                     const NextShrink *next) {
   if (!p || !plan || T < 0) return EDGELORA_ERR_INVALID_ARG;
   if (T == 0) return EDGELORA_OK;
   if (!W_dev || !x_dev || !y_dev) return EDGELORA_ERR_INVALID_ARG;
@@ -735,10 +673,103 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     return c;
   };
 
+  // The shrink of a pool as a job of the tile kernel: segment tiles for the long runs of a large
+  // batch (tile list from the plan) and gather tiles for every other token.  `decode`: no segment
+  // tiles, the K split count is chosen on the device from the number of adapters the batch touches,
+  // and whoever completes a tile last adds its splits into the final z plane.
+  const bool sgmv = T > kDecodeMaxT;
+  struct ShrinkJob {
+    GemmParams s;
+    CUtensorMap mx, ma, mg;
+    int grid = 1;
+    size_t smem = 0;
+  };
+  auto zsplits_of = [&](const edgelora_pool *q) {
+    if (!sgmv) return 1;
+    const int kbt = (q->cfg.h_in + kBlockK - 1) / kBlockK;
+    const int tiles_est = std::max(1, T / kTileM);
+    int z = std::max(1, std::min({8, q->sms / tiles_est, kbt / 4}));
+    const int kb_per = (kbt + z - 1) / z;
+    return (kbt + kb_per - 1) / kb_per;
+  };
+  auto shrink_job = [&](edgelora_pool *q, const uint16_t *xq, bool decode, int ring_rows, ShrinkJob *out) -> int {
+    const int kbt = (q->cfg.h_in + kBlockK - 1) / kBlockK;
+    const int Rq = q->R_pad;
+    GemmParams s{};
+    s.mode = kModeSgmv;
+    s.T = T;
+    s.h_in = q->cfg.h_in;
+    s.h_out = q->cfg.h_out;
+    s.kb_total = kbt;
+    s.R_pad = Rq;
+    s.BN = Rq;
+    s.max_tokens = q->cfg.max_tokens;
+    s.zsplits = decode ? 1 : zsplits_of(q);
+    s.splits = decode ? q->opt_gather_splits : s.zsplits;  // 0: the kernel picks the gather tiles' split count
+    while (s.splits > 1 && (s.splits - 1) * ((kbt + s.splits - 1) / s.splits) >= kbt) --s.splits;  // no empty split
+    s.kb_per = (kbt + s.zsplits - 1) / s.zsplits;
+    s.gather = 1;
+    s.finalize = decode ? 1 : 0;
+    // token rows of one gather pass: what the ring's C region holds (given when the job rides on
+    // another job's ring), 64 on its own ring (deep pipeline; a tile rarely has more tokens)
+    s.gN = ring_rows > 0 ? std::min(256, ring_rows / 16 * 16) : std::min(64, round_up(T, 16));
+    s.ring_rows = ring_rows > 0 ? ring_rows : std::max(Rq, s.gN);
+    s.acc_cols = s.ring_rows;
+    s.stages = stages_for(s.ring_rows, std::max(s.kb_per, 8), kSmemBudget);
+    s.n_acc = 2;
+    s.tmem_cols = pow2_cols(2 * s.acc_cols);
+    // upper bound of its tiles (the true count is on the device): segment tiles x splits + one gather
+    // tile per 128 / R_pad adapters x splits
+    const int max_gt = (std::min(T, q->cfg.n_slots) * Rq + kTileM - 1) / kTileM;
+    s.n_mtiles = (plan->pv.max_sgmv_tiles + max_gt) * std::max(s.zsplits, 1);
+    s.ids_valid = plan->pv.ids_valid;
+    s.ids = plan->pv.ids_valid;
+    s.n_slots = q->cfg.n_slots;
+    s.slots = q->slots_dev;
+    s.B_pool = q->B_pool;
+    s.zws = q->zws;
+    s.zws_out = q->zws;
+    s.sgmv_tiles = plan->pv.sgmv_tiles;
+    s.counts = plan->pv.counts;
+    s.mt_count = plan->pv.mt_count;
+    s.mt_list = plan->pv.mt_list;
+    s.perm_short = plan->pv.perm_short;
+    s.gs_short = plan->pv.gs_short;
+    s.group_adapter = plan->pv.group_adapter;
+    s.tile_counters = q->group_counters;
+    s.status = q->status_dev;
+    s.wait_cycles = q->wait_cycles;
+    out->s = s;
+    out->grid = q->sms;
+    out->smem = smem_for(s.stages, s.ring_rows);
+    int rc2 = get_tmap(q, &out->mx, xq, q->cfg.h_in, T, 0, kTileM);
+    if (rc2) return rc2;
+    rc2 = get_tmap(q, &out->mg, xq, q->cfg.h_in, T, 0, 1);
+    if (rc2) return rc2;
+    return get_tmap(q, &out->ma, q->A_pool, q->cfg.h_in, Rq, q->cfg.n_slots, Rq);
+  };
+  // decode batches above this size take the plan kernel + tensor-core gather tiles; smaller ones
+  // the single shrink kernel that derives the routing itself (a launch less)
+  const int kGatherMinT = p->opt_gather_min_t;
+
   if (regime == 1) {
     // ---------------------------------------------------------------- decode
     const int32_t *ids_in = ids_dev ? ids_dev : plan->pv.ids_valid;
     plan->last_T = T;
+    if (T > kGatherMinT) {
+      if (ids_dev) {
+        ProfScope ps(p, 0, stream);
+        launch_plan(ids_dev, T, plan->n_slots, plan->pv, pdl_first, stream);
+        CUDA_TRY(cudaGetLastError());
+        ++launches;
+      }
+      ShrinkJob sj;
+      int rc = shrink_job(p, x, true, 0, &sj);
+      if (rc) return rc;
+      ProfScope ps(p, 2, stream);
+      CUDA_TRY(launch_gemm(sj.mx, sj.ma, sj.mg, sj.s, sj.grid, sj.smem, ids_dev ? pdl : pdl_first, stream));
+      ++launches;
+    } else
     {
       ProfScope ps(p, 1, stream);
       // When calls overlap (EDGELORA_OPT_PDL = 2) a small batch's shrink runs under the previous
@@ -803,6 +834,8 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     while (splits > 1 && g.stages * stage_bytes < N * kTileM * 4 + (N / splits) * R * 4 && g.stages < kMaxStages)
       ++g.stages;
     g.n_acc = 1;
+    g.ring_rows = N;
+    g.acc_cols = N;
     g.tmem_cols = pow2_cols(N);
     CUtensorMap mr, mc, mb;
     int rc = get_tmap(p, &mr, W_dev, h_in, h_out, 0, kTileM);
@@ -831,49 +864,26 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
       CUDA_TRY(cudaGetLastError());
       ++launches;
     }
-    const bool sgmv = T > kDecodeMaxT;
-    // segment-shrink split-K factor (number of partial z planes the consumers sum)
-    int zsplits = 1;
-    if (sgmv) {
-      const int tiles_est = std::max(1, T / kTileM);
-      zsplits = std::max(1, std::min({8, p->sms / tiles_est, kb_total / 4}));
-      const int kb_per = (kb_total + zsplits - 1) / zsplits;
-      zsplits = (kb_total + kb_per - 1) / kb_per;
-    }
-    g.zsplits = zsplits;
-    {
-      ProfScope ps(p, 1, stream);
-      launch_bgmv_shrink(x, p->A_pool, p->slots_dev, plan->pv, p->zws, T, h_in, R, p->cfg.n_slots,
-                         zsplits, p->cfg.max_tokens, p->sms, p->status_dev, ids_dev ? pdl : pdl_first, stream);
-      CUDA_TRY(cudaGetLastError());
+    g.zsplits = zsplits_of(p);
+    if (!skip_shrink) {  // this site's shrink on its own, in front of its base product
+      ShrinkJob sj;
+      int rc = shrink_job(p, x, false, 0, &sj);
+      if (rc) return rc;
+      ProfScope ps(p, 2, stream);
+      CUDA_TRY(launch_gemm(sj.mx, sj.ma, sj.mg, sj.s, sj.grid, sj.smem, ids_dev ? pdl : pdl_first, stream));
       ++launches;
     }
     CUtensorMap mx;
     int rc = get_tmap(p, &mx, x, h_in, T, 0, kTileM);
     if (rc) return rc;
-    if (sgmv) {
-      GemmParams s = g;
-      s.mode = kModeSgmv;
-      s.BN = R;
-      s.splits = zsplits;
-      s.kb_per = (kb_total + zsplits - 1) / zsplits;
-      s.stages = stages_for(R, s.kb_per, kSmemBudget);
-      s.n_acc = 2;
-      s.tmem_cols = pow2_cols(2 * R);
-      CUtensorMap mc;
-      rc = get_tmap(p, &mc, p->A_pool, h_in, R, p->cfg.n_slots, R);
-      if (rc) return rc;
-      const int grid = std::max(1, std::min(p->sms, plan->pv.max_sgmv_tiles * zsplits));
-      ProfScope ps(p, 2, stream);
-      CUDA_TRY(launch_gemm(mx, mc, mc, s, grid, smem_for(s.stages, R), pdl, stream));
-      ++launches;
-    }
     const int n_mtiles = (T + kTileM - 1) / kTileM;
     const int tiles256 = n_mtiles * ((h_out + 255) / 256);
     int BN = (tiles256 >= p->sms || h_out <= 128) ? 256 : 128;
     BN = std::min(BN, round_up(h_out, 32));
     g.mode = kModePrefill;
     g.BN = BN;
+    g.ring_rows = BN;
+    g.acc_cols = BN;
     g.splits = 1;
     g.kb_per = kb_total;
     g.n_mtiles = n_mtiles;
@@ -886,15 +896,42 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
     if (rc) return rc;
     rc = get_tmap(p, &mb, p->B_pool, R, h_out, p->cfg.n_slots, BN);
     if (rc) return rc;
-    const int grid = std::min(p->sms, g.n_mtiles * g.n_ntiles);
-    ProfScope ps(p, 3, stream);
-    CUDA_TRY(launch_gemm(mx, mc, mb, g, grid, smem_for(g.stages, BN), pdl, stream));
-    ++launches;
+    int grid = std::min(p->sms, g.n_mtiles * g.n_ntiles);
+    // The next site of a set (independent of this one): its shrink rides on this site's
+    // base-product launch as extra tiles, on this launch's ring.
+    ShrinkJob nj;
+    bool fuse_next = false;
+    if (next && next->pool) {
+      edgelora_pool *q = next->pool;
+      if (q->cfg.max_tokens < T || q->cfg.n_slots != plan->n_slots) return EDGELORA_ERR_INVALID_ARG;
+      if (q->R_pad <= BN) {
+        rc = shrink_job(q, next->x, false, BN, &nj);
+        if (rc) return rc;
+        fuse_next = true;
+        grid = std::min(p->sms, g.n_mtiles * g.n_ntiles + nj.s.n_mtiles);
+      } else {  // cannot share the ring (a tiny site): on its own, before this site's base product
+        rc = shrink_job(q, next->x, false, 0, &nj);
+        if (rc) return rc;
+        ProfScope ps(q, 2, stream);
+        CUDA_TRY(launch_gemm(nj.mx, nj.ma, nj.mg, nj.s, nj.grid, nj.smem, pdl, stream));
+        ++launches;
+      }
+    }
+    {
+      ProfScope ps(p, 3, stream);
+      if (fuse_next)
+        CUDA_TRY(launch_gemm2(mx, mc, mb, g, nj.mx, nj.ma, nj.mg, nj.s, grid, smem_for(g.stages, BN), pdl, stream));
+      else
+        CUDA_TRY(launch_gemm(mx, mc, mb, g, grid, smem_for(g.stages, BN), pdl, stream));
+      ++launches;
+    }
     p->last_info[2] = grid;
     p->last_info[3] = 1;
   }
 
-  if (!capturing) {
+  // (inside a set of sites the set records the events once, after its last site: an event between
+  // two kernels would keep them from overlapping)
+  if (!capturing && !next && !skip_shrink) {
     CUDA_TRY(cudaEventRecord(p->use_ev, stream));
     p->use_recorded = true;
   }
@@ -905,6 +942,9 @@ static int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t
   p->total_launches += launches;
   return EDGELORA_OK;
 }
+}  // namespace edgelora
+
+extern "C" {
 
 int edgelora_lora_linear(edgelora_pool_t *pool, const void *W_dev, const void *x_dev,
                          const int32_t *adapter_id_dev, int32_t T, void *y_dev, void *stream) {

@@ -1,133 +1,11 @@
-// Gather-by-token shrink (BGMV): z[t] = s_a * A_a x[t] for tokens scattered across adapters
+// Shrink for small decode batches: z[t] = s_a * A_a x[t] for tokens scattered across adapters
 // (paper Section 2.1 for A: r x h_in; Section 4.3: tokens that share an adapter are handled as one
-// sub-batch so the adapter is fetched once).
-//
-// One work item per (group, rank row i), strided over the CTAs: a CTA streams row i of A_a once
-// from HBM with 128-bit loads and dots it against the x rows of up to eight tokens of the group at
-// a time; partial sums are reduced with warp shuffles and a small shared-memory stage.  It walks the plan's "short" token
-// lists: in large batches tokens that belong to long runs are left to the segment shrink.
+// sub-batch so the adapter is fetched once), with the routing derived inside the kernel so that a
+// step of a few microseconds needs no routing launch.  Larger batches take the tensor-core gather
+// tiles of the tile kernel (gemm.cu).
 #include "internal.cuh"
 #include "launch.cuh"
 #include "ptx.cuh"
-
-namespace edgelora {
-
-constexpr int kBgmvThreads = 256;
-constexpr int kBgmvTok = 8;
-
-__device__ __forceinline__ float dot8(const uint4 &a, const uint4 &b) {
-  float s = ptx::bf16_lo(a.x) * ptx::bf16_lo(b.x);
-  s = fmaf(ptx::bf16_hi(a.x), ptx::bf16_hi(b.x), s);
-  s = fmaf(ptx::bf16_lo(a.y), ptx::bf16_lo(b.y), s);
-  s = fmaf(ptx::bf16_hi(a.y), ptx::bf16_hi(b.y), s);
-  s = fmaf(ptx::bf16_lo(a.z), ptx::bf16_lo(b.z), s);
-  s = fmaf(ptx::bf16_hi(a.z), ptx::bf16_hi(b.z), s);
-  s = fmaf(ptx::bf16_lo(a.w), ptx::bf16_lo(b.w), s);
-  s = fmaf(ptx::bf16_hi(a.w), ptx::bf16_hi(b.w), s);
-  return s;
-}
-
-__global__ void __launch_bounds__(kBgmvThreads)
-bgmv_shrink_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ A_pool,
-                   const SlotRow *__restrict__ slots, PlanView pv, float *__restrict__ zws,
-                   int32_t T, int32_t h_in, int32_t R_pad, int32_t zsplits, int32_t max_tokens,
-                   int32_t max_groups, uint32_t *status) {
-  __shared__ float red[kBgmvThreads / 32][kBgmvTok];
-  __shared__ int32_t tok[kBgmvTok];
-
-  ptx::pdl_launch_dependents();
-  ptx::pdl_wait_prior_grids();  // the plan comes from the previous kernel
-
-  // Work items (group, rank row) are strided over a grid sized for the machine, not for the worst
-  // case of groups: most batches have far fewer groups than slots, and CTAs that only find out
-  // that they have nothing to do cost more than the items themselves.
-  // The plan arrays are cold by the time they are read here (a step streams gigabytes between
-  // two uses), so an item is a chain of dependent DRAM round trips; loads that do not depend on
-  // each other are issued together: {group count, the group's adapter and token range} (g is
-  // below the host's bound on groups, so these reads stay inside the arrays whatever the count
-  // turns out to be), then {slot row, first tokens}, then the rows themselves.
-  for (int wi = blockIdx.x; wi / R_pad < max_groups; wi += gridDim.x) {
-  const int g = wi / R_pad;
-  const int i = wi % R_pad;
-  const int n_groups = pv.counts[0];
-  const int a = pv.group_adapter[g];
-  const int g0 = pv.gs_short[g], g1 = pv.gs_short[g + 1];
-  if (g >= n_groups) break;
-  if (a < 0) continue;
-  int32_t first_tok = 0;
-  if (static_cast<int>(threadIdx.x) < min(kBgmvTok, g1 - g0)) first_tok = pv.perm_short[g0 + threadIdx.x];
-  const SlotRow row = slots[a];
-  if (row.rank <= 0) {
-    if (threadIdx.x == 0 && i == 0) atomicOr(status, EDGELORA_STATUS_SLOT_EMPTY);
-    continue;
-  }
-  const bool live_row = i < row.rank;
-  const uint4 *Arow =
-      reinterpret_cast<const uint4 *>(A_pool + (static_cast<size_t>(a) * R_pad + i) * h_in);
-  const int n8 = h_in >> 3;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const size_t zsplit_stride = static_cast<size_t>(max_tokens) * R_pad;
-
-  for (int base = g0; base < g1; base += kBgmvTok) {
-    const int n_tok = min(kBgmvTok, g1 - base);
-    __syncthreads();
-    if (threadIdx.x < n_tok) tok[threadIdx.x] = base == g0 ? first_tok : pv.perm_short[base + threadIdx.x];
-    __syncthreads();
-
-    if (!live_row) {  // padding rows of the block: z is defined as zero there
-      for (int q = threadIdx.x; q < n_tok * zsplits; q += kBgmvThreads)
-        zws[(q / n_tok) * zsplit_stride + static_cast<size_t>(tok[q % n_tok]) * R_pad + i] = 0.f;
-      continue;
-    }
-
-    float acc[kBgmvTok];
-    const uint4 *xrow[kBgmvTok];
-#pragma unroll
-    for (int q = 0; q < kBgmvTok; ++q) {
-      acc[q] = 0.f;
-      xrow[q] = reinterpret_cast<const uint4 *>(x + static_cast<size_t>(tok[min(q, n_tok - 1)]) * h_in);
-    }
-    // every load of a K step is issued before the first product: with the loads inside the
-    // per-token branches a step cost one memory round trip per token (4 us per token on a
-    // 14336-wide row)
-    for (int k = threadIdx.x; k < n8; k += kBgmvThreads) {
-      const uint4 av = __ldg(Arow + k);
-      uint4 xv[kBgmvTok];
-#pragma unroll
-      for (int q = 0; q < kBgmvTok; ++q) xv[q] = q < n_tok ? __ldg(xrow[q] + k) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-      for (int q = 0; q < kBgmvTok; ++q) acc[q] += dot8(av, xv[q]);
-    }
-#pragma unroll
-    for (int q = 0; q < kBgmvTok; ++q) {
-#pragma unroll
-      for (int d = 16; d > 0; d >>= 1) acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], d);
-      if (lane == 0) red[warp][q] = acc[q];
-    }
-    __syncthreads();
-    if (threadIdx.x < n_tok) {
-      float s = 0.f;
-#pragma unroll
-      for (int w = 0; w < kBgmvThreads / 32; ++w) s += red[w][threadIdx.x];
-      const size_t off = static_cast<size_t>(tok[threadIdx.x]) * R_pad + i;
-      zws[off] = row.scale * s;
-      for (int sp = 1; sp < zsplits; ++sp) zws[sp * zsplit_stride + off] = 0.f;
-    }
-  }
-  }
-}
-
-void launch_bgmv_shrink(const uint16_t *x, const uint16_t *A_pool, const SlotRow *slots,
-                        const PlanView &pv, float *zws, int32_t T, int32_t h_in, int32_t R_pad,
-                        int32_t n_slots, int32_t zsplits, int32_t max_tokens, int32_t sms,
-                        uint32_t *status, bool pdl, cudaStream_t stream) {
-  const int max_groups = (T < n_slots + 1) ? T : n_slots + 1;
-  const int grid = max_groups * R_pad < sms * 8 ? max_groups * R_pad : sms * 8;
-  launch_ex(bgmv_shrink_kernel, dim3(grid), dim3(kBgmvThreads), 0, stream, pdl, 1, x,
-            A_pool, slots, pv, zws, T, h_in, R_pad, zsplits, max_tokens, max_groups, status);
-}
-
-}  // namespace edgelora
 
 namespace edgelora {
 

@@ -67,27 +67,57 @@ def test_down_proj_many_tenant_full_size():
     projection_check(w, y, 4)
 
 
-def full_set_sites():
-    """All 7 sites of layers 0, 15 and 31, and one site (rotating) of every other layer."""
-    sites = [(l, s) for l in (0, 15, 31) for s in range(7)]
-    sites += [(l, l % 7) for l in range(32) if l not in (0, 15, 31)]
-    return sites
+def full_set_single_sites():
+    """One site (rotating through the seven projections) of every layer except 0, 15 and 31."""
+    return [(l, l % 7) for l in range(32) if l not in (0, 15, 31)]
+
+
+def full_set_rows(batch):
+    # the whole first token tile (64 decode tokens + the head of the first run), run boundaries, a
+    # few random rows
+    rows = boundary_rows(batch.ids, 4, 5)
+    return np.array(sorted(set(range(128)) | set(rows.tolist()[:10]) | {1087, 1088, 2111}))
+
+
+@pytest.mark.parametrize("layer", [0, 15, 31])
+def test_full_projection_set_whole_layers_through_the_site_set(layer):
+    # the seven projections of a decoder layer as one set of sites: one plan, the sites back to
+    # back with the next site's shrink riding on the current site's launches (what bench.py times)
+    import torch
+    batch = wl.full_set_batch()
+    assert batch.ids.shape[0] == 2112
+    rows = full_set_rows(batch)
+    sites = [wl.full_set_site(batch, layer, s) for s in range(7)]
+    pools = [make_pool(w, 2112) for w in sites]
+    Ws = [to_dev_bf16(w.W) for w in sites]
+    widths = (4096, 14336)
+    sset = B.edgelora_siteset_create([p.handle for p in pools], Ws, [widths.index(w.h_in) for w in sites], 2, 2112)
+    try:
+        ys = [torch.full((2112, w.h_out), float("nan"), dtype=torch.bfloat16, device="cuda") for w in sites]
+        B.edgelora_siteset_run(sset, [to_dev_bf16(batch.x4096), to_dev_bf16(batch.x14336)],
+                               torch.from_numpy(batch.ids).cuda(), ys)
+        torch.cuda.synchronize()
+        for w, pool, y in zip(sites, pools, ys):
+            assert pool.status() == (0, 0)
+            yh = from_dev_bf16(y)
+            assert_parity(yh[rows], oracle_of(w, rows), w.name)
+            projection_check(w, yh, 5 + layer)
+    finally:
+        B.edgelora_siteset_destroy(sset)
+        for p in pools:
+            p.close()
 
 
 def test_full_projection_set_sampled_sites():
     import torch
     batch = wl.full_set_batch()
-    assert batch.ids.shape[0] == 2112
-    # the whole first token tile (64 decode tokens + the head of the first run), run boundaries, a
-    # few random rows
-    rows = boundary_rows(batch.ids, 4, 5)
-    rows = np.array(sorted(set(range(128)) | set(rows.tolist()[:10]) | {1087, 1088, 2111}))
+    rows = full_set_rows(batch)
     ids_dev = torch.from_numpy(batch.ids).cuda()
     plan = B.edgelora_plan_create(2112, batch.n_slots)
     xs = {4096: to_dev_bf16(batch.x4096), 14336: to_dev_bf16(batch.x14336)}
     try:
         B.edgelora_plan_build(plan, ids_dev)             # one plan reused by every site
-        for (layer, site) in full_set_sites():
+        for (layer, site) in full_set_single_sites():
             w = wl.full_set_site(batch, layer, site)
             pool = make_pool(w, 2112)
             try:
@@ -96,8 +126,6 @@ def test_full_projection_set_sampled_sites():
                 assert pool.status() == (0, 0)
                 yh = from_dev_bf16(y)
                 assert_parity(yh[rows], oracle_of(w, rows), w.name)
-                if layer in (0, 31):
-                    projection_check(w, yh, 5 + site)
             finally:
                 pool.close()
     finally:

@@ -361,10 +361,10 @@ def test_profiling_option_reports_every_kernel():
         B.edgelora_pool_set_option(pool.handle, B.OPT_PROFILE, 1)
         run_gpu(w, pool=pool)
         t = B.edgelora_pool_kernel_times(pool.handle)
-        assert t["plan"]["launches"] == 1 and t["shrink_bgmv"]["launches"] == 1
-        assert t["shrink_sgmv"]["launches"] == 1 and t["base_gemm"]["launches"] == 1
+        assert t["plan"]["launches"] == 1 and t["shrink_small_decode"]["launches"] == 0
+        assert t["shrink_tiles"]["launches"] == 1 and t["base_gemm"]["launches"] == 1
         assert t["base_gemm"]["ms"] > 0
         info = B.edgelora_pool_last_launch(pool.handle)
-        assert info["launches"] == 4 and info["regime"] == "prefill"
+        assert info["launches"] == 3 and info["regime"] == "prefill"
     finally:
         pool.close()
