@@ -88,9 +88,10 @@ typedef struct {
 #define EDGELORA_OPT_SHRINK_ITEMS 5  /* tuning: work items the decode shrink aims for, 0 = auto   */
 #define EDGELORA_OPT_GATHER_SPLITS 7 /* tuning: K splits of the tensor-core gather shrink in decode, 0 = chosen
                                         on the device from the number of adapters the batch touches  */
-#define EDGELORA_OPT_GATHER_MIN_T 8  /* tuning: decode batches above this many tokens (default 64) use the
-                                        routing kernel + tensor-core gather shrink; smaller ones the
-                                        single shrink kernel with the routing inside                 */
+#define EDGELORA_OPT_GATHER_MIN_T 8  /* tuning: decode batches above this many tokens use the routing
+                                        kernel + tensor-core gather shrink, the others the single shrink
+                                        kernel with the routing inside.  Default 256: every decode batch
+                                        takes the single kernel (it is the faster one as measured)   */
 #define EDGELORA_OPT_WAIT_CYCLES 6   /* limit of every bounded in-kernel wait of the layer, in units
                                         of 1024 SM clock cycles; 0 = default (about two seconds).
                                         A wait that runs out raises EDGELORA_STATUS_TIMEOUT           */

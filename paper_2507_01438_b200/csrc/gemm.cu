@@ -236,6 +236,86 @@ __device__ __forceinline__ void load_z_packed(const GemmParams &p, int32_t t, in
   }
 }
 
+// The copies of one pass over a gather tile, K blocks [kb0, kb1).  A K block needs one copy per
+// group of the tile (its A block, R_pad rows of the R operand) and one per token quad (four rows of
+// x into the C operand).  A TMA copy is issued from a warp's uniform datapath, one lane after the
+// other at roughly a hundred cycles each, so the copies of a K block are dealt out to kGatherParts
+// warps (the producer warp is part 0 and also posts the byte count; the four builder warps, idle
+// during shrink tiles, are parts 1..4): copy i goes to part i % kGatherParts, lane i / kGatherParts.
+// The parts other than the producer follow it the way the builder warps follow it through LoRA
+// K blocks: the producer announces a free stage on the stage's "go" barrier, every other part
+// waits for that, issues its copies and arrives on the stage's "z full" barrier, which the MMA
+// warp waits for beside the byte count.  (Waiting on the stage's empty barrier directly would not
+// do: a part that has nothing to copy for a while can get several ring revolutions ahead, and a
+// parity wait cannot tell revolutions apart.)  A copy that lands before the byte count is posted
+// only drives the barrier's transaction count below zero for a moment.
+constexpr int kGatherParts = 5;
+__device__ __forceinline__ bool gather_pass_copies(const GemmParams &jp, const TileCoord &tc, int32_t t0,
+                                                   const CUtensorMap *ma, const CUtensorMap *mg, uint8_t *smem,
+                                                   uint32_t stage_bytes, uint64_t *full_bar, uint64_t *empty_bar,
+                                                   uint64_t *zgo_bar, uint64_t *zfull_bar,
+                                                   volatile uint32_t *abort_flag, uint32_t nstages, long long wl,
+                                                   int part, int lane, uint32_t &stage, uint32_t &phase,
+                                                   uint32_t &gophase) {
+  const uint32_t r_bytes = kTileM * kBlockK * 2;
+  const uint32_t a_bytes = static_cast<uint32_t>(jp.R_pad) * kBlockK * 2;
+  const int32_t n = min(jp.gN, tc.ntok - t0);
+  const int32_t n_quads = (n + 3) >> 2;
+  // live groups of the tile (an empty slot has no A block to fetch), for the byte count
+  int32_t slot_l = -1;
+  if (lane < tc.ng) {
+    const int32_t a = jp.group_adapter[tc.g0 + lane];
+    if (a >= 0 && jp.slots[a].rank > 0) slot_l = a;
+  }
+  const uint32_t live_mask = __ballot_sync(0xffffffffu, slot_l >= 0);
+  const uint32_t tx = __popc(live_mask) * a_bytes + static_cast<uint32_t>(n_quads) * 4 * kBlockK * 2;
+  // this lane's copy
+  const int32_t item = part + kGatherParts * lane;
+  int32_t my_slot = -1, my_quad = -1, tok[4] = {0, 0, 0, 0};
+  const int32_t slot_of_item = __shfl_sync(0xffffffffu, slot_l, item < tc.ng ? item : 0);
+  if (item < tc.ng) {
+    my_slot = slot_of_item;
+  } else {
+    if (item - tc.ng < n_quads) {
+      my_quad = item - tc.ng;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)  // rows past the pass's last token repeat it (they land in unused columns)
+        tok[i] = jp.perm_short[tc.tok0 + t0 + min(my_quad * 4 + i, n - 1)];
+    }
+  }
+  for (int32_t kb = tc.kb0; kb < tc.kb1; ++kb) {
+    int got = 1;
+    if (lane == 0) {
+      if (part == 0)
+        got = (ptx::mbar_wait(&empty_bar[stage], phase ^ 1, wl) && !*abort_flag) ? 1 : 0;
+      else
+        got = (ptx::mbar_wait(&zgo_bar[stage], (gophase >> stage) & 1u, wl) && !*abort_flag) ? 1 : 0;
+    }
+    if (!__shfl_sync(0xffffffffu, got, 0)) return false;
+    gophase ^= 1u << stage;
+    uint8_t *sr = smem + static_cast<size_t>(stage) * stage_bytes;
+    if (part == 0 && lane == 0) {
+      ptx::mbar_arrive(&zgo_bar[stage]);
+      ptx::mbar_arrive_expect_tx(&full_bar[stage], tx);
+    }
+    if (my_slot >= 0)
+      ptx::tma_load_2d(sr + static_cast<size_t>(item) * a_bytes, ma, &full_bar[stage], kb * kBlockK,
+                       my_slot * jp.R_pad);
+    if (my_quad >= 0)
+      ptx::tma_gather4_2d(sr + r_bytes + static_cast<size_t>(my_quad) * (4 * kBlockK * 2), mg, &full_bar[stage],
+                          kb * kBlockK, tok[0], tok[1], tok[2], tok[3]);
+    if (part != 0) {
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&zfull_bar[stage]);
+    }
+    if (++stage == nstages) {
+      stage = 0;
+      phase ^= 1;
+    }
+  }
+  return true;
+}
+
 // kMinBlocks = 2 caps the registers so that two CTAs share an SM (small decode tiles); with 1 the
 // builder keeps both of its z rows in registers without spilling.
 template <int kMinBlocks>
@@ -243,7 +323,8 @@ __global__ void __launch_bounds__(kGemmThreads, kMinBlocks)
 lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_constant__ CUtensorMap tmap_c,
                  const __grid_constant__ CUtensorMap tmap_b, const GemmParams p,
                  const __grid_constant__ CUtensorMap tmap_r2, const __grid_constant__ CUtensorMap tmap_c2,
-                 const __grid_constant__ CUtensorMap tmap_g2, const GemmParams p2) {
+                 const __grid_constant__ CUtensorMap tmap_g2, const GemmParams p2,
+                 const __grid_constant__ CUtensorMap tmap_y) {
   extern __shared__ uint8_t smem_raw[];
   // tiles need 1024-byte alignment for the 128-byte swizzle
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -276,6 +357,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   uint32_t *s_key = reinterpret_cast<uint32_t *>(extra + 2432);             // [256] sort keys
   volatile int32_t *s_last = reinterpret_cast<volatile int32_t *>(extra + 80);  // gather tiles: last arriver
   uint64_t *ep_bar = reinterpret_cast<uint64_t *>(extra + 88);              // rendezvous of the epilogue warps
+  uint8_t *y_stage = reinterpret_cast<uint8_t *>(bars) + 4096;              // prefill epilogue: 4 x 4 KB, 1024-aligned
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wl = p.wait_cycles;  // limit of every bounded wait below
@@ -294,6 +376,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       if (p2.gather) ptx::prefetch_tensormap(&tmap_g2);
     }
     if (p.mode == kModeSgmv && p.gather) ptx::prefetch_tensormap(&tmap_b);
+    if (p.y_tma) ptx::prefetch_tensormap(&tmap_y);
     for (int s = 0; s < p.stages; ++s) {
       ptx::mbar_init(&full_bar[s], 1);
       ptx::mbar_init(&empty_bar[s], 1);
@@ -344,7 +427,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     // The whole warp walks the loop (state stays uniform); lane 0 waits and issues the tile loads,
     // and for gather tiles every lane issues its share of the one-row loads.
     {
-      uint32_t stage = 0, phase = 0;
+      uint32_t stage = 0, phase = 0, unused_go = 0;
       bool ok = true, waited = p.mode == kModeSgmv;
       auto wait_empty = [&]() {  // lane 0 polls, the warp learns the result
         int got = 1;
@@ -365,43 +448,11 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         const CUtensorMap *mr = second ? &tmap_r2 : &tmap_r, *mc = second ? &tmap_c2 : &tmap_c;
         const TileCoord tc = tile_coord(jp, local);
         if (tc.kind == 1) {
-          // gather tile: lane i fetches the A block of the tile's i-th group (rows [i R_pad, ...) of
-          // the R tile), lane l the x rows of tokens l, l + 32, ... of the pass
+          // gather tile: this warp is part 0 of the copies (see gather_pass_copies)
           const CUtensorMap *mg = second ? &tmap_g2 : &tmap_b;
-          int32_t my_slot = -1;
-          if (lane < tc.ng) {
-            const int32_t a = jp.group_adapter[tc.g0 + lane];
-            if (a >= 0 && jp.slots[a].rank > 0) my_slot = a;
-          }
-          const uint32_t n_live = __popc(__ballot_sync(0xffffffffu, my_slot >= 0));
-          const uint32_t a_bytes = static_cast<uint32_t>(jp.R_pad) * kBlockK * 2;
-          for (int32_t t0 = 0; ok && t0 < tc.ntok; t0 += jp.gN) {
-            const int32_t n = min(jp.gN, tc.ntok - t0);
-            int32_t tok[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              const int c = q * 32 + lane;
-              tok[q] = c < n ? jp.perm_short[tc.tok0 + t0 + c] : -1;
-            }
-            const uint32_t tx = n_live * a_bytes + static_cast<uint32_t>(n) * kBlockK * 2;
-            for (int32_t kb = tc.kb0; kb < tc.kb1; ++kb) {
-              if (!wait_empty()) {
-                ok = false;
-                break;
-              }
-              uint8_t *sr = smem + static_cast<size_t>(stage) * stage_bytes;
-              if (lane == 0) ptx::mbar_arrive_expect_tx(&full_bar[stage], tx);
-              __syncwarp();
-              if (my_slot >= 0)
-                ptx::tma_load_3d(sr + static_cast<size_t>(lane) * a_bytes, mc, &full_bar[stage], kb * kBlockK, 0, my_slot);
-#pragma unroll
-              for (int q = 0; q < 8; ++q)
-                if (tok[q] >= 0)
-                  ptx::tma_load_2d(sr + r_bytes + static_cast<size_t>(q * 32 + lane) * (kBlockK * 2), mg,
-                                   &full_bar[stage], kb * kBlockK, tok[q]);
-              advance();
-            }
-          }
+          for (int32_t t0 = 0; ok && t0 < tc.ntok; t0 += jp.gN)
+            ok = gather_pass_copies(jp, tc, t0, mc, mg, smem, stage_bytes, full_bar, empty_bar, zgo_bar, zfull_bar,
+                                    abort_flag, nstages, wl, 0, lane, stage, phase, unused_go);
           continue;
         }
         const uint32_t tx_bytes = r_bytes + static_cast<uint32_t>(jp.BN) * kBlockK * 2;
@@ -415,7 +466,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
             ptx::mbar_arrive_expect_tx(&full_bar[stage], tx_bytes);
             ptx::tma_load_2d(sr, mr, &full_bar[stage], kb * kBlockK, tc.row_r);
             if (jp.mode == kModeSgmv)
-              ptx::tma_load_3d(sr + r_bytes, mc, &full_bar[stage], kb * kBlockK, 0, tc.slot);
+              ptx::tma_load_2d(sr + r_bytes, mc, &full_bar[stage], kb * kBlockK, tc.slot * jp.R_pad);
             else
               ptx::tma_load_2d(sr + r_bytes, mc, &full_bar[stage], kb * kBlockK, tc.row_c);
           }
@@ -497,6 +548,13 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
             if (!ptx::mbar_wait(&full_bar[stage], phase, wl) || *abort_flag) {
               ok = false;
               break;
+            }
+            if (tc.kind == 1) {  // the other parts of the tile's copies have been through this stage
+              if (!ptx::mbar_wait(&zfull_bar[stage], (zphase >> stage) & 1u, wl)) {
+                ok = false;
+                break;
+              }
+              zphase ^= 1u << stage;
             }
             ptx::tc_fence_after_sync();
             const uint32_t sr = ptx::smem_u32(smem + static_cast<size_t>(stage) * stage_bytes);
@@ -756,7 +814,37 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
             v[i + 16] = 0.f;
           }
         }
-        if (jp.mode == kModePrefill) {
+        if (jp.mode == kModePrefill && jp.y_tma) {
+          // row = token, columns = output features row_c + c0 + [0, 32).  The warp's 32 rows x 64
+          // columns go to its shared-memory stage as bf16 (rows of 128 bytes, 16-byte chunks
+          // swizzled by the row so that the lanes' stores spread over the banks) and leave with one
+          // TMA store: whole 128-byte lines to memory instead of 32 scattered pieces per
+          // instruction; rows and columns outside y are dropped by the copy.
+          uint8_t *my_stage = y_stage + quad * (32 * 128);
+          const int half = (c0 >> 5) & 1;  // which 64 bytes of the stage row
+          if (half == 0) {                 // the previous store of this warp has read the stage
+            if (lane == 0) ptx::bulk_wait_group_read0();
+            __syncwarp();
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint4 o;
+            o.x = ptx::pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
+            o.y = ptx::pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
+            o.z = ptx::pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
+            o.w = ptx::pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
+            const int chunk = half * 4 + q;
+            *reinterpret_cast<uint4 *>(my_stage + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = o;
+          }
+          if (half == 1 || c0 + 32 >= jp.BN) {
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              ptx::tma_store_2d(&tmap_y, my_stage, tc.row_c + (c0 & ~63), tc.row_r + quad * 32);
+              ptx::bulk_commit_group();
+            }
+          }
+        } else if (jp.mode == kModePrefill) {
           // row = token, columns = output features row_c + c0 + [0, 32)
           if (row < jp.T) {
             uint16_t *yrow = jp.y + static_cast<size_t>(row) * jp.h_out;
@@ -807,15 +895,33 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       *abort_flag = 1;
       atomicOr(p.status, EDGELORA_STATUS_TIMEOUT);
     }
-  } else if (has_lora) {
+  } else if (has_lora || has2 || (p.mode == kModeSgmv && p.gather)) {
     // ------------------------------------------------------------ z operand builder (warps 6..9)
+    // (and, during gather tiles, parts 1..4 of the tile's copies)
     const int btid = threadIdx.x - 192;  // 0..127
     const int bwarp = warp - 6;
     const int nch = p.R_pad >> 3;        // 16-byte chunks of one operand row that the MMAs read
     uint32_t count = 0;                  // K blocks so far: stage = count % stages
     uint32_t gophase = 0;                // one parity bit per stage for zgo_bar
     bool ok = true, waited = false;
-    if (p.mode == kModeDecode) {
+    // a shrink tile (of the second job, or of a first job that is a shrink job): gather tiles take
+    // this warp's part of the copies, segment tiles only move the ring on
+    auto shrink_tile = [&](const GemmParams &jp, int32_t local, const CUtensorMap *ma, const CUtensorMap *mg) {
+      const TileCoord t2 = tile_coord(jp, local);
+      if (t2.kind != 1) {
+        count += static_cast<uint32_t>(t2.kb1 - t2.kb0);
+        return true;
+      }
+      for (int32_t t0 = 0; t0 < t2.ntok; t0 += jp.gN) {
+        uint32_t stage = count % nstages, phase = (count / nstages) & 1u;
+        if (!gather_pass_copies(jp, t2, t0, ma, mg, smem, stage_bytes, full_bar, empty_bar, zgo_bar, zfull_bar,
+                                abort_flag, nstages, wl, 1 + bwarp, lane, stage, phase, gophase))
+          return false;
+        count += static_cast<uint32_t>(t2.kb1 - t2.kb0);
+      }
+      return true;
+    };
+    if (has_lora && p.mode == kModeDecode) {
       // The batch's adapters (paper Section 3.4: one u-batch per adapter), distinct and ascending,
       // straight from the caller's ids so that the B_a tiles can be fetched before the shrink
       // kernel has finished.  Thread b looks after tokens b and b + 128.
@@ -876,15 +982,19 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       if (btid == 0) ptx::mbar_arrive(lg_bar);
     }
     for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
-      if (tile >= n_tiles0) {  // a tile of the second job: no LoRA blocks, only the ring moves on
+      if (tile >= n_tiles0) {  // a tile of the second job: no LoRA blocks
         const int32_t local = second_job_tile(tile);
         if (local < 0) break;
-        const TileCoord t2 = tile_coord(p2, local);
-        count += static_cast<uint32_t>((t2.kb1 - t2.kb0) * tile_passes(p2, t2));
+        ok = shrink_tile(p2, local, &tmap_c2, &tmap_g2);
+        continue;
+      }
+      if (p.mode == kModeSgmv) {  // the first job is a shrink job
+        ok = shrink_tile(p, tile, &tmap_c, &tmap_b);
         continue;
       }
       const TileCoord tc = tile_coord(p, tile);
       count += static_cast<uint32_t>(tc.kb1 - tc.kb0);
+      if (!has_lora) continue;
       if (!waited) {  // z (and in prefill the tile lists) come from the kernels before this one
         ptx::pdl_wait_prior_grids();
         waited = true;
@@ -1106,6 +1216,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     }
   }
 
+  if (p.y_tma && warp >= 2 && warp < 6 && lane == 0) ptx::bulk_wait_group0();  // this warp's y stores
   ptx::tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) {
@@ -1131,9 +1242,9 @@ cudaError_t gemm_set_smem_limit(size_t smem_bytes) {
 
 cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
                         const CUtensorMap &tmap_b, const GemmParams &p, int32_t grid,
-                        size_t smem_bytes, bool pdl, cudaStream_t stream) {
+                        size_t smem_bytes, bool pdl, cudaStream_t stream, const CUtensorMap *tmap_y) {
   return launch_gemm2(tmap_row, tmap_col, tmap_b, p, tmap_row, tmap_col, tmap_b, no_job(), grid, smem_bytes,
-                      pdl, stream);
+                      pdl, stream, tmap_y);
 }
 
 // With a second job: p2.mode == kModeSgmv (a shrink job: segment tiles and, with p2.gather, gather
@@ -1142,13 +1253,15 @@ cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col
 cudaError_t launch_gemm2(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
                          const CUtensorMap &tmap_b, const GemmParams &p, const CUtensorMap &tmap_row2,
                          const CUtensorMap &tmap_col2, const CUtensorMap &tmap_g2, const GemmParams &p2,
-                         int32_t grid, size_t smem_bytes, bool pdl, cudaStream_t stream) {
+                         int32_t grid, size_t smem_bytes, bool pdl, cudaStream_t stream,
+                         const CUtensorMap *tmap_y) {
+  const CUtensorMap &my = tmap_y ? *tmap_y : tmap_row;  // unused unless p.y_tma
   const int cluster = (p.mode == kModeDecode && p.splits > 1) ? p.splits : 1;
   if (smem_bytes * 2 <= 225 * 1024 && p.BN <= 128 && p.acc_cols <= 128)  // two CTAs fit an SM
     return launch_ex(lora_gemm_kernel<2>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster,
-                     tmap_row, tmap_col, tmap_b, p, tmap_row2, tmap_col2, tmap_g2, p2);
+                     tmap_row, tmap_col, tmap_b, p, tmap_row2, tmap_col2, tmap_g2, p2, my);
   return launch_ex(lora_gemm_kernel<1>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster,
-                   tmap_row, tmap_col, tmap_b, p, tmap_row2, tmap_col2, tmap_g2, p2);
+                   tmap_row, tmap_col, tmap_b, p, tmap_row2, tmap_col2, tmap_g2, p2, my);
 }
 
 }  // namespace edgelora

@@ -61,6 +61,7 @@ struct GemmParams {
   int32_t tmem_cols;   // power of two >= n_acc * acc_cols, >= 32
   int32_t ring_rows;   // rows of the C region of a ring stage (>= BN; wider when gather passes need it)
   int32_t acc_cols;    // TMEM columns between the accumulators (>= BN, >= gN)
+  int32_t y_tma;       // prefill: y leaves through a shared-memory stage and TMA stores (needs the y map)
   int32_t kb_total;    // K blocks of 64 covering h_in
   int32_t kb_per;      // K blocks per split
   int32_t splits;
@@ -101,11 +102,13 @@ void launch_plan(const int32_t *ids, int32_t T, int32_t n_slots, const PlanView 
 void init_plan_kernel();
 cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
                         const CUtensorMap &tmap_b, const GemmParams &p, int32_t grid,
-                        size_t smem_bytes, bool pdl, cudaStream_t stream);
+                        size_t smem_bytes, bool pdl, cudaStream_t stream, const CUtensorMap *tmap_y = nullptr);
 cudaError_t launch_gemm2(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
                          const CUtensorMap &tmap_b, const GemmParams &p, const CUtensorMap &tmap_row2,
                          const CUtensorMap &tmap_col2, const CUtensorMap &tmap_g2, const GemmParams &p2,
-                         int32_t grid, size_t smem_bytes, bool pdl, cudaStream_t stream);
+                         int32_t grid, size_t smem_bytes, bool pdl, cudaStream_t stream,
+                         const CUtensorMap *tmap_y = nullptr);
+constexpr int kYStageBytes = 4 * 32 * 128;  // prefill epilogue: per epilogue warp 32 rows x 64 bf16
 cudaError_t gemm_set_smem_limit(size_t smem_bytes);
 cudaError_t shrink_set_smem_limit();
 cudaError_t launch_wait_selftest(uint32_t *status, long long wait_cycles, cudaStream_t stream);

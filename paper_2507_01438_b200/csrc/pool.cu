@@ -659,9 +659,10 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
   g.status = p->status_dev;
   g.wait_cycles = p->wait_cycles;
 
-  auto smem_for = [](int stages, int BN) {
+  auto smem_for = [](int stages, int BN, int extra = 0) {
     // alignment slack + operand ring + barriers (512) + decode extras (3456, rounded up)
-    return static_cast<size_t>(1024 + stages * (kTileM * kBlockK * 2 + BN * kBlockK * 2) + 4096);
+    // (+ the prefill epilogue's staging area, 1024-aligned because every part before it is)
+    return static_cast<size_t>(1024 + stages * (kTileM * kBlockK * 2 + BN * kBlockK * 2) + 4096 + extra);
   };
   auto stages_for = [&](int BN, int k_blocks_per_cta, size_t budget) {
     int s = static_cast<int>((budget - 5120) / (kTileM * kBlockK * 2 + BN * kBlockK * 2));
@@ -684,11 +685,15 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
     int grid = 1;
     size_t smem = 0;
   };
+  // Inside a set of sites the shrink tiles ride on another site's base-product launch, where few
+  // large items fit into the slack of its last wave better than many small ones; on its own the
+  // shrink is split until every SM has an item.
+  const bool in_set = skip_shrink || next != nullptr;
   auto zsplits_of = [&](const edgelora_pool *q) {
     if (!sgmv) return 1;
     const int kbt = (q->cfg.h_in + kBlockK - 1) / kBlockK;
     const int tiles_est = std::max(1, T / kTileM);
-    int z = std::max(1, std::min({8, q->sms / tiles_est, kbt / 4}));
+    int z = std::max(1, std::min({in_set ? 2 : 8, q->sms / tiles_est, kbt / 4}));
     const int kb_per = (kbt + z - 1) / z;
     return (kbt + kb_per - 1) / kb_per;
   };
@@ -746,7 +751,8 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
     if (rc2) return rc2;
     rc2 = get_tmap(q, &out->mg, xq, q->cfg.h_in, T, 0, 1);
     if (rc2) return rc2;
-    return get_tmap(q, &out->ma, q->A_pool, q->cfg.h_in, Rq, q->cfg.n_slots, Rq);
+    // the A blocks as one 2D matrix [n_slots * R_pad][h_in]: slot a is rows [a R_pad, (a + 1) R_pad)
+    return get_tmap(q, &out->ma, q->A_pool, q->cfg.h_in, static_cast<uint64_t>(Rq) * q->cfg.n_slots, 0, Rq);
   };
   // decode batches above this size take the plan kernel + tensor-core gather tiles; smaller ones
   // the single shrink kernel that derives the routing itself (a launch less)
@@ -888,10 +894,13 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
     g.kb_per = kb_total;
     g.n_mtiles = n_mtiles;
     g.n_ntiles = (h_out + BN - 1) / BN;
-    g.stages = stages_for(BN, kb_total, kSmemBudget);
+    g.stages = stages_for(BN, kb_total, kSmemBudget - kYStageBytes);
     g.n_acc = 2;
     g.tmem_cols = pow2_cols(2 * BN);
-    CUtensorMap mc, mb;
+    g.y_tma = 1;
+    CUtensorMap mc, mb, my;
+    rc = get_tmap(p, &my, y_dev, h_out, T, 0, 32, kBlockK);  // y in boxes of 32 rows x 64 columns
+    if (rc) return rc;
     rc = get_tmap(p, &mc, W_dev, h_in, h_out, 0, BN);
     if (rc) return rc;
     rc = get_tmap(p, &mb, p->B_pool, R, h_out, p->cfg.n_slots, BN);
@@ -920,9 +929,10 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
     {
       ProfScope ps(p, 3, stream);
       if (fuse_next)
-        CUDA_TRY(launch_gemm2(mx, mc, mb, g, nj.mx, nj.ma, nj.mg, nj.s, grid, smem_for(g.stages, BN), pdl, stream));
+        CUDA_TRY(launch_gemm2(mx, mc, mb, g, nj.mx, nj.ma, nj.mg, nj.s, grid, smem_for(g.stages, BN, kYStageBytes), pdl,
+                              stream, &my));
       else
-        CUDA_TRY(launch_gemm(mx, mc, mb, g, grid, smem_for(g.stages, BN), pdl, stream));
+        CUDA_TRY(launch_gemm(mx, mc, mb, g, grid, smem_for(g.stages, BN, kYStageBytes), pdl, stream, &my));
       ++launches;
     }
     p->last_info[2] = grid;

@@ -21,7 +21,7 @@ def make_pool(w: "wl.Workload", max_tokens=0) -> "B.Pool":
     return pool
 
 
-def run_gpu(w: "wl.Workload", regime: int = 0, pool=None, return_plan=False):
+def run_gpu(w: "wl.Workload", regime: int = 0, pool=None, return_plan=False, options=None):
     """Runs the layer once; returns y as fp32 numpy [T, h_out] (and the exported plan)."""
     import torch
     own = pool is None
@@ -29,6 +29,8 @@ def run_gpu(w: "wl.Workload", regime: int = 0, pool=None, return_plan=False):
         pool = make_pool(w)
     try:
         B.edgelora_pool_set_option(pool.handle, B.OPT_REGIME, regime)
+        for opt, value in (options or {}).items():
+            B.edgelora_pool_set_option(pool.handle, opt, value)
         W = to_dev_bf16(w.W)
         x = to_dev_bf16(w.x)
         ids = torch.from_numpy(w.ids).cuda()

@@ -12,7 +12,11 @@ from test_gpu_parity import check_plan, random_workload
 
 pytestmark = pytest.mark.gpu
 
+# decode batches take the tensor-core gather shrink only when asked to (a tuning option)
+GATHER = {B.OPT_GATHER_MIN_T: 16}
 
+
+@pytest.mark.parametrize("splits", [0, 3])
 @pytest.mark.parametrize("T,n_adapters,max_rank,h_in", [
     (256, 1, 16, 512),     # one adapter, 256 tokens: one tile, four passes of 64 tokens
     (200, 3, 64, 1088),    # rank 64: two adapters per tile, ~67 tokens each, ragged K (17 K blocks)
@@ -21,7 +25,7 @@ pytestmark = pytest.mark.gpu
     (65, 65, 8, 256),      # as many adapters as tokens (one token each), nine tiles
     (256, 100, 64, 896),   # 50 tiles of two adapters
 ])
-def test_decode_sized_batches(T, n_adapters, max_rank, h_in):
+def test_decode_sized_batches(T, n_adapters, max_rank, h_in, splits):
     rng = np.random.Generator(np.random.PCG64(T + n_adapters))
     ranks = [int(r) for r in rng.integers(1, max_rank + 1, size=n_adapters)]
     ranks[0] = max_rank
@@ -30,7 +34,7 @@ def test_decode_sized_batches(T, n_adapters, max_rank, h_in):
         w.ids[:] = 0
     elif n_adapters >= T:
         w.ids = rng.permutation(n_adapters)[:T].astype(np.int32)
-    y, plan = run_gpu(w, 1, return_plan=True)
+    y, plan = run_gpu(w, 1, return_plan=True, options={**GATHER, B.OPT_GATHER_SPLITS: splits})
     assert_parity(y, oracle_of(w), f"T={T} adapters={n_adapters} rank<={max_rank}")
     check_plan(plan, w.ids, w.n_slots)
 
@@ -45,6 +49,7 @@ def test_empty_slot_inside_a_tile():
     from gpu_helpers import from_dev_bf16, make_pool, to_dev_bf16
     pool = make_pool(w)
     try:
+        B.edgelora_pool_set_option(pool.handle, B.OPT_GATHER_MIN_T, 16)
         y = from_dev_bf16(pool.linear(to_dev_bf16(w.W), to_dev_bf16(w.x), torch.from_numpy(ids).cuda()))
         rc, bits = pool.status()
         assert rc == B.ERR_SLOT_EMPTY and bits == B.STATUS_SLOT_EMPTY
@@ -75,9 +80,9 @@ def test_repeated_calls_reuse_the_arrival_counters():
     from gpu_helpers import make_pool
     pool = make_pool(w)
     try:
-        first = run_gpu(w, pool=pool)
+        first = run_gpu(w, pool=pool, options=GATHER)
         assert_parity(first, oracle_of(w), "first call")
         for _ in range(3):
-            assert np.array_equal(run_gpu(w, pool=pool), first)
+            assert np.array_equal(run_gpu(w, pool=pool, options=GATHER), first)
     finally:
         pool.close()
