@@ -308,6 +308,12 @@ int edgelora_cache_acquire(edgelora_cache_t *cache, int64_t key, int32_t pin, in
 int edgelora_cache_select(edgelora_cache_t *cache, const float *scores, int32_t n, int32_t k,
                           int32_t pin, int64_t *key_out, int32_t *slot_out, int32_t *hit_out,
                           int64_t *evicted_key_out);
+/* Section 4.2: "during server initialization, the memory cache is prefilled with random adapters".
+ * Makes keys[0..n) (distinct, n <= n_blocks; which ones is the caller's draw) resident in an empty
+ * cache, block i for keys[i] (the lowest free block each time), without holds, and leaves the hit /
+ * miss counters at zero so that they describe the serving phase.  blocks_out may be NULL.  The
+ * caller loads those adapters into the pools' slots. */
+int edgelora_cache_prefill(edgelora_cache_t *cache, const int64_t *keys, int32_t n, int32_t *blocks_out);
 /* Drops one hold on `key` (EDGELORA_ERR_INVALID_ARG if it has none). */
 int edgelora_cache_release(edgelora_cache_t *cache, int64_t key);
 /* Block of `key` or -1, without touching recency or counts. */
@@ -315,6 +321,49 @@ int edgelora_cache_lookup(const edgelora_cache_t *cache, int64_t key, int32_t *s
 /* Counters since creation; any pointer may be NULL. */
 int edgelora_cache_stats(const edgelora_cache_t *cache, int64_t *hits, int64_t *misses,
                          int64_t *evictions, int32_t *resident);
+
+/* ---- Request batcher: the slot state machine of the server manager (Section 4 "Slot state
+ * machine": idle -> adapter selection (Algorithm 1) -> prompt processing -> generation; slots in the
+ * prompt or generation state are grouped into one batch per step; Section 5.1: gamma slots bound
+ * the requests in flight, the rest queue).  Host memory only, no CUDA call; one thread per batcher.
+ * The batcher borrows `cache` (whose blocks are the slots of the adapter pools) and holds a
+ * request's adapter there until the request finishes.  Time is virtual and the caller's. */
+typedef struct edgelora_batcher edgelora_batcher_t;
+/* n_slots = gamma; max_batch_tokens >= n_slots bounds the tokens of one step (every generating
+ * slot gives one token, the rest of the budget goes to prompts, which are cut and continued);
+ * top_k = candidates per request. */
+int edgelora_batcher_create(int32_t n_slots, int32_t max_batch_tokens, int32_t top_k,
+                            edgelora_cache_t *cache, edgelora_batcher_t **batcher_out);
+int edgelora_batcher_destroy(edgelora_batcher_t *batcher);
+/* A request: arrival time in seconds (calls in ascending arrival order), prompt and output length in
+ * tokens (>= 1), and the router's top_k adapters in descending order of confidence (host array). */
+int edgelora_batcher_submit(edgelora_batcher_t *batcher, int64_t request_id, double arrival,
+                            int32_t in_len, int32_t out_len, const int64_t *candidates);
+/* Forms the next step's batch.  Admits arrived requests (arrival order, lowest idle slot first),
+ * chooses their adapters (the first resident candidate, else the first candidate is loaded; the
+ * choice is held until the request ends; a slot waits in the selection state while every block is
+ * held), then lists the tokens: one per generating slot (slot order), then the prompt tokens of the
+ * slots in the prompt state (slot order).  token_block[i] is the pool slot of token i's adapter,
+ * token_slot[i] the batcher slot it belongs to (arrays of `capacity` >= max_batch_tokens entries);
+ * load_key / load_block (n_slots entries each) name the adapters the caller must load into those
+ * pool slots before running the step.  When nothing is in flight the clock jumps to the next
+ * arrival.  Returns 1 with a batch, 0 when every submitted request is finished, or an error
+ * (EDGELORA_ERR_CACHE_FULL: nothing runs and every block is held). */
+int edgelora_batcher_next_batch(edgelora_batcher_t *batcher, int32_t capacity, int32_t *token_block,
+                                int32_t *token_slot, int32_t *n_tokens_out, int32_t *n_decode_out,
+                                int64_t *load_key, int32_t *load_block, int32_t *n_loads_out,
+                                double *now_out);
+/* The step handed out by the last edgelora_batcher_next_batch took `seconds`: the clock advances,
+ * prompts move on, the step that ends a prompt also yields the request's first token, every
+ * generating slot yields one token, finished requests leave their slot and release their adapter. */
+int edgelora_batcher_complete_step(edgelora_batcher_t *batcher, double seconds);
+/* The finished requests so far, in order of completion (any array may be NULL; capacity 0 only
+ * returns the count): ids, arrival / first-token / finish times, the adapter used and whether it
+ * was resident when chosen.  Section 5.1's metrics (throughput, average latency, average
+ * first-token latency, SLO attainment) and Section 3.3's hit rate follow from these. */
+int edgelora_batcher_finished(const edgelora_batcher_t *batcher, int32_t capacity, int64_t *request_id,
+                              double *arrival, double *first_token, double *finish, int64_t *adapter,
+                              int32_t *hit, int32_t *n_out);
 
 /* Scoring head of the adapter router (Section 3.2: a score s_j in [0, 1] per adapter j for a
  * prompt): scores_dev[b][j] = sigmoid(sum_k Wr_dev[j][k] * h_dev[b][k] + bias_dev[j]).

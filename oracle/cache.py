@@ -73,6 +73,14 @@ class AdapterCache:
             self.pins[key] = 1
         return block, False, evicted
 
+    def prefill(self, keys) -> List[int]:
+        """Section 4.2: before serving starts the cache is filled with (the caller's choice of)
+        adapters; the counters then start at zero."""
+        assert not self.slot and len(set(keys)) == len(keys) <= self.n_blocks
+        blocks = [self.acquire(int(k))[0] for k in keys]
+        self.hits = self.misses = 0
+        return blocks
+
     def release(self, key: int) -> None:
         assert self.pins.get(key, 0) > 0
         self.pins[key] -= 1

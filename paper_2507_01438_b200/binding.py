@@ -35,6 +35,8 @@ EXPORTS = (
     "edgelora_router_scores", "edgelora_plan_sync_status", "edgelora_pool_selftest_wait",
     "edgelora_siteset_create", "edgelora_siteset_destroy", "edgelora_siteset_run",
     "edgelora_siteset_run_host", "edgelora_siteset_plan",
+    "edgelora_cache_prefill", "edgelora_batcher_create", "edgelora_batcher_destroy", "edgelora_batcher_submit",
+    "edgelora_batcher_next_batch", "edgelora_batcher_complete_step", "edgelora_batcher_finished",
 )
 
 
@@ -78,10 +80,18 @@ def lib() -> ctypes.CDLL:
     L.edgelora_cache_destroy.argtypes = [vp]
     L.edgelora_cache_acquire.argtypes = [vp, i64, i32, cp(i32), cp(i32), cp(i64)]
     L.edgelora_cache_release.argtypes = [vp, i64]
+    L.edgelora_cache_prefill.argtypes = [vp, vp, i32, vp]
     L.edgelora_router_scores.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
     L.edgelora_cache_select.argtypes = [vp, vp, i32, i32, i32, cp(i64), cp(i32), cp(i32), cp(i64)]
     L.edgelora_cache_lookup.argtypes = [vp, i64, cp(i32)]
     L.edgelora_cache_stats.argtypes = [vp, cp(i64), cp(i64), cp(i64), cp(i32)]
+    f64 = ctypes.c_double
+    L.edgelora_batcher_create.argtypes = [i32, i32, i32, vp, cp(vp)]
+    L.edgelora_batcher_destroy.argtypes = [vp]
+    L.edgelora_batcher_submit.argtypes = [vp, i64, f64, i32, i32, vp]
+    L.edgelora_batcher_next_batch.argtypes = [vp, i32, vp, vp, cp(i32), cp(i32), vp, vp, cp(i32), cp(f64)]
+    L.edgelora_batcher_complete_step.argtypes = [vp, f64]
+    L.edgelora_batcher_finished.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, cp(i32)]
     L.edgelora_plan_create.argtypes = [i32, i32, cp(vp)]
     L.edgelora_plan_destroy.argtypes = [vp]
     L.edgelora_plan_build.argtypes = [vp, vp, i32, vp]
@@ -393,6 +403,14 @@ def edgelora_router_scores(Wr, bias, h, scores=None, stream=None):
     return scores
 
 
+def edgelora_cache_prefill(cache, keys) -> np.ndarray:
+    """Makes `keys` resident in an empty cache before serving starts; returns their blocks."""
+    k = np.ascontiguousarray(keys, dtype=np.int64)
+    blocks = np.zeros(len(k), dtype=np.int32)
+    _check(lib().edgelora_cache_prefill(cache, k.ctypes.data, len(k), blocks.ctypes.data), "cache_prefill")
+    return blocks
+
+
 def edgelora_cache_release(cache, key: int) -> None:
     _check(lib().edgelora_cache_release(cache, key), "cache_release")
 
@@ -446,3 +464,57 @@ class Pool:
             self.close()
         except Exception:
             pass
+
+
+def edgelora_batcher_create(n_slots: int, max_batch_tokens: int, top_k: int, cache) -> int:
+    out = ctypes.c_void_p()
+    _check(lib().edgelora_batcher_create(n_slots, max_batch_tokens, top_k, cache, ctypes.byref(out)),
+           "batcher_create")
+    return out.value
+
+
+def edgelora_batcher_destroy(batcher) -> None:
+    _check(lib().edgelora_batcher_destroy(batcher), "batcher_destroy")
+
+
+def edgelora_batcher_submit(batcher, request_id: int, arrival: float, in_len: int, out_len: int, candidates) -> None:
+    c = np.ascontiguousarray(candidates, dtype=np.int64)
+    _check(lib().edgelora_batcher_submit(batcher, request_id, float(arrival), int(in_len), int(out_len),
+                                         c.ctypes.data), "batcher_submit")
+
+
+def edgelora_batcher_next_batch(batcher, max_batch_tokens: int, n_slots: int):
+    """None when every request is finished, else a dict: now, token_block, token_slot, n_decode, loads."""
+    tb = np.zeros(max_batch_tokens, dtype=np.int32)
+    ts = np.zeros(max_batch_tokens, dtype=np.int32)
+    lk = np.zeros(n_slots, dtype=np.int64)
+    lb = np.zeros(n_slots, dtype=np.int32)
+    n, nd, nl, now = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32(), ctypes.c_double()
+    rc = lib().edgelora_batcher_next_batch(batcher, max_batch_tokens, tb.ctypes.data, ts.ctypes.data,
+                                           ctypes.byref(n), ctypes.byref(nd), lk.ctypes.data, lb.ctypes.data,
+                                           ctypes.byref(nl), ctypes.byref(now))
+    if rc < 0:
+        raise EdgeLoraError(rc, "batcher_next_batch")
+    if rc == 0:
+        return None
+    return {"now": now.value, "token_block": tb[:n.value], "token_slot": ts[:n.value], "n_decode": nd.value,
+            "loads": [(int(k), int(b)) for k, b in zip(lk[:nl.value], lb[:nl.value])]}
+
+
+def edgelora_batcher_complete_step(batcher, seconds: float) -> None:
+    _check(lib().edgelora_batcher_complete_step(batcher, float(seconds)), "batcher_complete_step")
+
+
+def edgelora_batcher_finished(batcher) -> dict:
+    n = ctypes.c_int32()
+    _check(lib().edgelora_batcher_finished(batcher, 0, None, None, None, None, None, None, ctypes.byref(n)),
+           "batcher_finished")
+    k = n.value
+    out = {"id": np.zeros(k, np.int64), "arrival": np.zeros(k), "first_token": np.zeros(k),
+           "finish": np.zeros(k), "adapter": np.zeros(k, np.int64), "hit": np.zeros(k, np.int32)}
+    if k:
+        _check(lib().edgelora_batcher_finished(batcher, k, out["id"].ctypes.data, out["arrival"].ctypes.data,
+                                               out["first_token"].ctypes.data, out["finish"].ctypes.data,
+                                               out["adapter"].ctypes.data, out["hit"].ctypes.data,
+                                               ctypes.byref(n)), "batcher_finished")
+    return out

@@ -160,6 +160,20 @@ int edgelora_cache_release(edgelora_cache_t *c, int64_t key) {
   return EDGELORA_OK;
 }
 
+int edgelora_cache_prefill(edgelora_cache_t *c, const int64_t *keys, int32_t n, int32_t *blocks_out) {
+  if (!c || !keys || n < 0 || n > c->n_blocks) return EDGELORA_ERR_INVALID_ARG;
+  if (!c->where.empty()) return EDGELORA_ERR_INVALID_ARG;  // only before serving starts
+  for (int32_t i = 0; i < n; ++i) {
+    if (keys[i] < 0 || c->where.count(keys[i])) return EDGELORA_ERR_INVALID_ARG;  // distinct keys
+    int32_t blk = -1;
+    const int rc = edgelora_cache_acquire(c, keys[i], 0, &blk, nullptr, nullptr);
+    if (rc != EDGELORA_OK) return rc;
+    if (blocks_out) blocks_out[i] = blk;
+  }
+  c->misses = 0;  // the counters describe the serving phase
+  return EDGELORA_OK;
+}
+
 int edgelora_cache_stats(const edgelora_cache_t *c, int64_t *hits, int64_t *misses, int64_t *evictions,
                          int32_t *resident) {
   if (!c) return EDGELORA_ERR_INVALID_ARG;

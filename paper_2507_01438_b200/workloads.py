@@ -214,3 +214,36 @@ def full_set_site(batch: FullSetBatch, layer: int, site: int, seed: int = 4,
     x = batch.x4096 if h_in == 4096 else batch.x14336
     return Workload(f"full_set_L{layer}_{name}", h_in, h_out, batch.n_slots, batch.max_rank,
                     W, x, batch.ids, ad, "prefill")
+
+
+@dataclass
+class Trace:
+    """A synthetic request trace (paper Section 5.1, "Workload trace")."""
+    arrival: np.ndarray      # float64 [n] seconds, ascending
+    in_len: np.ndarray       # int32 [n] prompt tokens
+    out_len: np.ndarray      # int32 [n] tokens to generate
+    candidates: np.ndarray   # int64 [n, k] the router's k adapters in descending order of confidence
+
+
+def serving_trace(seed: int = 5, n_adapters: int = 100, alpha: float = 1.0, rate: float = 0.5,
+                  cv: float = 1.0, duration: float = 300.0, in_range=(8, 256), out_range=(8, 128),
+                  top_k: int = 3) -> Trace:
+    """Gamma arrivals (shape 1/cv^2, scale cv^2/rate), adapter by the bounded power law with
+    exponent alpha, lengths uniform over the closed ranges.  The first candidate of a request is its
+    power-law adapter; the other k-1 are further distinct draws from the same law, standing in for
+    the rest of the router's top-k list."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    gaps = rng.gamma(shape=1.0 / (cv * cv), scale=(cv * cv) / rate, size=int(duration * rate * 4) + 16)
+    t = np.cumsum(gaps)
+    t = t[t < duration]
+    n = len(t)
+    w = np.arange(1, n_adapters + 1, dtype=np.float64) ** (-alpha)
+    w /= w.sum()
+    rank_to_adapter = rng.permutation(n_adapters)
+    k = min(top_k, n_adapters)
+    cand = np.zeros((n, k), dtype=np.int64)
+    for i in range(n):
+        cand[i] = rank_to_adapter[rng.choice(n_adapters, size=k, replace=False, p=w)]
+    in_len = rng.integers(in_range[0], in_range[1] + 1, size=n).astype(np.int32)
+    out_len = rng.integers(out_range[0], out_range[1] + 1, size=n).astype(np.int32)
+    return Trace(t.astype(np.float64), in_len, out_len, cand)

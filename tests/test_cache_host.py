@@ -107,3 +107,21 @@ def test_cache_aware_selection_matches_the_oracle(policy, k):
         assert B.edgelora_cache_stats(c)["hits"] == ref.hits
     finally:
         B.edgelora_cache_destroy(c)
+
+
+def test_prefill_before_serving():
+    # Section 4.2: the cache starts full of (the caller's choice of) adapters, counters at zero
+    keys = [41, 7, 19, 3]
+    o = AdapterCache(6)
+    c = B.edgelora_cache_create(6)
+    try:
+        assert B.edgelora_cache_prefill(c, keys).tolist() == o.prefill(keys) == [0, 1, 2, 3]
+        assert B.edgelora_cache_stats(c) == {"hits": 0, "misses": 0, "evictions": 0, "resident": 4}
+        for key in (7, 99, 41, 100, 101, 3):
+            assert B.edgelora_cache_acquire(c, key) == o.acquire(key)
+        st = B.edgelora_cache_stats(c)
+        assert (st["hits"], st["misses"], st["evictions"]) == (o.hits, o.misses, o.evictions) == (3, 3, 1)
+        with pytest.raises(B.EdgeLoraError):
+            B.edgelora_cache_prefill(c, [1])                       # not empty any more
+    finally:
+        B.edgelora_cache_destroy(c)
