@@ -123,6 +123,18 @@ int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool
 int edgelora_pool_load_slot(edgelora_pool_t *pool, int32_t slot, int32_t rank, float scale,
                             const uint16_t *A_host, const uint16_t *B_host);
 
+/* Section 5.1 ("All LoRA adapters are quantized using the Q8_0 format"): the same load for an
+ * adapter stored in Q8_0, the published block format of 34 bytes per 32 consecutive values of a
+ * row: a half-precision scale d (2 bytes, little endian) followed by 32 signed bytes q, value
+ * d * q.  A_q8 is [rank][h_in / 32] blocks (h_in % 32 == 0), B_q8 is [h_out][ceil(rank / 32)]
+ * blocks whose entries past `rank` are ignored.  The 8-bit form crosses to the device (about half
+ * the bytes of the bfloat16 form) and is converted there, on the pool's side stream, into the
+ * block's bfloat16 layout (each value rounded to nearest even), so the layer calls are unchanged.
+ * Ordering, ownership and errors as for edgelora_pool_load_slot; the first call allocates a
+ * device scratch for one adapter. */
+int edgelora_pool_load_slot_q8(edgelora_pool_t *pool, int32_t slot, int32_t rank, float scale,
+                               const void *A_q8, const void *B_q8);
+
 /* Section 4.2: an evicted adapter's block returns to the pool.  Marks `slot` empty
  * (asynchronously, ordered like a load). */
 int edgelora_pool_evict_slot(edgelora_pool_t *pool, int32_t slot);

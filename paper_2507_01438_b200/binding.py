@@ -35,7 +35,7 @@ EXPORTS = (
     "edgelora_router_scores", "edgelora_plan_sync_status", "edgelora_pool_selftest_wait",
     "edgelora_siteset_create", "edgelora_siteset_destroy", "edgelora_siteset_run",
     "edgelora_siteset_run_host", "edgelora_siteset_plan",
-    "edgelora_cache_prefill", "edgelora_batcher_create", "edgelora_batcher_destroy", "edgelora_batcher_submit",
+    "edgelora_cache_prefill", "edgelora_pool_load_slot_q8", "edgelora_batcher_create", "edgelora_batcher_destroy", "edgelora_batcher_submit",
     "edgelora_batcher_next_batch", "edgelora_batcher_complete_step", "edgelora_batcher_finished",
 )
 
@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
     L.edgelora_pool_create.argtypes = [cp(PoolConfig), cp(vp)]
     L.edgelora_pool_load_slot.argtypes = [vp, i32, i32, ctypes.c_float, vp, vp]
     L.edgelora_pool_evict_slot.argtypes = [vp, i32]
+    L.edgelora_pool_load_slot_q8.argtypes = [vp, i32, i32, ctypes.c_float, vp, vp]
     L.edgelora_pool_wait_loads.argtypes = [vp]
     L.edgelora_lora_linear.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     L.edgelora_lora_linear_host.argtypes = [vp, vp, vp, vp, i32, vp, vp]
@@ -163,6 +164,14 @@ def edgelora_pool_load_slot(pool, slot: int, rank: int, scale: float, A: np.ndar
     A = np.ascontiguousarray(A, dtype=np.uint16)
     B = np.ascontiguousarray(B, dtype=np.uint16)
     _check(lib().edgelora_pool_load_slot(pool, slot, rank, scale, A.ctypes.data, B.ctypes.data), "pool_load_slot")
+
+
+def edgelora_pool_load_slot_q8(pool, slot: int, rank: int, scale: float, A_q8: np.ndarray, B_q8: np.ndarray) -> None:
+    """A_q8: uint8 [rank, h_in / 32, 34], B_q8: uint8 [h_out, ceil(rank / 32), 34] (Q8_0 blocks, host)."""
+    A_q8 = np.ascontiguousarray(A_q8, dtype=np.uint8)
+    B_q8 = np.ascontiguousarray(B_q8, dtype=np.uint8)
+    _check(lib().edgelora_pool_load_slot_q8(pool, slot, rank, scale, A_q8.ctypes.data, B_q8.ctypes.data),
+           "pool_load_slot_q8")
 
 
 def edgelora_pool_evict_slot(pool, slot: int) -> None:

@@ -380,6 +380,7 @@ int edgelora_pool_destroy(edgelora_pool_t *p) {
   if (p->load_ev) cudaEventDestroy(p->load_ev);
   if (p->use_ev) cudaEventDestroy(p->use_ev);
   if (p->zws) cudaFree(p->zws);
+  if (p->q8_dev) cudaFree(p->q8_dev);
   if (p->group_counters) cudaFree(p->group_counters);
   for (auto &r : p->prof) {
     cudaEventDestroy(r.start);
@@ -455,6 +456,48 @@ int edgelora_pool_load_slot(edgelora_pool_t *p, int32_t slot, int32_t rank, floa
   if (rank < 1) return EDGELORA_ERR_INVALID_ARG;
   if (rank > p->cfg.max_rank) return EDGELORA_ERR_RANK_TOO_LARGE;
   return stage_and_copy(p, slot, rank, scale, A_host, B_host);
+}
+
+int edgelora_pool_load_slot_q8(edgelora_pool_t *p, int32_t slot, int32_t rank, float scale, const void *A_q8,
+                               const void *B_q8) {
+  if (!p || !A_q8 || !B_q8) return EDGELORA_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= p->cfg.n_slots) return EDGELORA_ERR_BAD_SLOT;
+  if (rank < 1 || (p->cfg.h_in % 32)) return EDGELORA_ERR_INVALID_ARG;
+  if (rank > p->cfg.max_rank) return EDGELORA_ERR_RANK_TOO_LARGE;
+  const int h_in = p->cfg.h_in, h_out = p->cfg.h_out, R = p->R_pad;
+  const size_t a_bytes = static_cast<size_t>(rank) * (h_in / 32) * 34;
+  const size_t b_bytes = static_cast<size_t>(h_out) * ((rank + 31) / 32) * 34;
+  const size_t b_off = (a_bytes + 15) & ~static_cast<size_t>(15);
+  const size_t scratch = static_cast<size_t>(p->cfg.max_rank) * (h_in / 32) * 34 + 16 +
+                         static_cast<size_t>(h_out) * ((p->cfg.max_rank + 31) / 32) * 34;
+  if (!p->q8_dev) CUDA_TRY(cudaMalloc(&p->q8_dev, scratch));
+  StagingBuf &sb = p->staging[p->next_staging];
+  p->next_staging = (p->next_staging + 1) % kStagingBuffers;
+  if (sb.in_flight) {
+    CUDA_TRY(cudaEventSynchronize(sb.done));
+    sb.in_flight = false;
+  }
+  // the 8-bit form is smaller than the block the staging buffer was sized for
+  memcpy(sb.host, A_q8, a_bytes);
+  memcpy(sb.host + b_off, B_q8, b_bytes);
+  SlotRow *srow = reinterpret_cast<SlotRow *>(sb.host + (p->a_block + p->b_block) * 2);
+  SlotRow &mirror = p->slots_host[slot];
+  mirror.rank = rank;
+  mirror.scale = scale;
+  mirror.generation += 1;
+  *srow = mirror;
+  if (p->use_recorded) CUDA_TRY(cudaStreamWaitEvent(p->side, p->use_ev, 0));
+  // (the scratch is reused by every load: the copies and conversions of one pool run in order on
+  // its side stream)
+  CUDA_TRY(cudaMemcpyAsync(p->q8_dev, sb.host, b_off + b_bytes, cudaMemcpyHostToDevice, p->side));
+  CUDA_TRY(launch_q8_to_block(p->q8_dev, p->q8_dev + b_off, p->A_pool + p->a_block * slot,
+                              p->B_pool + p->b_block * slot, rank, R, h_in, h_out, p->sms, p->side));
+  CUDA_TRY(cudaMemcpyAsync(p->slots_dev + slot, srow, sizeof(SlotRow), cudaMemcpyHostToDevice, p->side));
+  CUDA_TRY(cudaEventRecord(sb.done, p->side));
+  sb.in_flight = true;
+  CUDA_TRY(cudaEventRecord(p->load_ev, p->side));
+  p->load_seq += 1;
+  return EDGELORA_OK;
 }
 
 int edgelora_pool_evict_slot(edgelora_pool_t *p, int32_t slot) {

@@ -60,6 +60,7 @@ struct edgelora_pool {
   int R_pad = 0, device = 0, sms = 0;
   bool owns_arena = false;
   uint8_t *arena = nullptr;
+  uint8_t *q8_dev = nullptr;  // device scratch for one adapter in Q8_0 form (first use of load_slot_q8)
   uint16_t *A_pool = nullptr, *B_pool = nullptr;
   size_t a_block = 0, b_block = 0;  // elements per slot
   SlotRow *slots_dev = nullptr;

@@ -247,3 +247,25 @@ def serving_trace(seed: int = 5, n_adapters: int = 100, alpha: float = 1.0, rate
     in_len = rng.integers(in_range[0], in_range[1] + 1, size=n).astype(np.int32)
     out_len = rng.integers(out_range[0], out_range[1] + 1, size=n).astype(np.int32)
     return Trace(t.astype(np.float64), in_len, out_len, cand)
+
+
+def q8_0_encode(values: np.ndarray) -> np.ndarray:
+    """Packs rows of float32 values into Q8_0 blocks (input preparation for adapters that arrive in
+    the paper's storage format): per 32 values d = max|v| / 127 as half precision, q = round(v / d).
+    Rows are padded with zeros to a multiple of 32.  Returns uint8 [..., n_blocks, 34]."""
+    v = np.asarray(values, dtype=np.float32)
+    n = v.shape[-1]
+    nb = (n + 31) // 32
+    pad = np.zeros(v.shape[:-1] + (nb * 32,), dtype=np.float32)
+    pad[..., :n] = v
+    blk = pad.reshape(v.shape[:-1] + (nb, 32))
+    d = (np.abs(blk).max(axis=-1) / np.float32(127.0)).astype(np.float16)
+    df = d.astype(np.float32)
+    q = np.zeros_like(blk)
+    nz = df > 0
+    q[nz] = np.rint(blk[nz] / df[nz][..., None])
+    q = np.clip(q, -127, 127).astype(np.int8)
+    out = np.zeros(v.shape[:-1] + (nb, 34), dtype=np.uint8)
+    out[..., 0:2] = np.ascontiguousarray(d.astype("<f2"))[..., None].view(np.uint8)   # little endian
+    out[..., 2:] = q.view(np.uint8)
+    return out

@@ -28,7 +28,7 @@ def lib():
 def declared_symbols():
     text = open(HEADER).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(edgelora_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(edgelora_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_header_and_binding_agree(lib):
