@@ -317,8 +317,10 @@ __device__ __forceinline__ bool gather_pass_copies(const GemmParams &jp, const T
 }
 
 // kMinBlocks = 2 caps the registers so that two CTAs share an SM (small decode tiles); with 1 the
-// builder keeps both of its z rows in registers without spilling.
-template <int kMinBlocks>
+// builder keeps both of its z rows in registers without spilling.  kShrink = false compiles the
+// kernel without the shrink jobs (segment and gather tiles, second job) and without the staged y
+// stores: the decode-mode launches, which need none of them, keep a smaller kernel.
+template <int kMinBlocks, bool kShrink>
 __global__ void __launch_bounds__(kGemmThreads, kMinBlocks)
 lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_constant__ CUtensorMap tmap_c,
                  const __grid_constant__ CUtensorMap tmap_b, const GemmParams p,
@@ -336,7 +338,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   // persistent grid, after the first job's tiles.  Its tile list comes from a plan on the device, so
   // the host passes an upper bound (p2.n_mtiles) and every role stops at the true count, which it
   // reads after the dependency wait.  Its N tile is never wider than the first job's.
-  const bool has2 = p2.mode == kModeSgmv;
+  const bool has2 = kShrink && p2.mode == kModeSgmv;
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + static_cast<size_t>(p.stages) * stage_bytes);
   uint64_t *full_bar = bars;                      // [stages]  TMA -> MMA
   uint64_t *empty_bar = bars + kMaxStages;        // [stages]  MMA -> TMA
@@ -375,8 +377,8 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       ptx::prefetch_tensormap(&tmap_c2);
       if (p2.gather) ptx::prefetch_tensormap(&tmap_g2);
     }
-    if (p.mode == kModeSgmv && p.gather) ptx::prefetch_tensormap(&tmap_b);
-    if (p.y_tma) ptx::prefetch_tensormap(&tmap_y);
+    if (kShrink && p.mode == kModeSgmv && p.gather) ptx::prefetch_tensormap(&tmap_b);
+    if (kShrink && p.y_tma) ptx::prefetch_tensormap(&tmap_y);
     for (int s = 0; s < p.stages; ++s) {
       ptx::mbar_init(&full_bar[s], 1);
       ptx::mbar_init(&empty_bar[s], 1);
@@ -447,7 +449,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         const GemmParams &jp = second ? p2 : p;
         const CUtensorMap *mr = second ? &tmap_r2 : &tmap_r, *mc = second ? &tmap_c2 : &tmap_c;
         const TileCoord tc = tile_coord(jp, local);
-        if (tc.kind == 1) {
+        if (kShrink && tc.kind == 1) {
           // gather tile: this warp is part 0 of the copies (see gather_pass_copies)
           const CUtensorMap *mg = second ? &tmap_g2 : &tmap_b;
           for (int32_t t0 = 0; ok && t0 < tc.ntok; t0 += jp.gN)
@@ -532,7 +534,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         uint32_t acc = 0, tmem_d = tmem_base;
         for (int32_t pass = 0; ok && pass < n_pass; ++pass, ++it) {
           // UMMA N: the job's N tile, or for a gather pass its token count rounded up to 16
-          const uint32_t n_cols = tc.kind == 1
+          const uint32_t n_cols = (kShrink && tc.kind == 1)
                                       ? static_cast<uint32_t>((min(jp.gN, tc.ntok - pass * jp.gN) + 15) & ~15)
                                       : static_cast<uint32_t>(jp.BN);
           const uint32_t idesc = ptx::umma_idesc_bf16(kTileM, n_cols);
@@ -549,7 +551,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
               ok = false;
               break;
             }
-            if (tc.kind == 1) {  // the other parts of the tile's copies have been through this stage
+            if (kShrink && tc.kind == 1) {  // the other parts of the tile's copies have been through this stage
               if (!ptx::mbar_wait(&zfull_bar[stage], (zphase >> stage) & 1u, wl)) {
                 ok = false;
                 break;
@@ -573,10 +575,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
           }
           if (!ok) break;
           // a gather pass is complete here; other tiles go on with their LoRA K blocks below
-          if (tc.kind == 1) ptx::umma_commit(&tfull_bar[acc]);
+          if (kShrink && tc.kind == 1) ptx::umma_commit(&tfull_bar[acc]);
         }
         if (!ok) break;
-        if (tc.kind == 1) continue;
+        if (kShrink && tc.kind == 1) continue;
         const uint32_t idesc = ptx::umma_idesc_bf16(kTileM, static_cast<uint32_t>(jp.BN));
         if (!ok) break;
         if (has_lora && !second) {
@@ -668,7 +670,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       if (second && (local = second_job_tile(tile)) < 0) break;
       const GemmParams &jp = second ? p2 : p;
       const TileCoord tc = tile_coord(jp, local);
-      if (tc.kind == 1) {
+      if (kShrink && tc.kind == 1) {
         // ---- gather tile: accumulator row m = (group m / R_pad of the tile, rank row m % R_pad),
         // column c = token perm_short[tok0 + pass * gN + c].  This thread writes z of its rank row
         // for the tokens of its group, scaled by s_a, into the partial plane of the tile's K split.
@@ -814,7 +816,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
             v[i + 16] = 0.f;
           }
         }
-        if (jp.mode == kModePrefill && jp.y_tma) {
+        if (kShrink && jp.mode == kModePrefill && jp.y_tma) {
           // row = token, columns = output features row_c + c0 + [0, 32).  The warp's 32 rows x 64
           // columns go to its shared-memory stage as bf16 (rows of 128 bytes, 16-byte chunks
           // swizzled by the row so that the lanes' stores spread over the banks) and leave with one
@@ -895,7 +897,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       *abort_flag = 1;
       atomicOr(p.status, EDGELORA_STATUS_TIMEOUT);
     }
-  } else if (has_lora || has2 || (p.mode == kModeSgmv && p.gather)) {
+  } else if (has_lora || has2 || (kShrink && p.mode == kModeSgmv && p.gather)) {
     // ------------------------------------------------------------ z operand builder (warps 6..9)
     // (and, during gather tiles, parts 1..4 of the tile's copies)
     const int btid = threadIdx.x - 192;  // 0..127
@@ -982,13 +984,13 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       if (btid == 0) ptx::mbar_arrive(lg_bar);
     }
     for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
-      if (tile >= n_tiles0) {  // a tile of the second job: no LoRA blocks
+      if (kShrink && tile >= n_tiles0) {  // a tile of the second job: no LoRA blocks
         const int32_t local = second_job_tile(tile);
         if (local < 0) break;
         ok = shrink_tile(p2, local, &tmap_c2, &tmap_g2);
         continue;
       }
-      if (p.mode == kModeSgmv) {  // the first job is a shrink job
+      if (kShrink && p.mode == kModeSgmv) {  // the first job is a shrink job
         ok = shrink_tile(p, tile, &tmap_c, &tmap_b);
         continue;
       }
@@ -1216,7 +1218,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     }
   }
 
-  if (p.y_tma && warp >= 2 && warp < 6 && lane == 0) ptx::bulk_wait_group0();  // this warp's y stores
+  if (kShrink && p.y_tma && warp >= 2 && warp < 6 && lane == 0) ptx::bulk_wait_group0();  // this warp's y stores
   ptx::tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) {
@@ -1233,11 +1235,13 @@ static GemmParams no_job() {
 }
 
 cudaError_t gemm_set_smem_limit(size_t smem_bytes) {
-  cudaError_t e = cudaFuncSetAttribute(lora_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem_bytes));
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(lora_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              static_cast<int>(smem_bytes));
+  cudaError_t e = cudaSuccess;
+  const int bytes = static_cast<int>(smem_bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(lora_gemm_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(lora_gemm_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(lora_gemm_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(lora_gemm_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  return e;
 }
 
 cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col,
@@ -1257,11 +1261,14 @@ cudaError_t launch_gemm2(const CUtensorMap &tmap_row, const CUtensorMap &tmap_co
                          const CUtensorMap *tmap_y) {
   const CUtensorMap &my = tmap_y ? *tmap_y : tmap_row;  // unused unless p.y_tma
   const int cluster = (p.mode == kModeDecode && p.splits > 1) ? p.splits : 1;
-  if (smem_bytes * 2 <= 225 * 1024 && p.BN <= 128 && p.acc_cols <= 128)  // two CTAs fit an SM
-    return launch_ex(lora_gemm_kernel<2>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster,
-                     tmap_row, tmap_col, tmap_b, p, tmap_row2, tmap_col2, tmap_g2, p2, my);
-  return launch_ex(lora_gemm_kernel<1>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster,
-                   tmap_row, tmap_col, tmap_b, p, tmap_row2, tmap_col2, tmap_g2, p2, my);
+  const bool two = smem_bytes * 2 <= 225 * 1024 && p.BN <= 128 && p.acc_cols <= 128;  // two CTAs fit an SM
+  const bool lean = p.mode == kModeDecode && p2.mode != kModeSgmv;                    // no shrink job, plain y stores
+#define EDGELORA_LAUNCH(MB, SH)                                                                                \
+  launch_ex(lora_gemm_kernel<MB, SH>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster, tmap_row, \
+            tmap_col, tmap_b, p, tmap_row2, tmap_col2, tmap_g2, p2, my)
+  if (two) return lean ? EDGELORA_LAUNCH(2, false) : EDGELORA_LAUNCH(2, true);
+  return lean ? EDGELORA_LAUNCH(1, false) : EDGELORA_LAUNCH(1, true);
+#undef EDGELORA_LAUNCH
 }
 
 }  // namespace edgelora
