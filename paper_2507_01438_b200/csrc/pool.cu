@@ -641,7 +641,7 @@ int edgelora_pool_selftest_wait(edgelora_pool_t *p, void *stream) {
 namespace edgelora {
 int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_dev, const void *W_dev,
                      const void *x_dev, int32_t T, void *y_dev, cudaStream_t stream, bool skip_shrink,
-                     const NextShrink *next) {
+                     const NextShrink *next, bool independent) {
   if (!p || !plan || T < 0) return EDGELORA_ERR_INVALID_ARG;
   if (T == 0) return EDGELORA_OK;
   if (!W_dev || !x_dev || !y_dev) return EDGELORA_ERR_INVALID_ARG;
@@ -654,7 +654,9 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
   const int h_in = p->cfg.h_in, h_out = p->cfg.h_out, R = p->R_pad;
   const bool capturing = stream_capturing(stream);
   const bool pdl = p->opt_pdl >= 1 && !p->opt_profile;        // between the kernels of this call
-  const bool pdl_first = p->opt_pdl >= 2 && !p->opt_profile;  // first kernel vs earlier stream work
+  // first kernel vs earlier stream work: when the pool's option says so, or when the caller (a set
+  // of sites) knows that this call does not consume what the call before it produces
+  const bool pdl_first = (p->opt_pdl >= 2 || (independent && p->opt_pdl >= 1)) && !p->opt_profile;
   const uint16_t *x = static_cast<const uint16_t *>(x_dev);
   int launches = 0;
 

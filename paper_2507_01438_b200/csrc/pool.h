@@ -111,9 +111,11 @@ struct NextShrink {
 };
 
 // The layer (see pool.cu).  `skip_shrink`: this site's shrinks were already issued (as part of the
-// previous site's launches); `next`: issue the next site's shrinks along with this site's kernels.
+// previous site's launches); `next`: issue the next site's shrinks along with this site's kernels;
+// `independent`: the call reads nothing the previous call on the stream writes, so its first
+// kernel may start under that call's tail.
 int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_dev, const void *W_dev,
                      const void *x_dev, int32_t T, void *y_dev, cudaStream_t stream,
-                     bool skip_shrink = false, const NextShrink *next = nullptr);
+                     bool skip_shrink = false, const NextShrink *next = nullptr, bool independent = false);
 
 }  // namespace edgelora

@@ -55,8 +55,10 @@ int run_sites(edgelora_siteset *s, const void *const *x_dev, const int32_t *ids_
       next.pool = s->pools[i + 1];
       next.x = static_cast<const uint16_t *>(x_dev[s->input_of[i + 1]]);
     }
+    // (decode-sized batches: the sites are independent given their inputs and results, so a
+    // site's shrink may start under the previous site's base product)
     rc = lora_linear_impl(s->pools[i], s->plan, nullptr, s->W[i], x_dev[s->input_of[i]], T, y_dev[i], stream,
-                          pipelined && i > 0, next.pool ? &next : nullptr);
+                          pipelined && i > 0, next.pool ? &next : nullptr, !pipelined && i > 0);
     if (rc != EDGELORA_OK) return rc;
   }
   if (pipelined && !capturing(stream)) {  // slot loads issued later wait for this step
