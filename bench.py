@@ -445,6 +445,39 @@ def bench_site(name, ctx, steps=None, warmup=None, pdl=None, graph=True, cpu_bud
     single_call = {"ms_median": 0.5 * (lat[19] + lat[20]), "ms_best": lat[0], "calls": 40,
                    "note": "one un-graphed call, launch to stream synchronise, wall clock, cold rotation"}
 
+    # ---- adapter swaps beside the layer (Section 3.3 / 4.2: a missing adapter is loaded into a free
+    # block while serving goes on): plain launches with 0, 1 and 4 loads per step into blocks the
+    # batch does not use, from page-locked host memory, copies on the pool's side stream
+    swap = None
+    if decode_like and w.n_slots <= 64:
+        spare_pools = []
+        for r in range(n_rep):
+            sp = B.Pool(w.h_in, w.h_out, w.n_slots + 4, w.max_rank, max_tokens=w.T)
+            sp.load_all(w.adapters)
+            spare_pools.append(sp)
+        ad0 = w.adapters[sorted(w.adapters)[0]]
+        Rp = 16 if w.max_rank <= 16 else (32 if w.max_rank <= 32 else 64)
+        if ad0.rank == Rp:
+            pa = torch.from_numpy(ad0.A.view(np.int16).copy()).pin_memory()
+            pb = torch.from_numpy(ad0.B.view(np.int16).copy()).pin_memory()
+            swap = {"adapter_bytes": int(ad0.A.nbytes + ad0.B.nbytes), "per_step": {}}
+            for n_sw in (0, 1, 4):
+                k_sw = 2000
+                for timed_pass in (False, True):
+                    torch.cuda.synchronize()
+                    t0 = time.perf_counter()
+                    for i in range(k_sw if timed_pass else 50):
+                        r = i % n_rep
+                        for j in range(n_sw):
+                            B.edgelora_pool_load_slot_pinned(spare_pools[r].handle, w.n_slots + j, Rp, ad0.scale, pa, pb)
+                        B.edgelora_lora_linear(spare_pools[r].handle, Ws[r], x, ids, ys[r], stream)
+                    torch.cuda.synchronize()
+                    dt = time.perf_counter() - t0
+                swap["per_step"][str(n_sw)] = {"us_per_step_wall": 1e6 * dt / k_sw, "swaps_per_s": n_sw * k_sw / dt,
+                                               "adapter_gb_per_s": n_sw * k_sw * swap["adapter_bytes"] / dt / 1e9}
+        for sp in spare_pools:
+            sp.close()
+
     # ---- end to end through the pipelined host-buffer entry point: every step copies x and the ids
     # from page-locked host memory and reads y back into page-locked host memory; the library
     # overlaps the copies of neighbouring steps with the layer (two sets of device mirrors per pool)
@@ -542,7 +575,7 @@ def bench_site(name, ctx, steps=None, warmup=None, pdl=None, graph=True, cpu_bud
         "gpu_launches": int(info["launches"] * steps),
         "iterations": iterations, "step_work": step_work, "step_roofline_frac": step_frac,
         "step_roofline_frac_of_nominal": step_frac_nominal, "roofline": roof, "e2e": e2e,
-        "variants": variants, "warm_l2": warm, "single_call_latency": single_call,
+        "variants": variants, "warm_l2": warm, "single_call_latency": single_call, "adapter_swaps": swap,
         "kernel_ms_profiled": {k: v for k, v in kt.items() if v["launches"]},
     }
     if ctx["rank"] == 0 and world == 1 and cpu_budget > 0:
@@ -921,7 +954,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic"}
     for k in ("config", "launch_info", "clocks", "e2e", "gpu_launches", "roofline", "step_work", "step_roofline_frac",
               "step_roofline_frac_of_nominal", "iterations", "variants", "warm_l2", "single_call_latency",
-              "kernel_ms_profiled", "cpu_baseline"):
+              "kernel_ms_profiled", "adapter_swaps", "cpu_baseline"):
         if k in head:
             line[k] = head[k]
     if per_config:

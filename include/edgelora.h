@@ -123,6 +123,16 @@ int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool
 int edgelora_pool_load_slot(edgelora_pool_t *pool, int32_t slot, int32_t rank, float scale,
                             const uint16_t *A_host, const uint16_t *B_host);
 
+/* The same load without the copy into the library's staging buffer, for adapters the caller keeps in
+ * page-locked host memory in the block's own layout (Section 3.3: adapters that are not resident
+ * wait in host memory; a server that pins that memory once swaps at the speed of the link instead
+ * of the speed of a host memcpy).  rank must equal the pool's padded rank (16, 32 or 64), A_pinned
+ * is [rank][h_in], B_pinned [h_out][rank].  Unlike edgelora_pool_load_slot the buffers must stay
+ * valid and unchanged until edgelora_pool_wait_loads (or a later layer call's completion).
+ * EDGELORA_ERR_INVALID_ARG when the memory is not page-locked or the rank is not the padded one. */
+int edgelora_pool_load_slot_pinned(edgelora_pool_t *pool, int32_t slot, int32_t rank, float scale,
+                                   const uint16_t *A_pinned, const uint16_t *B_pinned);
+
 /* Section 5.1 ("All LoRA adapters are quantized using the Q8_0 format"): the same load for an
  * adapter stored in Q8_0, the published block format of 34 bytes per 32 consecutive values of a
  * row: a half-precision scale d (2 bytes, little endian) followed by 32 signed bytes q, value

@@ -35,7 +35,7 @@ EXPORTS = (
     "edgelora_router_scores", "edgelora_plan_sync_status", "edgelora_pool_selftest_wait",
     "edgelora_siteset_create", "edgelora_siteset_destroy", "edgelora_siteset_run",
     "edgelora_siteset_run_host", "edgelora_siteset_plan",
-    "edgelora_cache_prefill", "edgelora_pool_load_slot_q8", "edgelora_batcher_create", "edgelora_batcher_destroy", "edgelora_batcher_submit",
+    "edgelora_cache_prefill", "edgelora_pool_load_slot_q8", "edgelora_pool_load_slot_pinned", "edgelora_batcher_create", "edgelora_batcher_destroy", "edgelora_batcher_submit",
     "edgelora_batcher_next_batch", "edgelora_batcher_complete_step", "edgelora_batcher_finished",
 )
 
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
     L.edgelora_pool_load_slot.argtypes = [vp, i32, i32, ctypes.c_float, vp, vp]
     L.edgelora_pool_evict_slot.argtypes = [vp, i32]
     L.edgelora_pool_load_slot_q8.argtypes = [vp, i32, i32, ctypes.c_float, vp, vp]
+    L.edgelora_pool_load_slot_pinned.argtypes = [vp, i32, i32, ctypes.c_float, vp, vp]
     L.edgelora_pool_wait_loads.argtypes = [vp]
     L.edgelora_lora_linear.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     L.edgelora_lora_linear_host.argtypes = [vp, vp, vp, vp, i32, vp, vp]
@@ -164,6 +165,12 @@ def edgelora_pool_load_slot(pool, slot: int, rank: int, scale: float, A: np.ndar
     A = np.ascontiguousarray(A, dtype=np.uint16)
     B = np.ascontiguousarray(B, dtype=np.uint16)
     _check(lib().edgelora_pool_load_slot(pool, slot, rank, scale, A.ctypes.data, B.ctypes.data), "pool_load_slot")
+
+
+def edgelora_pool_load_slot_pinned(pool, slot: int, rank: int, scale: float, A_pinned, B_pinned) -> int:
+    """A_pinned / B_pinned: page-locked CPU tensors (int16 view of bf16) in the block layout; they
+    must stay alive until the load has landed.  Returns the C return code."""
+    return lib().edgelora_pool_load_slot_pinned(pool, slot, rank, scale, A_pinned.data_ptr(), B_pinned.data_ptr())
 
 
 def edgelora_pool_load_slot_q8(pool, slot: int, rank: int, scale: float, A_q8: np.ndarray, B_q8: np.ndarray) -> None:

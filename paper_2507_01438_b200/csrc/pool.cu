@@ -458,6 +458,41 @@ int edgelora_pool_load_slot(edgelora_pool_t *p, int32_t slot, int32_t rank, floa
   return stage_and_copy(p, slot, rank, scale, A_host, B_host);
 }
 
+int edgelora_pool_load_slot_pinned(edgelora_pool_t *p, int32_t slot, int32_t rank, float scale,
+                                   const uint16_t *A_pinned, const uint16_t *B_pinned) {
+  if (!p || !A_pinned || !B_pinned) return EDGELORA_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= p->cfg.n_slots) return EDGELORA_ERR_BAD_SLOT;
+  if (rank != p->R_pad) return EDGELORA_ERR_INVALID_ARG;  // already in the block's layout: nothing to pad
+  cudaPointerAttributes at{};
+  if (cudaPointerGetAttributes(&at, A_pinned) != cudaSuccess || at.type != cudaMemoryTypeHost ||
+      cudaPointerGetAttributes(&at, B_pinned) != cudaSuccess || at.type != cudaMemoryTypeHost) {
+    cudaGetLastError();
+    return EDGELORA_ERR_INVALID_ARG;  // not page-locked: use edgelora_pool_load_slot
+  }
+  // the slot row still goes through a staging buffer (16 bytes the library owns)
+  StagingBuf &sb = p->staging[p->next_staging];
+  p->next_staging = (p->next_staging + 1) % kStagingBuffers;
+  if (sb.in_flight) {
+    CUDA_TRY(cudaEventSynchronize(sb.done));
+    sb.in_flight = false;
+  }
+  SlotRow *srow = reinterpret_cast<SlotRow *>(sb.host + (p->a_block + p->b_block) * 2);
+  SlotRow &mirror = p->slots_host[slot];
+  mirror.rank = rank;
+  mirror.scale = scale;
+  mirror.generation += 1;
+  *srow = mirror;
+  if (p->use_recorded) CUDA_TRY(cudaStreamWaitEvent(p->side, p->use_ev, 0));
+  CUDA_TRY(cudaMemcpyAsync(p->A_pool + p->a_block * slot, A_pinned, p->a_block * 2, cudaMemcpyHostToDevice, p->side));
+  CUDA_TRY(cudaMemcpyAsync(p->B_pool + p->b_block * slot, B_pinned, p->b_block * 2, cudaMemcpyHostToDevice, p->side));
+  CUDA_TRY(cudaMemcpyAsync(p->slots_dev + slot, srow, sizeof(SlotRow), cudaMemcpyHostToDevice, p->side));
+  CUDA_TRY(cudaEventRecord(sb.done, p->side));
+  sb.in_flight = true;
+  CUDA_TRY(cudaEventRecord(p->load_ev, p->side));
+  p->load_seq += 1;
+  return EDGELORA_OK;
+}
+
 int edgelora_pool_load_slot_q8(edgelora_pool_t *p, int32_t slot, int32_t rank, float scale, const void *A_q8,
                                const void *B_q8) {
   if (!p || !A_q8 || !B_q8) return EDGELORA_ERR_INVALID_ARG;

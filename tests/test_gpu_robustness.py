@@ -148,3 +148,24 @@ def test_status_of_a_plan_built_on_its_own():
         assert got["ids_valid"].tolist() == [0, 1, -1, -1, 2, -1, 1]
     finally:
         B.edgelora_plan_destroy(plan)
+
+
+def test_load_from_page_locked_memory():
+    import torch
+    w = random_workload(83, 50, 256, 384, ranks=[16, 16, 16], max_rank=16)
+    pool = B.Pool(w.h_in, w.h_out, w.n_slots, w.max_rank, max_tokens=64)
+    try:
+        keep = []
+        for a, ad in w.adapters.items():
+            A = torch.from_numpy(ad.A.view(np.int16).copy()).pin_memory()
+            Bm = torch.from_numpy(ad.B.view(np.int16).copy()).pin_memory()
+            keep += [A, Bm]
+            assert B.edgelora_pool_load_slot_pinned(pool.handle, a, 16, ad.scale, A, Bm) == B.OK
+        y = pool.linear(to_dev_bf16(w.W), to_dev_bf16(w.x), torch.from_numpy(w.ids).cuda())
+        assert pool.status() == (0, 0)
+        assert_parity(from_dev_bf16(y), oracle_of(w), "adapters loaded from page-locked memory")
+        pageable = torch.from_numpy(w.adapters[0].A.view(np.int16).copy())
+        assert B.edgelora_pool_load_slot_pinned(pool.handle, 0, 16, 1.0, pageable, keep[1]) == B.ERR_INVALID_ARG
+        assert B.edgelora_pool_load_slot_pinned(pool.handle, 0, 8, 1.0, keep[0], keep[1]) == B.ERR_INVALID_ARG
+    finally:
+        pool.close()
