@@ -48,6 +48,11 @@ SITE_WORKLOADS = {
     "down_proj_many_tenant": (lambda: wl.down_proj_many_tenant(), "hbm",
                               "configs[3]: down_proj 14336->4096, 1000 adapters r64, T=256 Zipf(1.1), 10% base-only"),
     "tiny": (lambda: wl.tiny(), "hbm", "configs[0]: 256->256, 4 adapters r8, T=16"),
+    # next row N2: the same batch over a pool that keeps A in Q8_0 (paper Section 5.1); only the
+    # adapters the batch touches are drawn and loaded, the other slots of the 1000 stay empty
+    "down_proj_many_tenant_q8": (lambda: wl.down_proj_many_tenant(only_used=True), "hbm",
+                                 "configs[3] with Q8_0 adapters: down_proj 14336->4096, pool of 1000 slots keeping A "
+                                 "in Q8_0, rank 64, T=256 Zipf(1.1), 10% base-only"),
     # smaller resident pool, same layer and batch recipe: sized for multi-pass profiler captures
     "down_proj_200_tenants": (lambda: wl.down_proj_many_tenant(n_adapters=200), "hbm",
                               "profiling-size variant of configs[3]: down_proj 14336->4096, 200 adapters r64, T=256"),
@@ -273,19 +278,32 @@ def bench_site(name, ctx, steps=None, warmup=None, pdl=None, graph=True, cpu_bud
     world, barrier, sampler = ctx["world"], ctx["barrier"], ctx["sampler"]
     builder, bound, desc = SITE_WORKLOADS[name]
     decode_like = bound == "hbm"
+    q8 = name.endswith("_q8")
     w = builder()
     warmup = max(3, warmup if warmup is not None else (50 if decode_like else 5))
 
     # ---- resident state: n_rep replicas of (W, pool) so that every step reads cold data from HBM
     ws_bytes = w.algorithmic_bytes()
+    q8_blocks = {}
+    if q8:   # A in Q8_0: 34 bytes per 32 values instead of 64
+        ws_bytes -= sum(w.adapters[a].rank * w.h_in * 2 - w.adapters[a].rank * (w.h_in // 32) * 34
+                        for a in w.distinct_adapters())
+        cpu_budget = 0.0
+        for a, ad in w.adapters.items():
+            q8_blocks[a] = (wl.q8_0_encode(wl.bf16_bits_to_f32(ad.A)), wl.q8_0_encode(wl.bf16_bits_to_f32(ad.B)))
     n_rep = 2 if not decode_like else max(2, int(np.ceil(3 * L2_BYTES / ws_bytes)))
     pdl_mode = pdl if pdl is not None else 1            # the library's default: calls may depend on each other
     to_bf16 = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
     Ws, pools = [], []
     for r in range(n_rep):
         Ws.append(to_bf16(w.W) if r == 0 else Ws[0].clone())
-        pool = B.Pool(w.h_in, w.h_out, w.n_slots, w.max_rank, max_tokens=w.T)
-        pool.load_all(w.adapters)
+        pool = B.Pool(w.h_in, w.h_out, w.n_slots, w.max_rank, max_tokens=w.T, flags=B.FLAG_A_Q8 if q8 else 0)
+        if q8:
+            for a, ad in w.adapters.items():
+                B.edgelora_pool_load_slot_q8(pool.handle, a, ad.rank, ad.scale, q8_blocks[a][0], q8_blocks[a][1])
+            B.edgelora_pool_wait_loads(pool.handle)
+        else:
+            pool.load_all(w.adapters)
         B.edgelora_pool_set_option(pool.handle, B.OPT_PDL, pdl_mode)
         pools.append(pool)
     x = to_bf16(w.x)
@@ -449,7 +467,7 @@ def bench_site(name, ctx, steps=None, warmup=None, pdl=None, graph=True, cpu_bud
     # block while serving goes on): plain launches with 0, 1 and 4 loads per step into blocks the
     # batch does not use, from page-locked host memory, copies on the pool's side stream
     swap = None
-    if decode_like and w.n_slots <= 64:
+    if decode_like and w.n_slots <= 64 and not q8:
         spare_pools = []
         for r in range(n_rep):
             sp = B.Pool(w.h_in, w.h_out, w.n_slots + 4, w.max_rank, max_tokens=w.T)

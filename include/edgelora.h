@@ -75,6 +75,12 @@ typedef struct {
 } edgelora_pool_config;
 
 #define EDGELORA_FLAG_NONE 0u
+/* The pool keeps every adapter's A in Q8_0 in device memory (Section 5.1: adapters are stored in
+ * Q8_0), 34/64 of the bfloat16 bytes, which are the bytes that bound a many-adapter decode step; B
+ * stays bfloat16.  Such a pool needs h_in % 256 == 0, takes adapters through
+ * edgelora_pool_load_slot_q8 only, and serves decode batches (T <= 256) only: the shrink kernel
+ * decodes the blocks as it streams them.  Other calls return EDGELORA_ERR_INVALID_ARG. */
+#define EDGELORA_FLAG_A_Q8 1u
 
 /* Options for edgelora_pool_set_option(). */
 #define EDGELORA_OPT_REGIME 1    /* 0 auto (T <= 256 => decode), 1 force decode, 2 force prefill */

@@ -150,9 +150,12 @@ def edgelora_pool_bytes_required(h_in, h_out, n_slots, max_rank) -> int:
     return out.value
 
 
-def edgelora_pool_create(h_in, h_out, n_slots, max_rank, max_tokens=0, arena=None) -> int:
+FLAG_A_Q8 = 1
+
+
+def edgelora_pool_create(h_in, h_out, n_slots, max_rank, max_tokens=0, arena=None, flags=0) -> int:
     """Returns the opaque pool handle.  ``arena`` may be a torch CUDA tensor lent for the slot blocks."""
-    cfg = PoolConfig(h_in, h_out, n_slots, max_rank, max_tokens, 0,
+    cfg = PoolConfig(h_in, h_out, n_slots, max_rank, max_tokens, flags,
                      arena.data_ptr() if arena is not None else None,
                      arena.numel() * arena.element_size() if arena is not None else 0)
     out = ctypes.c_void_p()
@@ -447,8 +450,8 @@ def edgelora_cache_stats(cache) -> dict:
 class Pool:
     """Small convenience wrapper: owns a pool handle and loads a workload's adapters."""
 
-    def __init__(self, h_in, h_out, n_slots, max_rank, max_tokens=0, arena=None):
-        self.handle = edgelora_pool_create(h_in, h_out, n_slots, max_rank, max_tokens, arena)
+    def __init__(self, h_in, h_out, n_slots, max_rank, max_tokens=0, arena=None, flags=0):
+        self.handle = edgelora_pool_create(h_in, h_out, n_slots, max_rank, max_tokens, arena, flags)
         self.h_in, self.h_out, self.n_slots, self.max_rank = h_in, h_out, n_slots, max_rank
         self._arena = arena
 

@@ -115,11 +115,11 @@ cudaError_t launch_q8_to_block(const uint8_t *A_q8, const uint8_t *B_q8, uint16_
                                int32_t rank, int32_t R_pad, int32_t h_in, int32_t h_out, int32_t sms,
                                cudaStream_t stream);
 cudaError_t launch_wait_selftest(uint32_t *status, long long wait_cycles, cudaStream_t stream);
-cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &tmap_x,
+cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &tmap_d, const CUtensorMap &tmap_x,
                                  const int32_t *ids, const SlotRow *slots, const PlanView &pv,
                                  float *zws, int32_t *group_counters, int32_t T, int32_t h_in,
                                  int32_t R_pad, int32_t n_slots, int32_t max_tokens,
-                                 int32_t target_items, int32_t grid, uint32_t *status, bool pdl,
+                                 int32_t target_items, int32_t grid, uint32_t *status, bool pdl, bool a_q8,
                                  cudaStream_t stream);
 
 }  // namespace edgelora

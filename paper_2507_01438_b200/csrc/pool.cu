@@ -65,12 +65,12 @@ EncodeTiledFn get_encode_fn() {
 // elements read as zero.  box_cols == 64: the 128-byte-swizzled operand tiles of the GEMM;
 // otherwise (the shrink's row segments) no swizzle.
 int encode_tmap(CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1, uint64_t d2,
-                uint32_t box_rows, uint32_t box_cols) {
+                uint32_t box_rows, uint32_t box_cols, uint64_t s1 = 0, uint64_t s2 = 0) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return EDGELORA_ERR_CUDA;
   const cuuint32_t rank = d2 ? 3 : 2;
   cuuint64_t dims[3] = {d0, d1, d2 ? d2 : 1};
-  cuuint64_t strides[2] = {d0 * 2, d0 * d1 * 2};
+  cuuint64_t strides[2] = {s1 ? s1 : d0 * 2, s2 ? s2 : d0 * d1 * 2};
   cuuint32_t box[3] = {box_cols, box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), dims,
@@ -91,8 +91,8 @@ namespace {
 // The descriptor is copied out: a later miss of the same call may reuse the cache entry it came
 // from (the cache is a ring), and the launch takes its descriptors by value anyway.
 int get_tmap(edgelora_pool *p, CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1,
-             uint64_t d2, uint32_t box_rows, uint32_t box_cols = kBlockK) {
-  TmapKey key{base, d0, d1, d2, box_rows, box_cols};
+             uint64_t d2, uint32_t box_rows, uint32_t box_cols = kBlockK, uint64_t s1 = 0, uint64_t s2 = 0) {
+  TmapKey key{base, d0, d1, d2, box_rows, box_cols, s1, s2};
   for (auto &e : p->tmaps)
     if (e.key == key) {
       *out = e.map;
@@ -100,7 +100,7 @@ int get_tmap(edgelora_pool *p, CUtensorMap *out, const void *base, uint64_t d0, 
     }
   TmapEntry e;
   e.key = key;
-  int rc = encode_tmap(&e.map, base, d0, d1, d2, box_rows, box_cols);
+  int rc = encode_tmap(&e.map, base, d0, d1, d2, box_rows, box_cols, s1, s2);
   if (rc != EDGELORA_OK) return rc;
   *out = e.map;
   if (p->tmaps.size() < static_cast<size_t>(kTmapCache)) {
@@ -141,6 +141,7 @@ int check_cfg(const edgelora_pool_config *c) {
   if (!c) return EDGELORA_ERR_INVALID_ARG;
   if (c->h_in < 8 || c->h_out < 8 || (c->h_in % 8) || (c->h_out % 8)) return EDGELORA_ERR_INVALID_ARG;
   if (c->n_slots < 1 || c->n_slots > 65534) return EDGELORA_ERR_INVALID_ARG;
+  if ((c->flags & EDGELORA_FLAG_A_Q8) && (c->h_in % 256)) return EDGELORA_ERR_INVALID_ARG;
   if (c->max_rank < 1) return EDGELORA_ERR_INVALID_ARG;
   if (c->max_rank > 64) return EDGELORA_ERR_RANK_TOO_LARGE;
   if (c->max_tokens < 0 || c->max_tokens > kMaxTokensLimit) return EDGELORA_ERR_TOO_MANY_TOKENS;
@@ -149,7 +150,10 @@ int check_cfg(const edgelora_pool_config *c) {
 
 size_t arena_bytes_for(const edgelora_pool_config *c) {
   const size_t R = pad_rank(c->max_rank);
-  const size_t per_slot = 2 * R * (static_cast<size_t>(c->h_in) + c->h_out);
+  // A: bfloat16 rows, or Q8_0 rows of 34 bytes per 32 values; B: bfloat16
+  const size_t a_row = (c->flags & EDGELORA_FLAG_A_Q8) ? static_cast<size_t>(c->h_in) / 32 * 34
+                                                       : static_cast<size_t>(c->h_in) * 2;
+  const size_t per_slot = R * a_row + 2 * R * static_cast<size_t>(c->h_out);
   return per_slot * c->n_slots;
 }
 
@@ -314,7 +318,9 @@ int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool
   p->R_pad = pad_rank(cfg->max_rank);
   p->device = dev;
   p->sms = prop.multiProcessorCount;
-  p->a_block = static_cast<size_t>(p->R_pad) * cfg->h_in;
+  p->a_q8 = (cfg->flags & EDGELORA_FLAG_A_Q8) != 0;
+  // elements (2 bytes each) of a slot's A and B blocks; Q8_0 rows are 17 such elements per 32 values
+  p->a_block = p->a_q8 ? static_cast<size_t>(p->R_pad) * (cfg->h_in / 32) * 17 : static_cast<size_t>(p->R_pad) * cfg->h_in;
   p->b_block = static_cast<size_t>(cfg->h_out) * p->R_pad;
   p->slots_host.assign(cfg->n_slots, SlotRow{0, 0.f, 0, 0});
   p->tmaps.reserve(kTmapCache);
@@ -341,7 +347,9 @@ int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool
   POOL_TRY(cudaMemset(p->slots_dev, 0, sizeof(SlotRow) * cfg->n_slots));
   POOL_TRY(cudaMalloc(&p->status_dev, 16));
   POOL_TRY(cudaMemset(p->status_dev, 0, 16));
-  const size_t stage_bytes = (p->a_block + p->b_block) * 2 + sizeof(SlotRow);
+  // room for a block in its own layout or, for Q8_0 loads, A and B as 8-bit blocks (+ alignment)
+  const size_t b_q8_bytes = static_cast<size_t>(cfg->h_out) * ((p->R_pad + 31) / 32) * 34;
+  const size_t stage_bytes = p->a_block * 2 + 16 + std::max(p->b_block * 2, b_q8_bytes) + sizeof(SlotRow);
   for (auto &sb : p->staging) {
     POOL_TRY(cudaMallocHost(&sb.host, stage_bytes));
     POOL_TRY(cudaEventCreateWithFlags(&sb.done, cudaEventDisableTiming));
@@ -407,8 +415,15 @@ int edgelora_pool_destroy(edgelora_pool_t *p) {
   return EDGELORA_OK;
 }
 
+// where the slot-table row sits in a staging buffer: behind the largest payload
+static size_t slot_row_offset(const edgelora_pool *p) {
+  const size_t b_q8_bytes = static_cast<size_t>(p->cfg.h_out) * ((p->R_pad + 31) / 32) * 34;
+  return p->a_block * 2 + 16 + std::max(p->b_block * 2, b_q8_bytes);
+}
+
 static int stage_and_copy(edgelora_pool *p, int32_t slot, int32_t rank, float scale,
                           const uint16_t *A_host, const uint16_t *B_host) {
+  if (p->a_q8 && rank > 0) return EDGELORA_ERR_INVALID_ARG;  // this pool takes Q8_0 adapters only
   StagingBuf &sb = p->staging[p->next_staging];
   p->next_staging = (p->next_staging + 1) % kStagingBuffers;
   if (sb.in_flight) {
@@ -418,7 +433,7 @@ static int stage_and_copy(edgelora_pool *p, int32_t slot, int32_t rank, float sc
   const int h_in = p->cfg.h_in, h_out = p->cfg.h_out, R = p->R_pad;
   uint16_t *sa = reinterpret_cast<uint16_t *>(sb.host);
   uint16_t *sbp = sa + p->a_block;
-  SlotRow *srow = reinterpret_cast<SlotRow *>(sbp + p->b_block);
+  SlotRow *srow = reinterpret_cast<SlotRow *>(sb.host + slot_row_offset(p));
   SlotRow &mirror = p->slots_host[slot];
   mirror.rank = rank;
   mirror.scale = scale;
@@ -462,7 +477,7 @@ int edgelora_pool_load_slot_pinned(edgelora_pool_t *p, int32_t slot, int32_t ran
                                    const uint16_t *A_pinned, const uint16_t *B_pinned) {
   if (!p || !A_pinned || !B_pinned) return EDGELORA_ERR_INVALID_ARG;
   if (slot < 0 || slot >= p->cfg.n_slots) return EDGELORA_ERR_BAD_SLOT;
-  if (rank != p->R_pad) return EDGELORA_ERR_INVALID_ARG;  // already in the block's layout: nothing to pad
+  if (rank != p->R_pad || p->a_q8) return EDGELORA_ERR_INVALID_ARG;  // already in the block's layout: nothing to pad
   cudaPointerAttributes at{};
   if (cudaPointerGetAttributes(&at, A_pinned) != cudaSuccess || at.type != cudaMemoryTypeHost ||
       cudaPointerGetAttributes(&at, B_pinned) != cudaSuccess || at.type != cudaMemoryTypeHost) {
@@ -476,7 +491,7 @@ int edgelora_pool_load_slot_pinned(edgelora_pool_t *p, int32_t slot, int32_t ran
     CUDA_TRY(cudaEventSynchronize(sb.done));
     sb.in_flight = false;
   }
-  SlotRow *srow = reinterpret_cast<SlotRow *>(sb.host + (p->a_block + p->b_block) * 2);
+  SlotRow *srow = reinterpret_cast<SlotRow *>(sb.host + slot_row_offset(p));
   SlotRow &mirror = p->slots_host[slot];
   mirror.rank = rank;
   mirror.scale = scale;
@@ -512,10 +527,45 @@ int edgelora_pool_load_slot_q8(edgelora_pool_t *p, int32_t slot, int32_t rank, f
     CUDA_TRY(cudaEventSynchronize(sb.done));
     sb.in_flight = false;
   }
+  if (p->a_q8) {
+    // the pool keeps A in Q8_0: rows [rank, R_pad) are zero blocks; only B is converted on the device
+    const size_t a_pad = p->a_block * 2;
+    {  // the pool's layout: the signed bytes of all rows, then the block scales of all rows
+      const int nb = h_in / 32;
+      const uint8_t *src = static_cast<const uint8_t *>(A_q8);
+      uint8_t *qplane = sb.host, *dplane = sb.host + static_cast<size_t>(R) * h_in;
+      memset(sb.host, 0, a_pad);
+      for (int r = 0; r < rank; ++r)
+        for (int b = 0; b < nb; ++b) {
+          const uint8_t *blk = src + (static_cast<size_t>(r) * nb + b) * 34;
+          memcpy(dplane + (static_cast<size_t>(r) * nb + b) * 2, blk, 2);
+          memcpy(qplane + static_cast<size_t>(r) * h_in + b * 32, blk + 2, 32);
+        }
+    }
+    const size_t b_off2 = (a_pad + 15) & ~static_cast<size_t>(15);
+    memcpy(sb.host + b_off2, B_q8, b_bytes);
+    SlotRow *srow2 = reinterpret_cast<SlotRow *>(sb.host + slot_row_offset(p));
+    SlotRow &m2 = p->slots_host[slot];
+    m2.rank = rank;
+    m2.scale = scale;
+    m2.generation += 1;
+    *srow2 = m2;
+    if (p->use_recorded) CUDA_TRY(cudaStreamWaitEvent(p->side, p->use_ev, 0));
+    CUDA_TRY(cudaMemcpyAsync(p->A_pool + p->a_block * slot, sb.host, a_pad, cudaMemcpyHostToDevice, p->side));
+    CUDA_TRY(cudaMemcpyAsync(p->q8_dev, sb.host + b_off2, b_bytes, cudaMemcpyHostToDevice, p->side));
+    CUDA_TRY(launch_q8_to_block(nullptr, p->q8_dev, nullptr, p->B_pool + p->b_block * slot, rank, R, h_in, h_out,
+                                p->sms, p->side));
+    CUDA_TRY(cudaMemcpyAsync(p->slots_dev + slot, srow2, sizeof(SlotRow), cudaMemcpyHostToDevice, p->side));
+    CUDA_TRY(cudaEventRecord(sb.done, p->side));
+    sb.in_flight = true;
+    CUDA_TRY(cudaEventRecord(p->load_ev, p->side));
+    p->load_seq += 1;
+    return EDGELORA_OK;
+  }
   // the 8-bit form is smaller than the block the staging buffer was sized for
   memcpy(sb.host, A_q8, a_bytes);
   memcpy(sb.host + b_off, B_q8, b_bytes);
-  SlotRow *srow = reinterpret_cast<SlotRow *>(sb.host + (p->a_block + p->b_block) * 2);
+  SlotRow *srow = reinterpret_cast<SlotRow *>(sb.host + slot_row_offset(p));
   SlotRow &mirror = p->slots_host[slot];
   mirror.rank = rank;
   mirror.scale = scale;
@@ -837,6 +887,9 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
   // decode batches above this size take the plan kernel + tensor-core gather tiles; smaller ones
   // the single shrink kernel that derives the routing itself (a launch less)
   const int kGatherMinT = p->opt_gather_min_t;
+  // a pool that keeps A in Q8_0 is served by the decode shrink kernel only (it decodes the blocks as
+  // it streams them); the tensor-core shrink tiles need bfloat16 operand tiles
+  if (p->a_q8 && (regime != 1 || T > kGatherMinT)) return EDGELORA_ERR_INVALID_ARG;
 
   if (regime == 1) {
     // ---------------------------------------------------------------- decode
@@ -868,14 +921,27 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
       const int max_chunks = target == 1 ? 1 : std::max(1, std::min(kMaxZSplits, n_ksteps / 4));
       const int max_items = std::min(T, p->cfg.n_slots) * (R / 8) * max_chunks;
       const int grid = std::max(1, std::min(p->sms - 1, (max_items + 7) / 8)) + 1;  // + the publishing CTA
-      CUtensorMap ma, mx;
-      int rc = get_tmap(p, &ma, p->A_pool, h_in, R, p->cfg.n_slots, 8, kShrinkStepElems);
+      CUtensorMap ma, mx, md;
+      // A rows: bfloat16, or for a pool that keeps A in Q8_0 two planes per slot: the signed bytes
+      // [R_pad][h_in] (taken as 16-bit elements: 128 per K step) and the half-precision block scales
+      // [R_pad][h_in / 32] (8 per K step); both planes have the slot's byte stride
+      int rc;
+      if (p->a_q8) {
+        const uint64_t slot_bytes = p->a_block * 2;
+        rc = get_tmap(p, &ma, p->A_pool, h_in / 2, R, p->cfg.n_slots, 8, kShrinkStepElems / 2, h_in, slot_bytes);
+        if (rc) return rc;
+        rc = get_tmap(p, &md, reinterpret_cast<const uint8_t *>(p->A_pool) + static_cast<size_t>(R) * h_in, h_in / 32, R,
+                      p->cfg.n_slots, 8, kShrinkStepElems / 32, h_in / 16, slot_bytes);
+      } else {
+        rc = get_tmap(p, &ma, p->A_pool, h_in, R, p->cfg.n_slots, 8, kShrinkStepElems);
+        md = ma;
+      }
       if (rc) return rc;
       rc = get_tmap(p, &mx, x, h_in, T, 0, 1, kShrinkStepElems);
       if (rc) return rc;
-      CUDA_TRY(launch_decode_shrink(ma, mx, ids_in, p->slots_dev, plan->pv, p->zws, p->group_counters,
+      CUDA_TRY(launch_decode_shrink(ma, md, mx, ids_in, p->slots_dev, plan->pv, p->zws, p->group_counters,
                                     T, h_in, R, p->cfg.n_slots, p->cfg.max_tokens, target, grid,
-                                    p->status_dev, pdl_first, stream));
+                                    p->status_dev, pdl_first, p->a_q8, stream));
       ++launches;
     }
     int N = 32;  // tokens on the UMMA N axis: a power of two so that the cluster's owners get

@@ -22,8 +22,10 @@ struct TmapKey {
   const void *base;
   uint64_t d0, d1, d2;
   uint32_t b1, b0;  // box rows, box columns (64 => 128-byte swizzle, otherwise no swizzle)
+  uint64_t s1, s2;  // byte strides of dimensions 1 and 2 (0 = dense)
   bool operator==(const TmapKey &o) const {
-    return base == o.base && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && b1 == o.b1 && b0 == o.b0;
+    return base == o.base && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && b1 == o.b1 && b0 == o.b0 && s1 == o.s1 &&
+           s2 == o.s2;
   }
 };
 struct TmapEntry {
@@ -58,7 +60,7 @@ struct edgelora_pool {
   using ProfRec = edgelora::ProfRec;
   edgelora_pool_config cfg{};
   int R_pad = 0, device = 0, sms = 0;
-  bool owns_arena = false;
+  bool owns_arena = false, a_q8 = false;  // a_q8: the A blocks are kept in Q8_0 (EDGELORA_FLAG_A_Q8)
   uint8_t *arena = nullptr;
   uint8_t *q8_dev = nullptr;  // device scratch for one adapter in Q8_0 form (first use of load_slot_q8)
   uint16_t *A_pool = nullptr, *B_pool = nullptr;

@@ -28,7 +28,8 @@ __device__ __forceinline__ float q8_value(const uint8_t *row_blocks, int32_t k) 
 __global__ void __launch_bounds__(256)
 q8_to_block_kernel(const uint8_t *__restrict__ A_q8, const uint8_t *__restrict__ B_q8, uint16_t *__restrict__ A_blk,
                    uint16_t *__restrict__ B_blk, int32_t rank, int32_t R_pad, int32_t h_in, int32_t h_out) {
-  const size_t a_pairs = static_cast<size_t>(R_pad) * h_in / 2, b_pairs = static_cast<size_t>(h_out) * R_pad / 2;
+  // (A_q8 == nullptr: only B is converted, for pools that keep A in Q8_0)
+  const size_t a_pairs = A_q8 ? static_cast<size_t>(R_pad) * h_in / 2 : 0, b_pairs = static_cast<size_t>(h_out) * R_pad / 2;
   const size_t a_row_bytes = static_cast<size_t>(h_in / kQ8Block) * kQ8Bytes;
   const size_t b_row_bytes = static_cast<size_t>((rank + kQ8Block - 1) / kQ8Block) * kQ8Bytes;
   for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < a_pairs + b_pairs;

@@ -3,6 +3,8 @@
 // sub-batch so the adapter is fetched once), with the routing derived inside the kernel so that a
 // step of a few microseconds needs no routing launch.  Larger batches take the tensor-core gather
 // tiles of the tile kernel (gemm.cu).
+#include <cuda_fp16.h>
+
 #include "internal.cuh"
 #include "launch.cuh"
 #include "ptx.cuh"
@@ -81,8 +83,22 @@ struct RingShape {
   static constexpr int kDepth = (kDsDepth * kDsStageBytes) / kStage > kDsMaxDepth ? kDsMaxDepth
                                                                                   : (kDsDepth * kDsStageBytes) / kStage;
 };
-template <int NT, int kDsDepthCfg>
-__device__ __forceinline__ bool shrink_rows8(const CUtensorMap *tmap_a, const CUtensorMap *tmap_x,
+// kQ8: the A rows are kept in Q8_0 (paper Section 5.1: per 32 values a half-precision scale d and 32
+// signed bytes q, value d * q), in the pool as two planes per slot: the bytes [R_pad][h_in] and the
+// scales [R_pad][h_in / 32].  A K step of 256 values is then 256 bytes + 8 scales per row: two boxes
+// per step (8 x 256 bytes at the start of the stage, 8 x 16 bytes behind them), and lane l decodes the
+// eight values it owns (one aligned 8-byte load, block l / 4) on the fly: sum_e q_e x_e in fp32,
+// times d once.  17/32 of the bytes of the bfloat16 rows.
+constexpr int kQ8QBytes = kShrinkStepElems;            // 256 bytes of q per row and step
+constexpr int kQ8DBytes = (kShrinkStepElems / 32) * 2;  // 16 bytes of scales per row and step
+// signed byte i of w as a float: the byte with its sign bit flipped is q + 128, placed in the
+// mantissa of 2^23 it reads 2^23 + 128 + q
+__device__ __forceinline__ float s8_to_float(uint32_t w_flipped, int i) {
+  return __uint_as_float(__byte_perm(w_flipped, 0x4B000000u, 0x7440u + i)) - 8388736.0f;
+}
+template <int NT, int kDsDepthCfg, bool kQ8>
+__device__ __forceinline__ bool shrink_rows8(const CUtensorMap *tmap_a, const CUtensorMap *tmap_d,
+                                             const CUtensorMap *tmap_x,
                                              int32_t slot, int32_t row0, const int32_t (&tok)[kDsTok],
                                              int step0, int step1, int stride, uint8_t *ring, uint64_t *bars,
                                              uint32_t &phase, int lane, float (&acc)[8 * kDsTok]) {
@@ -91,8 +107,10 @@ __device__ __forceinline__ bool shrink_rows8(const CUtensorMap *tmap_a, const CU
   auto issue = [&](int step, int stage) {
     if (lane == 0 && step < step1) {
       uint8_t *dst = ring + stage * kStage;
-      ptx::mbar_arrive_expect_tx_relaxed(&bars[stage], (8 + NT) * kDsRowBytes);
-      ptx::tma_load_3d(dst, tmap_a, &bars[stage], step * kShrinkStepElems, row0, slot);
+      ptx::mbar_arrive_expect_tx_relaxed(&bars[stage],
+                                         (kQ8 ? 8 * (kQ8QBytes + kQ8DBytes) : 8 * kDsRowBytes) + NT * kDsRowBytes);
+      ptx::tma_load_3d(dst, tmap_a, &bars[stage], step * (kQ8 ? kQ8QBytes / 2 : kShrinkStepElems), row0, slot);
+      if (kQ8) ptx::tma_load_3d(dst + 8 * kQ8QBytes, tmap_d, &bars[stage], step * (kShrinkStepElems / 32), row0, slot);
 #pragma unroll
       for (int q = 0; q < NT; ++q)
         ptx::tma_load_2d(dst + (8 + q) * kDsRowBytes, tmap_x, &bars[stage], step * kShrinkStepElems, tok[q]);
@@ -110,14 +128,38 @@ __device__ __forceinline__ bool shrink_rows8(const CUtensorMap *tmap_a, const CU
     float xf[NT][8];
 #pragma unroll
     for (int q = 0; q < NT; ++q) unpack8(src[(8 + q) * (kDsRowBytes / 16)], xf[q]);
+    if (kQ8) {
+      const uint8_t *st = ring + stage * kStage;
 #pragma unroll
-    for (int r = 0; r < 8; ++r) {
-      float af[8];
-      unpack8(src[r * (kDsRowBytes / 16)], af);
+      for (int r = 0; r < 8; ++r) {
+        const uint2 qq = *reinterpret_cast<const uint2 *>(st + r * kQ8QBytes + lane * 8);
+        const float d = __half2float(__ushort_as_half(
+            *reinterpret_cast<const unsigned short *>(st + 8 * kQ8QBytes + r * kQ8DBytes + (lane >> 2) * 2)));
+        const uint32_t w0 = qq.x ^ 0x80808080u, w1 = qq.y ^ 0x80808080u;
+        float qf[8];
 #pragma unroll
-      for (int q = 0; q < NT; ++q)
+        for (int e = 0; e < 4; ++e) {
+          qf[e] = s8_to_float(w0, e);
+          qf[4 + e] = s8_to_float(w1, e);
+        }
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[r * kDsTok + q] = fmaf(af[e], xf[q][e], acc[r * kDsTok + q]);
+        for (int q = 0; q < NT; ++q) {
+          float part = 0.f;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) part = fmaf(qf[e], xf[q][e], part);
+          acc[r * kDsTok + q] = fmaf(d, part, acc[r * kDsTok + q]);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        float af[8];
+        unpack8(src[r * (kDsRowBytes / 16)], af);
+#pragma unroll
+        for (int q = 0; q < NT; ++q)
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[r * kDsTok + q] = fmaf(af[e], xf[q][e], acc[r * kDsTok + q]);
+      }
     }
     if (++stage == kDsDepth) stage = 0;
   }
@@ -138,9 +180,10 @@ constexpr size_t ds_ring_bytes(int depth) {
 
 // kDsDepth = 4 fills an SM's shared memory (large batches: bandwidth); kDsDepth = 2 leaves room
 // for a CTA of the base-product kernel beside it (small batches: the two kernels overlap).
-template <int kDsDepth>
+template <int kDsDepth, bool kQ8>
 __global__ void __launch_bounds__(kShrinkThreads, 2)  // <= 128 registers: fits beside the base-product CTAs
-decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_x,
+decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_d,
+                     const __grid_constant__ CUtensorMap tmap_x,
                      const int32_t *__restrict__ ids, const SlotRow *__restrict__ slots,
                      PlanView pv, float *__restrict__ zws, int32_t *__restrict__ group_counters,
                      int32_t T, int32_t h_in, int32_t R_pad, int32_t n_slots, int32_t max_tokens,
@@ -403,10 +446,10 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       int32_t tok[kDsTok];
 #pragma unroll
       for (int qq = 0; qq < kDsTok; ++qq) tok[qq] = s_gtok[tb + min(qq, nt - 1)];
-      if (nt == 1) ok = shrink_rows8<1, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
-      else if (nt == 2) ok = shrink_rows8<2, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
-      else if (nt == 3) ok = shrink_rows8<3, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
-      else ok = shrink_rows8<4, kDsDepth>(&tmap_a, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
+      if (nt == 1) ok = shrink_rows8<1, kDsDepth, kQ8>(&tmap_a, &tmap_d, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
+      else if (nt == 2) ok = shrink_rows8<2, kDsDepth, kQ8>(&tmap_a, &tmap_d, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
+      else if (nt == 3) ok = shrink_rows8<3, kDsDepth, kQ8>(&tmap_a, &tmap_d, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
+      else ok = shrink_rows8<4, kDsDepth, kQ8>(&tmap_a, &tmap_d, &tmap_x, ad, rg * 8, tok, step0, step1, KS, ring, bars, phase, lane, acc);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       // lane L ends with the sum over lanes of value L (= row L / 4, token L % 4)
@@ -451,27 +494,29 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
 // The shared-memory limit is an attribute of (function, device): set for the current device, by
 // edgelora_pool_create, so that every device a pool lives on is configured.
 cudaError_t shrink_set_smem_limit() {
-  cudaError_t e = cudaFuncSetAttribute(decode_shrink_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(ds_ring_bytes(4)));
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(decode_shrink_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              static_cast<int>(ds_ring_bytes(2)));
+  cudaError_t e = cudaSuccess;
+  const int b4 = static_cast<int>(ds_ring_bytes(4)), b2 = static_cast<int>(ds_ring_bytes(2));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_shrink_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b4);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_shrink_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b2);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_shrink_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b4);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_shrink_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b2);
+  return e;
 }
 
-cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &tmap_x,
+cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &tmap_d, const CUtensorMap &tmap_x,
                                  const int32_t *ids, const SlotRow *slots, const PlanView &pv,
                                  float *zws, int32_t *group_counters, int32_t T, int32_t h_in,
                                  int32_t R_pad, int32_t n_slots, int32_t max_tokens,
-                                 int32_t target_items, int32_t grid, uint32_t *status, bool pdl,
+                                 int32_t target_items, int32_t grid, uint32_t *status, bool pdl, bool a_q8,
                                  cudaStream_t stream) {
   const int32_t late_ticket = pdl ? 1 : 0;  // pdl here = this launch may start under the call before it
-  if (T <= 64)
-    return launch_ex(decode_shrink_kernel<2>, dim3(grid), dim3(kShrinkThreads), ds_ring_bytes(2), stream, pdl, 1,
-                     tmap_a, tmap_x, ids, slots, pv, zws, group_counters, T, h_in, R_pad, n_slots,
-                     max_tokens, target_items, late_ticket, status);
-  return launch_ex(decode_shrink_kernel<4>, dim3(grid), dim3(kShrinkThreads), ds_ring_bytes(4), stream, pdl, 1,
-                   tmap_a, tmap_x, ids, slots, pv, zws, group_counters, T, h_in, R_pad, n_slots,
-                   max_tokens, target_items, late_ticket, status);
+#define EDGELORA_SHRINK(D, Q)                                                                                     \
+  launch_ex(decode_shrink_kernel<D, Q>, dim3(grid), dim3(kShrinkThreads), ds_ring_bytes(D), stream, pdl, 1, tmap_a, \
+            tmap_d, tmap_x, ids, slots, pv, zws, group_counters, T, h_in, R_pad, n_slots, max_tokens, target_items,        \
+            late_ticket, status)
+  if (T <= 64) return a_q8 ? EDGELORA_SHRINK(2, true) : EDGELORA_SHRINK(2, false);
+  return a_q8 ? EDGELORA_SHRINK(4, true) : EDGELORA_SHRINK(4, false);
+#undef EDGELORA_SHRINK
 }
 
 }  // namespace edgelora
