@@ -98,6 +98,8 @@ typedef struct {
                                         kernel + tensor-core gather shrink, the others the single shrink
                                         kernel with the routing inside.  Default 256: every decode batch
                                         takes the single kernel (it is the faster one as measured)   */
+#define EDGELORA_OPT_SHRINK_DEPTH 9  /* tuning: ring depth of the decode shrink for batches above 64 tokens:
+                                        2 (default, two CTAs per SM) or 4 (one CTA per SM); 0 = default */
 #define EDGELORA_OPT_WAIT_CYCLES 6   /* limit of every bounded in-kernel wait of the layer, in units
                                         of 1024 SM clock cycles; 0 = default (about two seconds).
                                         A wait that runs out raises EDGELORA_STATUS_TIMEOUT           */

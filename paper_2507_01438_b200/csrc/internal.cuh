@@ -120,6 +120,6 @@ cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &t
                                  float *zws, int32_t *group_counters, int32_t T, int32_t h_in,
                                  int32_t R_pad, int32_t n_slots, int32_t max_tokens,
                                  int32_t target_items, int32_t grid, uint32_t *status, bool pdl, bool a_q8,
-                                 cudaStream_t stream);
+                                 int32_t depth, cudaStream_t stream);
 
 }  // namespace edgelora

@@ -637,6 +637,10 @@ int edgelora_pool_set_option(edgelora_pool_t *p, int32_t option, int32_t value) 
       if (value < 0) return EDGELORA_ERR_INVALID_ARG;
       p->opt_shrink_items = value;
       return EDGELORA_OK;
+    case EDGELORA_OPT_SHRINK_DEPTH:
+      if (value != 0 && value != 2 && value != 4) return EDGELORA_ERR_INVALID_ARG;
+      p->opt_shrink_depth = value;
+      return EDGELORA_OK;
     case EDGELORA_OPT_GATHER_SPLITS:
       if (value < 0 || value > 8) return EDGELORA_ERR_INVALID_ARG;
       p->opt_gather_splits = value;
@@ -915,12 +919,17 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
       // call's base product, so its length does not matter but its tail does: one K chunk per
       // item (no pass that adds chunks) and few CTAs (they take SM resources from the base product).
       const bool overlapped = pdl_first && T <= 64;
-      const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : (overlapped ? 1 : 4 * 8 * p->sms);
+      // ring depth 2 lets two CTAs share an SM: twice the warps in flight with half the ring each,
+      // which suits a kernel bound by the per-warp chain of copy issue, wait and FMAs (measured on
+      // the 200-adapter down_proj: 45.8 us against 49.8 us with depth 4)
+      const int shrink_depth = T <= 64 ? 2 : (p->opt_shrink_depth == 4 ? 4 : 2);
+      const int cta_cap = shrink_depth == 2 && T > 64 ? 2 * p->sms : p->sms;
+      const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : (overlapped ? 1 : 4 * 8 * cta_cap);
       // at most T token blocks x (R / 8) row groups x K chunks warp items, eight warps per CTA
       const int n_ksteps = (h_in + kShrinkStepElems - 1) / kShrinkStepElems;
       const int max_chunks = target == 1 ? 1 : std::max(1, std::min(kMaxZSplits, n_ksteps / 4));
       const int max_items = std::min(T, p->cfg.n_slots) * (R / 8) * max_chunks;
-      const int grid = std::max(1, std::min(p->sms - 1, (max_items + 7) / 8)) + 1;  // + the publishing CTA
+      const int grid = std::max(1, std::min(cta_cap - 1, (max_items + 7) / 8)) + 1;  // + the publishing CTA
       CUtensorMap ma, mx, md;
       // A rows: bfloat16, or for a pool that keeps A in Q8_0 two planes per slot: the signed bytes
       // [R_pad][h_in] (taken as 16-bit elements: 128 per K step) and the half-precision block scales
@@ -941,7 +950,7 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
       if (rc) return rc;
       CUDA_TRY(launch_decode_shrink(ma, md, mx, ids_in, p->slots_dev, plan->pv, p->zws, p->group_counters,
                                     T, h_in, R, p->cfg.n_slots, p->cfg.max_tokens, target, grid,
-                                    p->status_dev, pdl_first, p->a_q8, stream));
+                                    p->status_dev, pdl_first, p->a_q8, shrink_depth, stream));
       ++launches;
     }
     int N = 32;  // tokens on the UMMA N axis: a power of two so that the cluster's owners get

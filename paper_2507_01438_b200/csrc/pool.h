@@ -77,7 +77,7 @@ struct edgelora_pool {
   edgelora_plan *plan = nullptr;
   float *zws = nullptr;
   int32_t *group_counters = nullptr;
-  int opt_decode_splits = 0, opt_shrink_items = 0, opt_gather_splits = 0, opt_gather_min_t = 256;
+  int opt_decode_splits = 0, opt_shrink_items = 0, opt_gather_splits = 0, opt_gather_min_t = 256, opt_shrink_depth = 0;
   uint32_t *status_dev = nullptr;
   std::vector<TmapEntry> tmaps;
   size_t tmap_next = 0;

@@ -508,13 +508,13 @@ cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &t
                                  float *zws, int32_t *group_counters, int32_t T, int32_t h_in,
                                  int32_t R_pad, int32_t n_slots, int32_t max_tokens,
                                  int32_t target_items, int32_t grid, uint32_t *status, bool pdl, bool a_q8,
-                                 cudaStream_t stream) {
+                                 int32_t depth, cudaStream_t stream) {
   const int32_t late_ticket = pdl ? 1 : 0;  // pdl here = this launch may start under the call before it
 #define EDGELORA_SHRINK(D, Q)                                                                                     \
   launch_ex(decode_shrink_kernel<D, Q>, dim3(grid), dim3(kShrinkThreads), ds_ring_bytes(D), stream, pdl, 1, tmap_a, \
             tmap_d, tmap_x, ids, slots, pv, zws, group_counters, T, h_in, R_pad, n_slots, max_tokens, target_items,        \
             late_ticket, status)
-  if (T <= 64) return a_q8 ? EDGELORA_SHRINK(2, true) : EDGELORA_SHRINK(2, false);
+  if (depth == 2) return a_q8 ? EDGELORA_SHRINK(2, true) : EDGELORA_SHRINK(2, false);
   return a_q8 ? EDGELORA_SHRINK(4, true) : EDGELORA_SHRINK(4, false);
 #undef EDGELORA_SHRINK
 }
