@@ -72,6 +72,17 @@ __device__ __forceinline__ int32_t gather_tiles(const GemmParams &p) {
   return (p.counts[4] + per - 1) / per;
 }
 
+// Prefill jobs: tiles are dealt round-robin to the CTAs of the persistent grid, so when the tile count
+// is not a multiple of the grid the CTAs from (count % grid) on get one tile fewer.  The tiles of the
+// first token tile go to those CTAs (as their first tile): in a serving batch the first token tile
+// holds the decode tokens (one token per generating request, many adapters, so many LoRA K blocks),
+// and its tiles are the longest of the launch.  Returns how many tiles are placed that way.
+__device__ __forceinline__ int32_t heavy_slots(const GemmParams &p, int32_t grid) {
+  const int32_t total = p.n_mtiles * p.n_ntiles, rem = total % grid;
+  if (p.mode != kModePrefill || p.n_mtiles < 2 || total <= grid || rem == 0) return 0;
+  return min(p.n_ntiles, grid - rem);
+}
+
 __device__ __forceinline__ int32_t total_tiles(const GemmParams &p) {
   if (p.mode == kModePrefill) return p.n_mtiles * p.n_ntiles;
   if (p.mode == kModeDecode) return p.n_mtiles * p.splits;
@@ -87,7 +98,26 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams &p, int32_t til
   c.g0 = c.ng = c.tok0 = c.ntok = c.gtile = 0;
   int32_t kb_per = p.kb_per;
   if (p.mode == kModePrefill) {
-    const int m = tile % p.n_mtiles, n = tile / p.n_mtiles;
+    int m, n;
+    const int32_t H = heavy_slots(p, gridDim.x);
+    const int32_t rem = (p.n_mtiles * p.n_ntiles) % static_cast<int32_t>(gridDim.x);
+    if (H > 0 && tile >= rem && tile < rem + H) {  // first-wave positions of the CTAs with a tile fewer
+      m = 0;
+      n = tile - rem;
+    } else if (H > 0) {  // the other tiles in their usual order, the H placed ones taken out
+      const int32_t u = tile < rem ? tile : tile - H;
+      if (u < H * (p.n_mtiles - 1)) {
+        n = u / (p.n_mtiles - 1);
+        m = 1 + u % (p.n_mtiles - 1);
+      } else {
+        const int32_t o = u + H;
+        n = o / p.n_mtiles;
+        m = o % p.n_mtiles;
+      }
+    } else {
+      m = tile % p.n_mtiles;
+      n = tile / p.n_mtiles;
+    }
     c.row_r = m * kTileM;
     c.row_c = n * p.BN;
     c.split = 0;
@@ -409,7 +439,9 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
 
   if (p.mode == kModeSgmv) ptx::pdl_wait_prior_grids();  // tile list comes from the plan kernel
   const int32_t n_tiles0 = total_tiles(p);
-  const int32_t n_tiles = n_tiles0 + (has2 ? p2.n_mtiles : 0);
+  // the second job's tiles start behind the CTAs that took the first token tile's tiles (above)
+  const int32_t n_hole = has2 ? heavy_slots(p, gridDim.x) : 0;
+  const int32_t n_tiles = n_tiles0 + n_hole + (has2 ? p2.n_mtiles : 0);
   const uint32_t nstages = static_cast<uint32_t>(p.stages);
   // Every role walks the same tile sequence: tiles below n_tiles0 belong to the first job; for the
   // others the true count of the second job is read once (after griddepcontrol.wait: the plan may
@@ -420,7 +452,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       ptx::pdl_wait_prior_grids();
       n2_true = total_tiles(p2);
     }
-    const int32_t local = tile - n_tiles0;
+    const int32_t local = tile - n_tiles0 - n_hole;
     return local < n2_true ? local : -1;
   };
 
@@ -445,6 +477,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
         const bool second = tile >= n_tiles0;
         int32_t local = tile;
+        if (second && tile < n_tiles0 + n_hole) continue;
         if (second && (local = second_job_tile(tile)) < 0) break;
         const GemmParams &jp = second ? p2 : p;
         const CUtensorMap *mr = second ? &tmap_r2 : &tmap_r, *mc = second ? &tmap_c2 : &tmap_c;
@@ -527,6 +560,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
         const bool second = tile >= n_tiles0;
         int32_t local = tile;
+        if (second && tile < n_tiles0 + n_hole) continue;
         if (second && (local = second_job_tile(tile)) < 0) break;
         const GemmParams &jp = second ? p2 : p;
         const TileCoord tc = tile_coord(jp, local);
@@ -667,6 +701,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
       const bool second = tile >= n_tiles0;
       int32_t local = tile;
+      if (second && tile < n_tiles0 + n_hole) continue;
       if (second && (local = second_job_tile(tile)) < 0) break;
       const GemmParams &jp = second ? p2 : p;
       const TileCoord tc = tile_coord(jp, local);
@@ -985,6 +1020,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     }
     for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
       if (kShrink && tile >= n_tiles0) {  // a tile of the second job: no LoRA blocks
+        if (tile < n_tiles0 + n_hole) continue;
         const int32_t local = second_job_tile(tile);
         if (local < 0) break;
         ok = shrink_tile(p2, local, &tmap_c2, &tmap_g2);

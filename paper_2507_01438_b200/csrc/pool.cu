@@ -827,7 +827,8 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
     if (!sgmv) return 1;
     const int kbt = (q->cfg.h_in + kBlockK - 1) / kBlockK;
     const int tiles_est = std::max(1, T / kTileM);
-    int z = std::max(1, std::min({in_set ? 2 : 8, q->sms / tiles_est, kbt / 4}));
+    // (inside a set: items of about 32 K blocks, so that a wide input does not make them long)
+    int z = std::max(1, std::min({in_set ? std::max(2, std::min(8, kbt / 32)) : 8, q->sms / tiles_est, kbt / 4}));
     const int kb_per = (kbt + z - 1) / z;
     return (kbt + kb_per - 1) / kb_per;
   };
@@ -1039,7 +1040,10 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
     if (rc) return rc;
     const int n_mtiles = (T + kTileM - 1) / kTileM;
     const int tiles256 = n_mtiles * ((h_out + 255) / 256);
-    int BN = (tiles256 >= p->sms || h_out <= 128) ? 256 : 128;
+    // 256-wide tiles unless they would leave three quarters of the SMs without a tile: a K block costs
+    // the producer warp about as much for a 128-wide W tile as for a 256-wide one, so narrow tiles
+    // only pay through parallelism
+    int BN = (tiles256 * 4 >= p->sms || h_out <= 128) ? 256 : 128;
     BN = std::min(BN, round_up(h_out, 32));
     g.mode = kModePrefill;
     g.BN = BN;
