@@ -554,9 +554,14 @@ def bench_site(name, ctx, steps=None, warmup=None, pdl=None, graph=True, cpu_bud
         # writes y once; its fp32 split-K partials are not counted
         gemm_bytes = 2 * w.h_in * w.h_out + 2 * w.T * (w.h_in + w.h_out) + \
             sum(2 * w.adapters[a].rank * w.h_out for a in w.distinct_adapters())
+        kernel_name = "lora_gemm_kernel (decode mode)"
+        if "shrink_small_decode" not in kt and "shrink_tiles" not in kt:
+            # one launch per call: the same kernel also reads every distinct A_a (its shrink teams)
+            gemm_bytes = ws_bytes
+            kernel_name = "lora_gemm_kernel (decode mode with the shrink teams in its grid: the whole call)"
         achieved = gemm_bytes / (gemm_us * 1e-6) / 1e9
         peak = pk["hbm_gbs"]
-        roof = {"bound": "hbm", "kernel": "lora_gemm_kernel (decode mode)", "achieved": achieved, "peak": peak,
+        roof = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "traffic": ncu_traffic(name),
                 "algorithmic_bytes": gemm_bytes, "kernel_us": gemm_us,
                 "kernel_us_is": "serialised latency of one launch between two CUDA events (launch gap included)",

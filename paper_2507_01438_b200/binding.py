@@ -19,7 +19,7 @@ ERR_INVALID_ARG, ERR_BAD_SLOT, ERR_RANK_TOO_LARGE, ERR_ARENA_TOO_SMALL = -1, -2,
 ERR_CUDA, ERR_BAD_ADAPTER_ID, ERR_SLOT_EMPTY, ERR_TIMEOUT, ERR_TOO_MANY_TOKENS = -5, -6, -7, -8, -9
 STATUS_BAD_ADAPTER_ID, STATUS_SLOT_EMPTY, STATUS_TIMEOUT = 0x1, 0x2, 0x4
 OPT_REGIME, OPT_PROFILE, OPT_PDL, OPT_DECODE_SPLITS, OPT_SHRINK_ITEMS, OPT_WAIT_CYCLES = 1, 2, 3, 4, 5, 6
-OPT_GATHER_SPLITS, OPT_GATHER_MIN_T, OPT_SHRINK_DEPTH = 7, 8, 9
+OPT_GATHER_SPLITS, OPT_GATHER_MIN_T, OPT_SHRINK_DEPTH, OPT_FUSED_DECODE = 7, 8, 9, 10
 KERNEL_NAMES = ("plan", "shrink_small_decode", "shrink_tiles", "base_gemm")
 
 EXPORTS = (

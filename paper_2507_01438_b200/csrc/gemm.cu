@@ -25,6 +25,10 @@
 // epilogue (each reads the 32 TMEM lanes of its quadrant), warps 6..9 build the z operand.
 // Every mbarrier wait is bounded; on a timeout the status word gets EDGELORA_STATUS_TIMEOUT and
 // all roles leave their loops.
+#include <cstdio>
+#include <cstdlib>
+
+#include "decode_route.cuh"
 #include "internal.cuh"
 #include "launch.cuh"
 #include "ptx.cuh"
@@ -167,8 +171,8 @@ __device__ __forceinline__ int32_t tile_passes(const GemmParams &p, const TileCo
 }
 
 // decode: first W row of the tile this CTA works on
-__device__ __forceinline__ int32_t tc_row0(const GemmParams &p) {
-  return static_cast<int32_t>(blockIdx.x) / p.splits * kTileM;
+__device__ __forceinline__ int32_t tc_row0(const GemmParams &p, int32_t bid) {
+  return bid / p.splits * kTileM;
 }
 
 // The LoRA K blocks of a tile: entries [e0, e1) step `de` of `list`.  Entries whose slot is
@@ -346,20 +350,171 @@ __device__ __forceinline__ bool gather_pass_copies(const GemmParams &jp, const T
   return true;
 }
 
+__device__ __forceinline__ int32_t ld_acquire_gpu(const int32_t *ptr) {
+  int32_t v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+
+// Fused decode launches (batches of at most 64 tokens): z[t] = s_a A_a x[t] on the CUDA cores, by
+// "teams" of four warps: the four builder warps of every CTA of the decode job (idle there, because
+// the expand is added by the owners of the cluster reduction) and two teams in every spare CTA.
+// A team item is (token, eight rank rows, K chunk): chunk c covers the K steps c, c + ks, ... of 256
+// elements; warp w of the team takes every fourth of them, lane l the elements [8 l, 8 l + 8) of a
+// step (one 16-byte load of x and eight of A in flight per lane).  The four warps' sums meet in
+// shared memory and are added in a fixed order; the partial result goes to plane c of f.z, and the
+// expand adds the planes in order.  Rows at or past the rank are never read by the expand and are
+// not written.  s_tid / s_trank / s_tscale: the tokens' validated ids, ranks and scales in shared
+// memory; s_red: 48 floats; bar_id: a named barrier of the team's 128 threads.
+template <int kBarId>
+__device__ __forceinline__ void shrink_team_items(const GemmParams &p, const FusedDecode &f, int team, int n_teams,
+                                                  int wt, int lane, const int32_t *s_tid, const int32_t *s_trank,
+                                                  const float *s_tscale, float *s_red, bool &waited) {
+  const int n_ksteps = (p.h_in + kShrinkStepElems - 1) / kShrinkStepElems;
+  const int n_rgn = p.R_pad >> 3, KS = f.ks;
+  const int n_items = p.T * n_rgn * KS;
+  const size_t zplane = static_cast<size_t>(p.max_tokens) * p.R_pad;
+  const int row_u4 = p.h_in >> 3;  // 16-byte pieces of a row (h_in is a multiple of 8)
+  int par = 0;
+  for (int item = team; item < n_items; item += n_teams) {
+    const int c = item % KS, tr = item / KS;
+    const int t = tr / n_rgn, rg = tr - t * n_rgn;
+    const int at = s_tid[t], rank = s_trank[t];
+    if (at < 0) continue;
+    if (rank <= 0) {
+      if (wt == 0 && lane == 0 && c == 0 && rg == 0) atomicOr(p.status, EDGELORA_STATUS_SLOT_EMPTY);
+      continue;
+    }
+    if (rg * 8 >= rank) continue;  // zero padding of the block
+    const uint4 *Arow =
+        reinterpret_cast<const uint4 *>(f.A_pool + (static_cast<size_t>(at) * p.R_pad + rg * 8) * p.h_in);
+    const uint4 *xrow = reinterpret_cast<const uint4 *>(f.x + static_cast<size_t>(t) * p.h_in);
+    float acc[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) acc[r] = 0.f;
+    for (int s0 = c + KS * wt; s0 < n_ksteps; s0 += 4 * KS) {
+      const int k0 = s0 * 32 + lane;
+      if (k0 >= row_u4) continue;
+      uint4 av[8];
+      const uint4 xv = __ldcg(xrow + k0);
+#pragma unroll
+      for (int r = 0; r < 8; ++r) av[r] = __ldg(Arow + static_cast<size_t>(r) * row_u4 + k0);
+      const float xf[8] = {ptx::bf16_lo(xv.x), ptx::bf16_hi(xv.x), ptx::bf16_lo(xv.y), ptx::bf16_hi(xv.y),
+                           ptx::bf16_lo(xv.z), ptx::bf16_hi(xv.z), ptx::bf16_lo(xv.w), ptx::bf16_hi(xv.w)};
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        float v = acc[r];
+        v = fmaf(ptx::bf16_lo(av[r].x), xf[0], v);
+        v = fmaf(ptx::bf16_hi(av[r].x), xf[1], v);
+        v = fmaf(ptx::bf16_lo(av[r].y), xf[2], v);
+        v = fmaf(ptx::bf16_hi(av[r].y), xf[3], v);
+        v = fmaf(ptx::bf16_lo(av[r].z), xf[4], v);
+        v = fmaf(ptx::bf16_hi(av[r].z), xf[5], v);
+        v = fmaf(ptx::bf16_lo(av[r].w), xf[6], v);
+        v = fmaf(ptx::bf16_hi(av[r].w), xf[7], v);
+        acc[r] = v;
+      }
+    }
+    float out = 0.f;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      float v = acc[r];
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+      if (lane == r) out = v;
+    }
+    // buffer `par` is written again two items later, behind the next item's barrier, which warp 0
+    // reaches only after it has read this item's sums
+    if (wt > 0 && lane < 8) s_red[(par * 3 + wt - 1) * 8 + lane] = out;
+    named_bar_sync(kBarId, 128);
+    if (wt == 0) {
+      if (!waited) {  // first write of this team to memory that earlier kernels may read
+        ptx::pdl_wait_prior_grids();
+        waited = true;
+      }
+      if (lane < 8) {
+        const float sum = ((out + s_red[(par * 3 + 0) * 8 + lane]) + s_red[(par * 3 + 1) * 8 + lane]) +
+                          s_red[(par * 3 + 2) * 8 + lane];
+        f.z[c * zplane + static_cast<size_t>(t) * p.R_pad + rg * 8 + lane] = s_tscale[t] * sum;
+      }
+    }
+    par ^= 1;
+  }
+  if (wt == 0) {
+    __syncwarp();  // the lanes' z stores happen before lane 0's release
+    if (lane == 0) {
+      ptx::pdl_wait_prior_grids();  // the counters belong to the kernel before this one until it is done
+      __threadfence();
+      atomicAdd(f.sync, 1);
+    }
+  }
+}
+
+// A spare CTA of a fused decode launch: two shrink teams (warps 0..3 and 4..7); the first spare CTA
+// also publishes the routing plan.
+__device__ __forceinline__ void fused_shrink_cta(const GemmParams &p, const FusedDecode &f, uint8_t *smem, int n_teams) {
+  int32_t *s_id = reinterpret_cast<int32_t *>(smem);  // [256] validated ids
+  int32_t *s_cnt = s_id + 256;                        // [256] scratch of the plan publication
+  int32_t *s_rank = s_cnt + 256;                      // [256]
+  float *s_scale = reinterpret_cast<float *>(s_rank + 256);  // [256]
+  float *s_red = s_scale + 256;                              // [2][48]
+  int *s_wt = reinterpret_cast<int *>(s_red + 96);           // [9]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  ptx::pdl_launch_dependents();
+  int a = -1;
+  bool bad = false;
+  if (tid < p.T) {
+    a = p.ids[tid];
+    if (a < -1 || a >= p.n_slots) {
+      a = -1;
+      bad = true;
+    }
+  }
+  SlotRow row = {0, 0.f, 0, 0};
+  if (a >= 0) row = p.slots[a];
+  if (tid < 256) {
+    s_id[tid] = a;
+    s_rank[tid] = row.rank;
+    s_scale[tid] = row.scale;
+  }
+  const int any_bad = __syncthreads_or(bad ? 1 : 0);
+  bool waited = false;
+  if (f.x_wait) {
+    ptx::pdl_wait_prior_grids();
+    waited = true;
+  }
+  if (warp < 4)
+    shrink_team_items<2>(p, f, static_cast<int>(blockIdx.x) * 2, n_teams, warp, lane, s_id, s_rank, s_scale, s_red,
+                         waited);
+  else if (warp < 8)
+    shrink_team_items<3>(p, f, static_cast<int>(blockIdx.x) * 2 + 1, n_teams, warp - 4, lane, s_id, s_rank, s_scale,
+                         s_red + 48, waited);
+  if (blockIdx.x == 0) publish_decode_plan(f.pv, a, p.T, any_bad, f.ks, s_id, s_cnt, s_wt);
+}
+
 // kMinBlocks = 2 caps the registers so that two CTAs share an SM (small decode tiles); with 1 the
 // builder keeps both of its z rows in registers without spilling.  kShrink = false compiles the
 // kernel without the shrink jobs (segment and gather tiles, second job) and without the staged y
 // stores: the decode-mode launches, which need none of them, keep a smaller kernel.
-template <int kMinBlocks, bool kShrink>
+// kFused: a decode launch whose first f.n_ctas CTAs are shrink CTAs (fused_shrink_cta); the job's
+// own CTAs are numbered from there.
+template <int kMinBlocks, bool kShrink, bool kFused>
 __global__ void __launch_bounds__(kGemmThreads, kMinBlocks)
 lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_constant__ CUtensorMap tmap_c,
                  const __grid_constant__ CUtensorMap tmap_b, const GemmParams p,
                  const __grid_constant__ CUtensorMap tmap_r2, const __grid_constant__ CUtensorMap tmap_c2,
                  const __grid_constant__ CUtensorMap tmap_g2, const GemmParams p2,
-                 const __grid_constant__ CUtensorMap tmap_y) {
+                 const __grid_constant__ CUtensorMap tmap_y, const FusedDecode f) {
   extern __shared__ uint8_t smem_raw[];
   // tiles need 1024-byte alignment for the 128-byte swizzle
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int32_t cta0 = kFused ? f.n_ctas : 0;  // whole clusters: the cluster ranks of the others are unchanged
+  const int32_t ngrid0 = static_cast<int32_t>(gridDim.x) - cta0;
+  if (kFused && static_cast<int32_t>(blockIdx.x) < cta0) {
+    fused_shrink_cta(p, f, smem, 2 * cta0 + ngrid0);
+    return;
+  }
+  const int32_t bid = static_cast<int32_t>(blockIdx.x) - cta0, ngrid = ngrid0;
   const uint32_t r_bytes = kTileM * kBlockK * 2;              // 16 KB
   const uint32_t c_bytes = static_cast<uint32_t>(p.BN) * kBlockK * 2;
   // the ring is laid out for the first job: its C region holds ring_rows rows
@@ -390,6 +545,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
   volatile int32_t *s_last = reinterpret_cast<volatile int32_t *>(extra + 80);  // gather tiles: last arriver
   uint64_t *ep_bar = reinterpret_cast<uint64_t *>(extra + 88);              // rendezvous of the epilogue warps
   uint8_t *y_stage = reinterpret_cast<uint8_t *>(bars) + 4096;              // prefill epilogue: 4 x 4 KB, 1024-aligned
+  uint8_t *b_stage = y_stage;  // fused decode: B_a rows of the owner's tokens, then their z (never both uses at once)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wl = p.wait_cycles;  // limit of every bounded wait below
@@ -456,13 +612,14 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     return local < n2_true ? local : -1;
   };
 
+  bool fused_z_ok = true;  // fused launches: set by the epilogue warps' wait for the shrink teams
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     // The whole warp walks the loop (state stays uniform); lane 0 waits and issues the tile loads,
     // and for gather tiles every lane issues its share of the one-row loads.
     {
       uint32_t stage = 0, phase = 0, unused_go = 0;
-      bool ok = true, waited = p.mode == kModeSgmv;
+      bool ok = true, waited = p.mode == kModeSgmv, x_waited = false;
       auto wait_empty = [&]() {  // lane 0 polls, the warp learns the result
         int got = 1;
         if (lane == 0) got = (ptx::mbar_wait(&empty_bar[stage], phase ^ 1, wl) && !*abort_flag) ? 1 : 0;
@@ -474,7 +631,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
           phase ^= 1;
         }
       };
-      for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+      for (int32_t tile = bid; ok && tile < n_tiles; tile += ngrid) {
         const bool second = tile >= n_tiles0;
         int32_t local = tile;
         if (second && tile < n_tiles0 + n_hole) continue;
@@ -491,7 +648,27 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
           continue;
         }
         const uint32_t tx_bytes = r_bytes + static_cast<uint32_t>(jp.BN) * kBlockK * 2;
-        for (int32_t kb = tc.kb0; kb < tc.kb1; ++kb) {
+        int32_t kb_first = tc.kb0;
+        if (kFused && f.x_wait && !x_waited) {
+          // x may be an output of the kernel before this one, W is not: the W tiles of the first ring
+          // revolution are requested before the dependency wait, the x tiles after it
+          const int32_t npre = min(static_cast<int32_t>(nstages), tc.kb1 - tc.kb0);  // the ring is empty: no waits
+          if (lane == 0)
+            for (int32_t i = 0; i < npre; ++i) {
+              ptx::mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
+              ptx::tma_load_2d(smem + static_cast<size_t>(i) * stage_bytes, mr, &full_bar[i], (tc.kb0 + i) * kBlockK,
+                               tc.row_r);
+            }
+          ptx::pdl_wait_prior_grids();
+          if (lane == 0)
+            for (int32_t i = 0; i < npre; ++i)
+              ptx::tma_load_2d(smem + static_cast<size_t>(i) * stage_bytes + r_bytes, mc, &full_bar[i],
+                               (tc.kb0 + i) * kBlockK, tc.row_c);
+          for (int32_t i = 0; i < npre; ++i) advance();
+          kb_first += npre;
+          x_waited = true;
+        }
+        for (int32_t kb = kb_first; kb < tc.kb1; ++kb) {
           if (!wait_empty()) {
             ok = false;
             break;
@@ -557,7 +734,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       uint32_t stage = 0, phase = 0, zphase = 0;  // zphase: one parity bit per stage
       bool ok = true, waited = p.mode == kModeSgmv;
       int32_t it = 0;
-      for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+      for (int32_t tile = bid; ok && tile < n_tiles; tile += ngrid) {
         const bool second = tile >= n_tiles0;
         int32_t local = tile;
         if (second && tile < n_tiles0 + n_hole) continue;
@@ -665,7 +842,44 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     const int quad = warp & 3;                      // TMEM lanes [32*quad, 32*quad+32)
     const int row_in_tile = quad * 32 + lane;
     const bool clustered = p.mode == kModeDecode && p.splits > 1;
-    if (clustered && p.expand_in_reduce) {
+    if (kFused && clustered && f.b_stage) {
+      // This CTA will finish tokens [rank * cols_per, ...) of its row tile: the B_a rows they need (the
+      // tile's 128 rows of the token's adapter, contiguous in the pool) are copied into shared memory
+      // now, one bulk copy per token, while the main loop runs (the ids are the caller's input, the
+      // pool is not written by this kernel).  One warp per token; cols_per <= 16.
+      const int cols_per = p.BN / p.splits;
+      const int t0 = static_cast<int>(cluster_cta_rank()) * cols_per;
+      const uint32_t tok_bytes = kTileM * p.R_pad * 2;
+      const uint32_t copy_bytes = static_cast<uint32_t>(min(kTileM, p.h_out - tc_row0(p, bid)) * p.R_pad * 2);
+      int32_t a_of[4];
+      uint32_t my_bytes = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int cl = quad + 4 * i;
+        int32_t a = -1, rank = 0;
+        if (cl < cols_per && t0 + cl < p.T) {
+          a = p.ids[t0 + cl];
+          if (a < 0 || a >= p.n_slots) a = -1;
+          if (a >= 0) rank = p.slots[a].rank;
+        }
+        if (rank <= 0) a = -1;
+        a_of[i] = a;
+        if (cl < cols_per && lane == 0) {  // kept for the expand at the end
+          s_vid[cl] = a;
+          s_lg[cl] = rank;
+        }
+        if (a >= 0) my_bytes += copy_bytes;
+      }
+      if (lane == 0) {
+        ptx::mbar_arrive_expect_tx(ep_bar, my_bytes);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (a_of[i] >= 0)
+            ptx::bulk_load_1d(b_stage + static_cast<size_t>(quad + 4 * i) * tok_bytes,
+                              p.B_pool + (static_cast<size_t>(a_of[i]) * p.h_out + tc_row0(p, bid)) * p.R_pad,
+                              copy_bytes, ep_bar);
+      }
+    } else if (clustered && p.expand_in_reduce) {
       // This CTA will finish tokens [rank * cols_per, ...) of its row tile; pull the B_a rows they
       // need into L2 now (the ids are the caller's input, the pool is not written by the shrink).
       const int cols_per = p.BN / p.splits;
@@ -684,12 +898,55 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         if (t0 + cl < p.T) {
           if (a >= 0 && a < p.n_slots) {
             const uint8_t *rows = reinterpret_cast<const uint8_t *>(
-                p.B_pool + (static_cast<size_t>(a) * p.h_out + tc_row0(p)) * p.R_pad);
-            const int bytes = min(kTileM, p.h_out - tc_row0(p)) * p.R_pad * 2;  // this tile's rows, contiguous
+                p.B_pool + (static_cast<size_t>(a) * p.h_out + tc_row0(p, bid)) * p.R_pad);
+            const int bytes = min(kTileM, p.h_out - tc_row0(p, bid)) * p.R_pad * 2;  // this tile's rows, contiguous
             for (int off = lane * 128; off < bytes; off += 32 * 128)
               asm volatile("prefetch.global.L2 [%0];" ::"l"(rows + off));
           }
         }
+      }
+    }
+    if (kFused && clustered) {
+      // z comes from the shrink teams of this grid (every CTA of the launch is resident, so all of them
+      // run).  These warps have nothing to do until the accumulator is complete: bounded wait for the
+      // teams' arrival counter now, then this thread's share of the owner's z (tokens x R_pad floats,
+      // at most 128 16-byte pieces; the K chunks' planes added in order) goes to shared memory, behind
+      // the staged B_a rows.
+      const int cols_per = p.BN / p.splits, etid = threadIdx.x - 64;
+      const int my_rank = static_cast<int>(cluster_cta_rank());
+      // the counter belongs to the kernel before this one (another launch of this pool, which leaves it
+      // at zero) until that kernel is done
+      ptx::pdl_wait_prior_grids();
+      // one thread of the CTA polls; the named barrier of the four warps passes its acquire on
+      if (warp == 2 && lane == 0) {
+        int got = 1;
+        const long long t_start = clock64();
+        while (ld_acquire_gpu(f.sync) < 2 * cta0 + ngrid) {
+          if (clock64() - t_start > wl) {
+            got = 0;
+            break;
+          }
+        }
+        if (!got) atomicOr(p.status, EDGELORA_STATUS_TIMEOUT);
+        *s_last = got;  // (the gather tiles' flag: unused in this launch)
+      }
+      named_bar_sync(1, 128);
+      fused_z_ok = *s_last != 0;
+      const int tok = my_rank * cols_per + etid / (p.R_pad >> 2);
+      if (f.b_stage && fused_z_ok && etid < cols_per * (p.R_pad >> 2)) {
+        float4 z_mine = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (tok < p.T) {
+          const size_t zplane4 = static_cast<size_t>(p.max_tokens) * p.R_pad / 4;
+          const float4 *zp = reinterpret_cast<const float4 *>(f.z) +
+                             static_cast<size_t>(my_rank) * cols_per * (p.R_pad >> 2) + etid;
+          z_mine = __ldcg(zp);
+          for (int sp = 1; sp < f.ks; ++sp) {
+            const float4 w = __ldcg(zp + sp * zplane4);
+            z_mine.x += w.x; z_mine.y += w.y; z_mine.z += w.z; z_mine.w += w.w;
+          }
+        }
+        // read by the expand, behind two cluster barriers
+        reinterpret_cast<float4 *>(b_stage + static_cast<size_t>(cols_per) * kTileM * p.R_pad * 2)[etid] = z_mine;
       }
     }
     // Earlier kernels may still read y, and z comes from the shrink kernel.  With the expand in
@@ -698,7 +955,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     bool ok = true;
     int32_t it = 0;
     uint32_t ep_phase = 0;
-    for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+    for (int32_t tile = bid; ok && tile < n_tiles; tile += ngrid) {
       const bool second = tile >= n_tiles0;
       int32_t local = tile;
       if (second && tile < n_tiles0 + n_hole) continue;
@@ -932,6 +1189,32 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       *abort_flag = 1;
       atomicOr(p.status, EDGELORA_STATUS_TIMEOUT);
     }
+  } else if (kFused) {
+    // ------------------------------------------------------------ shrink team (warps 6..9)
+    const int btid = threadIdx.x - 192;  // 0..127
+    int32_t *s_tid = reinterpret_cast<int32_t *>(s_key) + 64;  // s_key is free: no LoRA K blocks in this launch
+    int32_t *s_trank = s_tid + 64;
+    float *s_tscale = reinterpret_cast<float *>(s_trank + 64);
+    if (btid < 64) {
+      int32_t a = -1;
+      if (btid < p.T) {
+        a = p.ids[btid];
+        if (a < 0 || a >= p.n_slots) a = -1;
+      }
+      SlotRow row = {0, 0.f, 0, 0};
+      if (a >= 0) row = p.slots[a];
+      s_tid[btid] = a;
+      s_trank[btid] = row.rank;
+      s_tscale[btid] = row.scale;
+    }
+    named_bar_sync(2, 128);
+    bool waited = false;
+    if (f.x_wait) {
+      ptx::pdl_wait_prior_grids();
+      waited = true;
+    }
+    shrink_team_items<2>(p, f, 2 * cta0 + bid, 2 * cta0 + ngrid, warp - 6, lane, s_tid, s_trank, s_tscale,
+                         reinterpret_cast<float *>(s_key), waited);
   } else if (has_lora || has2 || (kShrink && p.mode == kModeSgmv && p.gather)) {
     // ------------------------------------------------------------ z operand builder (warps 6..9)
     // (and, during gather tiles, parts 1..4 of the tile's copies)
@@ -1018,7 +1301,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       named_bar_sync(2, 128);
       if (btid == 0) ptx::mbar_arrive(lg_bar);
     }
-    for (int32_t tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+    for (int32_t tile = bid; ok && tile < n_tiles; tile += ngrid) {
       if (kShrink && tile >= n_tiles0) {  // a tile of the second job: no LoRA blocks
         if (tile < n_tiles0 + n_hole) continue;
         const int32_t local = second_job_tile(tile);
@@ -1115,6 +1398,8 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     const bool sender = epi || (wide && warp >= 6);
     const int c_first = (wide && warp >= 6) ? 32 : 0, c_step = wide ? 64 : 32;
     const bool have_acc = sender && !*abort_flag;  // this CTA's accumulator is complete (tfull waited)
+    const bool z_ok = fused_z_ok;  // fused launches: the wait for the shrink teams ended in time
+    float4 *z_stage = reinterpret_cast<float4 *>(b_stage + static_cast<size_t>(cols_per) * kTileM * p.R_pad * 2);
     __syncwarp();
     cluster_sync_all();
     if (have_acc) {
@@ -1126,7 +1411,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       for (int32_t c0 = c_first; c0 < p.BN; c0 += c_step) {
         float v[32];
         ptx::tmem_ld_32x32(taddr + c0, v);
-        if (p.expand_in_reduce) {  // buf[src][token][row]
+        if (p.expand_in_reduce && !(kFused && f.b_stage)) {  // buf[src][token][row]
 #pragma unroll
           for (int jj = 0; jj < 32; ++jj) {
             const int col = c0 + jj;
@@ -1151,7 +1436,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     if (epi || wide) {
       const float *buf = reinterpret_cast<const float *>(smem);
       const int n_units = cols_per * 32;  // unit = (token, 4 adjacent W rows)
-      const int row0 = blockIdx.x / p.splits * kTileM;
+      const int row0 = bid / p.splits * kTileM;
       auto sum_partials = [&](int cl, int r4) {
         float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int sp = 0; sp < p.splits; ++sp) {
@@ -1188,6 +1473,80 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
               p.y[static_cast<size_t>(t0 + i) * p.h_out + j] =
                   static_cast<uint16_t>(ptx::pack_bf16x2(o[i], 0.f) & 0xFFFFu);
         }
+      } else if (kFused && f.b_stage) {
+        // Small batches, one launch: unit = (token quad, W row), as above, and everything the expand
+        // needs is in shared memory by now: B_a[row][0..R_pad) of each token's adapter (lanes take
+        // adjacent rows: 32-byte pieces side by side) and the tokens' z (the same for every lane).
+        const int qpo = cols_per >> 2;
+        const float4 *buf4 = reinterpret_cast<const float4 *>(smem);
+        const int n_units = qpo * kTileM;  // at most 4 per thread (cols_per <= 16)
+        const int nch = p.R_pad >> 3;
+        float4 base[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int u = etid + i * 128;
+          float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (u < n_units)
+            for (int sp = 0; sp < p.splits; ++sp) {
+              const float4 w = buf4[(sp * qpo + (u >> 7)) * kTileM + (u & 127)];
+              a4.x += w.x; a4.y += w.y; a4.z += w.z; a4.w += w.w;
+            }
+          base[i] = a4;
+        }
+        ptx::pdl_wait_prior_grids();  // earlier kernels may still read y
+        bool b_ok = true;
+        {
+          int got = 1;
+          if (lane == 0) got = ptx::mbar_wait(ep_bar, 0, wl) ? 1 : 0;  // the staged B_a rows
+          if (!__shfl_sync(0xffffffffu, got, 0)) {
+            if (lane == 0) atomicOr(p.status, EDGELORA_STATUS_TIMEOUT);
+            b_ok = false;
+          }
+        }
+        const int j = row0 + (etid & 127);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int u = etid + i * 128;
+          if (u >= n_units || j >= p.h_out) break;
+          const int qd = u >> 7, r = u & 127;
+          float o[4] = {base[i].x, base[i].y, base[i].z, base[i].w};
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int cl = qd * 4 + k;
+            const int32_t a = (z_ok && b_ok) ? s_vid[cl] : -1, rank = s_lg[cl];
+            if (a < 0) continue;
+            const uint4 *Brow = reinterpret_cast<const uint4 *>(b_stage + static_cast<size_t>(cl) * kTileM * p.R_pad * 2) + r * nch;
+            const float4 *zt = z_stage + cl * (p.R_pad >> 2);
+            float add = 0.f;
+            for (int c = 0; c < nch && c * 8 < rank; ++c) {
+              const uint4 bb = Brow[c];
+              const float4 u0 = zt[2 * c], u1 = zt[2 * c + 1];
+              add = fmaf(ptx::bf16_lo(bb.x), u0.x, add);
+              add = fmaf(ptx::bf16_hi(bb.x), u0.y, add);
+              add = fmaf(ptx::bf16_lo(bb.y), u0.z, add);
+              add = fmaf(ptx::bf16_hi(bb.y), u0.w, add);
+              add = fmaf(ptx::bf16_lo(bb.z), u1.x, add);
+              add = fmaf(ptx::bf16_hi(bb.z), u1.y, add);
+              add = fmaf(ptx::bf16_lo(bb.w), u1.z, add);
+              add = fmaf(ptx::bf16_hi(bb.w), u1.w, add);
+            }
+            o[k] += add;
+          }
+          const int t0q = static_cast<int>(my_rank) * cols_per + qd * 4;
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if (t0q + k < p.T)
+              p.y[static_cast<size_t>(t0q + k) * p.h_out + j] =
+                  static_cast<uint16_t>(ptx::pack_bf16x2(o[k], 0.f) & 0xFFFFu);
+        }
+        if (lane == 0) {
+          // this warp is past its wait for the shrink teams: the last such warp of the grid puts both
+          // counters back to zero for the next launch
+          if (atomicAdd(f.sync + 1, 1) == ngrid * 4 - 1) {
+            f.sync[0] = 0;
+            f.sync[1] = 0;
+          }
+        }
       } else {
         // Small batches.  Everything that does not need z first: the base product's sums stay in
         // registers (at most 4 units per thread: cols_per <= 16).  Then wait for the shrink kernel
@@ -1201,6 +1560,16 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         }
         ptx::pdl_wait_prior_grids();
         const int nch = p.R_pad >> 3;
+        const int n_zp = kFused ? f.ks : 1;
+        const size_t zplane4 = static_cast<size_t>(p.max_tokens) * p.R_pad / 4;
+        auto load_z4 = [&](const float4 *ptr) {
+          float4 v = __ldcg(ptr);
+          for (int sp = 1; sp < n_zp; ++sp) {
+            const float4 w = __ldcg(ptr + sp * zplane4);
+            v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+          }
+          return v;
+        };
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int u = etid + i * 128;
@@ -1209,11 +1578,11 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
           const int t = static_cast<int>(my_rank) * cols_per + cl, j = row0 + r4;
           if (t >= p.T || j >= p.h_out) continue;
           float4 acc4 = base[i];
-          const int32_t a = s_vid[cl], rank = s_lg[cl];  // stored by the epilogue warps at the start
+          const int32_t a = z_ok ? s_vid[cl] : -1, rank = s_lg[cl];  // stored by the epilogue warps at the start
           if (a >= 0) {
             const uint4 *Brow = reinterpret_cast<const uint4 *>(
                 p.B_pool + (static_cast<size_t>(a) * p.h_out + j) * p.R_pad);
-            const float4 *zt = reinterpret_cast<const float4 *>(p.zws + static_cast<size_t>(t) * p.R_pad);
+            const float4 *zt = reinterpret_cast<const float4 *>((kFused ? f.z : p.zws) + static_cast<size_t>(t) * p.R_pad);
             float add[4] = {0.f, 0.f, 0.f, 0.f};
             for (int c0 = 0; c0 < nch && c0 * 8 < rank; c0 += 2) {
               uint4 b[2][4];
@@ -1224,8 +1593,8 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
                 const bool on = c < nch && c * 8 < rank;
 #pragma unroll
                 for (int r = 0; r < 4; ++r) b[cc][r] = on ? __ldg(Brow + r * nch + c) : make_uint4(0u, 0u, 0u, 0u);
-                z4[cc][0] = on ? __ldcg(zt + 2 * c) : make_float4(0.f, 0.f, 0.f, 0.f);
-                z4[cc][1] = on ? __ldcg(zt + 2 * c + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+                z4[cc][0] = on ? load_z4(zt + 2 * c) : make_float4(0.f, 0.f, 0.f, 0.f);
+                z4[cc][1] = on ? load_z4(zt + 2 * c + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
               }
 #pragma unroll
               for (int cc = 0; cc < 2; ++cc) {
@@ -1250,6 +1619,14 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
           }
           store4(t, j, acc4);
         }
+        if (kFused && lane == 0) {
+          // this warp is past its wait for the shrink teams: the last such warp of the grid puts both
+          // counters back to zero for the next launch
+          if (atomicAdd(f.sync + 1, 1) == ngrid * 4 - 1) {
+            f.sync[0] = 0;
+            f.sync[1] = 0;
+          }
+        }
       }
     }
   }
@@ -1269,14 +1646,23 @@ static GemmParams no_job() {
   none.mode = -1;
   return none;
 }
+static FusedDecode not_fused() {
+  FusedDecode f{};
+  return f;
+}
 
 cudaError_t gemm_set_smem_limit(size_t smem_bytes) {
   cudaError_t e = cudaSuccess;
   const int bytes = static_cast<int>(smem_bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(lora_gemm_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(lora_gemm_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(lora_gemm_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(lora_gemm_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+#define EDGELORA_SMEM(MB, SH, FU)                                                                               \
+  if (e == cudaSuccess)                                                                                         \
+    e = cudaFuncSetAttribute(lora_gemm_kernel<MB, SH, FU>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  EDGELORA_SMEM(1, true, false)
+  EDGELORA_SMEM(2, true, false)
+  EDGELORA_SMEM(1, false, false)
+  EDGELORA_SMEM(2, false, false)
+  EDGELORA_SMEM(1, false, true)
+#undef EDGELORA_SMEM
   return e;
 }
 
@@ -1285,6 +1671,10 @@ cudaError_t launch_gemm(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col
                         size_t smem_bytes, bool pdl, cudaStream_t stream, const CUtensorMap *tmap_y) {
   return launch_gemm2(tmap_row, tmap_col, tmap_b, p, tmap_row, tmap_col, tmap_b, no_job(), grid, smem_bytes,
                       pdl, stream, tmap_y);
+}
+
+static bool two_per_sm(size_t smem_bytes, int32_t BN, int32_t acc_cols) {
+  return smem_bytes * 2 <= 225 * 1024 && BN <= 128 && acc_cols <= 128;
 }
 
 // With a second job: p2.mode == kModeSgmv (a shrink job: segment tiles and, with p2.gather, gather
@@ -1297,14 +1687,45 @@ cudaError_t launch_gemm2(const CUtensorMap &tmap_row, const CUtensorMap &tmap_co
                          const CUtensorMap *tmap_y) {
   const CUtensorMap &my = tmap_y ? *tmap_y : tmap_row;  // unused unless p.y_tma
   const int cluster = (p.mode == kModeDecode && p.splits > 1) ? p.splits : 1;
-  const bool two = smem_bytes * 2 <= 225 * 1024 && p.BN <= 128 && p.acc_cols <= 128;  // two CTAs fit an SM
-  const bool lean = p.mode == kModeDecode && p2.mode != kModeSgmv;                    // no shrink job, plain y stores
-#define EDGELORA_LAUNCH(MB, SH)                                                                                \
-  launch_ex(lora_gemm_kernel<MB, SH>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster, tmap_row, \
-            tmap_col, tmap_b, p, tmap_row2, tmap_col2, tmap_g2, p2, my)
+  const bool two = two_per_sm(smem_bytes, p.BN, p.acc_cols);        // two CTAs fit an SM
+  const bool lean = p.mode == kModeDecode && p2.mode != kModeSgmv;  // no shrink job, plain y stores
+#define EDGELORA_LAUNCH(MB, SH)                                                                                    \
+  launch_ex(lora_gemm_kernel<MB, SH, false>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, cluster,      \
+            tmap_row, tmap_col, tmap_b, p, tmap_row2, tmap_col2, tmap_g2, p2, my, not_fused())
   if (two) return lean ? EDGELORA_LAUNCH(2, false) : EDGELORA_LAUNCH(2, true);
   return lean ? EDGELORA_LAUNCH(1, false) : EDGELORA_LAUNCH(1, true);
 #undef EDGELORA_LAUNCH
+}
+
+cudaError_t launch_gemm_fused(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col, const GemmParams &p,
+                              const FusedDecode &f, size_t smem_bytes, bool pdl, cudaStream_t stream) {
+  const int32_t grid = f.n_ctas + p.n_mtiles * p.splits;
+  return launch_ex(lora_gemm_kernel<1, false, true>, dim3(grid), dim3(kGemmThreads), smem_bytes, stream, pdl, p.splits,
+                   tmap_row, tmap_col, tmap_row, p, tmap_row, tmap_col, tmap_row, no_job(), tmap_row, f);
+}
+
+int32_t gemm_fused_max_ctas(int32_t cluster, size_t smem_bytes) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(cluster) * 64);
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, lora_gemm_kernel<1, false, true>, &cfg);
+  if (getenv("EDGELORA_LOG"))
+    fprintf(stderr, "edgelora: one-launch decode, clusters of %d, %zu bytes of shared memory: %s, %d clusters fit\n",
+            cluster, smem_bytes, cudaGetErrorString(e), n);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return n * cluster;
 }
 
 }  // namespace edgelora

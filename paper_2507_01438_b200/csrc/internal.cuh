@@ -96,6 +96,23 @@ struct GemmParams {
   uint32_t *status;
 };
 
+// Small decode batches in one launch (paper Section 3.4, both LoRA products and the base product of
+// one layer call): the first n_ctas CTAs of the tile kernel's grid compute z = s_a A_a x on the CUDA
+// cores while the others stream W; the owners of the cluster reduction wait (bounded) for the
+// shrink CTAs' arrival counter before they add B_a z.
+struct FusedDecode {
+  int32_t n_ctas;          // 0 = not fused; otherwise a multiple of the cluster size
+  int32_t ks;              // K chunks of the shrink = partial z planes the expand adds, in order
+  int32_t x_wait;          // 1: x may be an output of the kernel before this one: wait before reading it
+  int32_t b_stage;         // 1: the launch's shared memory has room, behind the ring and the barriers, for the
+                           // B_a rows (tokens per owner x 128 rows x R_pad) and z of an owner's tokens
+  const uint16_t *A_pool;  // [S][R_pad][h_in]
+  const uint16_t *x;       // [T][h_in]
+  float *z;                // [ks][max_tokens][R_pad]
+  int32_t *sync;           // [2] {shrink CTAs done, expand warps past their wait}; zero between launches
+  PlanView pv;             // published by the first shrink CTA
+};
+
 // kernels (defined in plan.cu, shrink.cu, gemm.cu)
 void launch_plan(const int32_t *ids, int32_t T, int32_t n_slots, const PlanView &pv, bool pdl,
                  cudaStream_t stream);
@@ -108,6 +125,11 @@ cudaError_t launch_gemm2(const CUtensorMap &tmap_row, const CUtensorMap &tmap_co
                          const CUtensorMap &tmap_col2, const CUtensorMap &tmap_g2, const GemmParams &p2,
                          int32_t grid, size_t smem_bytes, bool pdl, cudaStream_t stream,
                          const CUtensorMap *tmap_y = nullptr);
+// Decode job with the shrink in the same grid: grid = f.n_ctas + p.n_mtiles * p.splits CTAs.
+cudaError_t launch_gemm_fused(const CUtensorMap &tmap_row, const CUtensorMap &tmap_col, const GemmParams &p,
+                              const FusedDecode &f, size_t smem_bytes, bool pdl, cudaStream_t stream);
+// How many CTAs of such a launch (in whole clusters) can be resident at once on the current device.
+int32_t gemm_fused_max_ctas(int32_t cluster, size_t smem_bytes);
 constexpr int kYStageBytes = 4 * 32 * 128;  // prefill epilogue: per epilogue warp 32 rows x 64 bf16
 cudaError_t gemm_set_smem_limit(size_t smem_bytes);
 cudaError_t shrink_set_smem_limit();

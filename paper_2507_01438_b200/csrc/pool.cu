@@ -641,6 +641,10 @@ int edgelora_pool_set_option(edgelora_pool_t *p, int32_t option, int32_t value) 
       if (value != 0 && value != 2 && value != 4) return EDGELORA_ERR_INVALID_ARG;
       p->opt_shrink_depth = value;
       return EDGELORA_OK;
+    case EDGELORA_OPT_FUSED_DECODE:
+      if (value != 0 && value != 1) return EDGELORA_ERR_INVALID_ARG;
+      p->opt_fused_decode = value;
+      return EDGELORA_OK;
     case EDGELORA_OPT_GATHER_SPLITS:
       if (value < 0 || value > 8) return EDGELORA_ERR_INVALID_ARG;
       p->opt_gather_splits = value;
@@ -694,6 +698,9 @@ int edgelora_pool_sync_status(edgelora_pool_t *p, uint32_t *bits_out) {
   CUDA_TRY(cudaMemset(p->plan->pv.status, 0, 4));
   const uint32_t bits = a | b;
   if (bits_out) *bits_out = bits;
+  // a wait that ran out can leave arrival counters between their values: nothing is in flight now
+  if (bits & EDGELORA_STATUS_TIMEOUT)
+    CUDA_TRY(cudaMemset(p->group_counters, 0, sizeof(int32_t) * (kDecodeMaxT * 8 + 32)));
   if (bits & EDGELORA_STATUS_TIMEOUT) return EDGELORA_ERR_TIMEOUT;
   if (bits & EDGELORA_STATUS_BAD_ADAPTER_ID) return EDGELORA_ERR_BAD_ADAPTER_ID;
   if (bits & EDGELORA_STATUS_SLOT_EMPTY) return EDGELORA_ERR_SLOT_EMPTY;
@@ -900,60 +907,63 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
     // ---------------------------------------------------------------- decode
     const int32_t *ids_in = ids_dev ? ids_dev : plan->pv.ids_valid;
     plan->last_T = T;
-    if (T > kGatherMinT) {
-      if (ids_dev) {
-        ProfScope ps(p, 0, stream);
-        launch_plan(ids_dev, T, plan->n_slots, plan->pv, pdl_first, stream);
-        CUDA_TRY(cudaGetLastError());
+    auto launch_shrink = [&]() -> int {
+      if (T > kGatherMinT) {
+        if (ids_dev) {
+          ProfScope ps(p, 0, stream);
+          launch_plan(ids_dev, T, plan->n_slots, plan->pv, pdl_first, stream);
+          CUDA_TRY(cudaGetLastError());
+          ++launches;
+        }
+        ShrinkJob sj;
+        int rc = shrink_job(p, x, true, 0, &sj);
+        if (rc) return rc;
+        ProfScope ps(p, 2, stream);
+        CUDA_TRY(launch_gemm(sj.mx, sj.ma, sj.mg, sj.s, sj.grid, sj.smem, ids_dev ? pdl : pdl_first, stream));
+        ++launches;
+      } else
+      {
+        ProfScope ps(p, 1, stream);
+        // When calls overlap (EDGELORA_OPT_PDL = 2) a small batch's shrink runs under the previous
+        // call's base product, so its length does not matter but its tail does: one K chunk per
+        // item (no pass that adds chunks) and few CTAs (they take SM resources from the base product).
+        const bool overlapped = pdl_first && T <= 64;
+        // ring depth 2 lets two CTAs share an SM: twice the warps in flight with half the ring each,
+        // which suits a kernel bound by the per-warp chain of copy issue, wait and FMAs (measured on
+        // the 200-adapter down_proj: 45.8 us against 49.8 us with depth 4)
+        const int shrink_depth = T <= 64 ? 2 : (p->opt_shrink_depth == 4 ? 4 : 2);
+        const int cta_cap = shrink_depth == 2 && T > 64 ? 2 * p->sms : p->sms;
+        const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : (overlapped ? 1 : 4 * 8 * cta_cap);
+        // at most T token blocks x (R / 8) row groups x K chunks warp items, eight warps per CTA
+        const int n_ksteps = (h_in + kShrinkStepElems - 1) / kShrinkStepElems;
+        const int max_chunks = target == 1 ? 1 : std::max(1, std::min(kMaxZSplits, n_ksteps / 4));
+        const int max_items = std::min(T, p->cfg.n_slots) * (R / 8) * max_chunks;
+        const int grid = std::max(1, std::min(cta_cap - 1, (max_items + 7) / 8)) + 1;  // + the publishing CTA
+        CUtensorMap ma, mx, md;
+        // A rows: bfloat16, or for a pool that keeps A in Q8_0 two planes per slot: the signed bytes
+        // [R_pad][h_in] (taken as 16-bit elements: 128 per K step) and the half-precision block scales
+        // [R_pad][h_in / 32] (8 per K step); both planes have the slot's byte stride
+        int rc;
+        if (p->a_q8) {
+          const uint64_t slot_bytes = p->a_block * 2;
+          rc = get_tmap(p, &ma, p->A_pool, h_in / 2, R, p->cfg.n_slots, 8, kShrinkStepElems / 2, h_in, slot_bytes);
+          if (rc) return rc;
+          rc = get_tmap(p, &md, reinterpret_cast<const uint8_t *>(p->A_pool) + static_cast<size_t>(R) * h_in, h_in / 32, R,
+                        p->cfg.n_slots, 8, kShrinkStepElems / 32, h_in / 16, slot_bytes);
+        } else {
+          rc = get_tmap(p, &ma, p->A_pool, h_in, R, p->cfg.n_slots, 8, kShrinkStepElems);
+          md = ma;
+        }
+        if (rc) return rc;
+        rc = get_tmap(p, &mx, x, h_in, T, 0, 1, kShrinkStepElems);
+        if (rc) return rc;
+        CUDA_TRY(launch_decode_shrink(ma, md, mx, ids_in, p->slots_dev, plan->pv, p->zws, p->group_counters,
+                                      T, h_in, R, p->cfg.n_slots, p->cfg.max_tokens, target, grid,
+                                      p->status_dev, pdl_first, p->a_q8, shrink_depth, stream));
         ++launches;
       }
-      ShrinkJob sj;
-      int rc = shrink_job(p, x, true, 0, &sj);
-      if (rc) return rc;
-      ProfScope ps(p, 2, stream);
-      CUDA_TRY(launch_gemm(sj.mx, sj.ma, sj.mg, sj.s, sj.grid, sj.smem, ids_dev ? pdl : pdl_first, stream));
-      ++launches;
-    } else
-    {
-      ProfScope ps(p, 1, stream);
-      // When calls overlap (EDGELORA_OPT_PDL = 2) a small batch's shrink runs under the previous
-      // call's base product, so its length does not matter but its tail does: one K chunk per
-      // item (no pass that adds chunks) and few CTAs (they take SM resources from the base product).
-      const bool overlapped = pdl_first && T <= 64;
-      // ring depth 2 lets two CTAs share an SM: twice the warps in flight with half the ring each,
-      // which suits a kernel bound by the per-warp chain of copy issue, wait and FMAs (measured on
-      // the 200-adapter down_proj: 45.8 us against 49.8 us with depth 4)
-      const int shrink_depth = T <= 64 ? 2 : (p->opt_shrink_depth == 4 ? 4 : 2);
-      const int cta_cap = shrink_depth == 2 && T > 64 ? 2 * p->sms : p->sms;
-      const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : (overlapped ? 1 : 4 * 8 * cta_cap);
-      // at most T token blocks x (R / 8) row groups x K chunks warp items, eight warps per CTA
-      const int n_ksteps = (h_in + kShrinkStepElems - 1) / kShrinkStepElems;
-      const int max_chunks = target == 1 ? 1 : std::max(1, std::min(kMaxZSplits, n_ksteps / 4));
-      const int max_items = std::min(T, p->cfg.n_slots) * (R / 8) * max_chunks;
-      const int grid = std::max(1, std::min(cta_cap - 1, (max_items + 7) / 8)) + 1;  // + the publishing CTA
-      CUtensorMap ma, mx, md;
-      // A rows: bfloat16, or for a pool that keeps A in Q8_0 two planes per slot: the signed bytes
-      // [R_pad][h_in] (taken as 16-bit elements: 128 per K step) and the half-precision block scales
-      // [R_pad][h_in / 32] (8 per K step); both planes have the slot's byte stride
-      int rc;
-      if (p->a_q8) {
-        const uint64_t slot_bytes = p->a_block * 2;
-        rc = get_tmap(p, &ma, p->A_pool, h_in / 2, R, p->cfg.n_slots, 8, kShrinkStepElems / 2, h_in, slot_bytes);
-        if (rc) return rc;
-        rc = get_tmap(p, &md, reinterpret_cast<const uint8_t *>(p->A_pool) + static_cast<size_t>(R) * h_in, h_in / 32, R,
-                      p->cfg.n_slots, 8, kShrinkStepElems / 32, h_in / 16, slot_bytes);
-      } else {
-        rc = get_tmap(p, &ma, p->A_pool, h_in, R, p->cfg.n_slots, 8, kShrinkStepElems);
-        md = ma;
-      }
-      if (rc) return rc;
-      rc = get_tmap(p, &mx, x, h_in, T, 0, 1, kShrinkStepElems);
-      if (rc) return rc;
-      CUDA_TRY(launch_decode_shrink(ma, md, mx, ids_in, p->slots_dev, plan->pv, p->zws, p->group_counters,
-                                    T, h_in, R, p->cfg.n_slots, p->cfg.max_tokens, target, grid,
-                                    p->status_dev, pdl_first, p->a_q8, shrink_depth, stream));
-      ++launches;
-    }
+      return 0;
+    };
     int N = 32;  // tokens on the UMMA N axis: a power of two so that the cluster's owners get
     while (N < T) N <<= 1;  // equal power-of-two column blocks
     const int row_tiles = (h_out + kTileM - 1) / kTileM;
@@ -1007,16 +1017,66 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
     rc = get_tmap(p, &mb, p->B_pool, R, h_out, p->cfg.n_slots, kTileM);
     if (rc) return rc;
     const int grid = row_tiles * splits;
-    {
+    // Small batches in one launch: the shrink runs on the idle builder warps of the base product's CTAs
+    // and on spare CTAs in front of them (SMs the grid leaves empty), and the owners of the cluster
+    // reduction wait for its arrival counter.  CTAs of one grid wait for one another here, so every
+    // cluster of the launch must be resident at once: checked against the device's occupancy figure.
+    bool fused = false;
+    if (getenv("EDGELORA_LOG"))
+      fprintf(stderr, "edgelora: decode T %d N %d splits %d grid %d expand_in_reduce %d ctas_per_sm %d\n", T, N, splits,
+              grid, g.expand_in_reduce, ctas_per_sm);
+    // (Calls that may overlap the call before them keep the two launches: a one-launch grid holds every
+    // SM until its last CTA is done, so consecutive calls cannot overlap; measured on 4096 -> 4096,
+    // T = 32: 17.0 us per step in one launch against 9.7 us in two when the calls are independent, and
+    // 16.9 against 19.7 us when each call waits for the one before.)
+    if (p->opt_fused_decode && !pdl_first && g.expand_in_reduce && T <= 64 && T <= kGatherMinT && ids_dev &&
+        !p->a_q8 && h_in % 8 == 0) {
+      FusedDecode f{};
+      // room behind the ring for the B_a rows and z of an owner's tokens, when it fits
+      const size_t stage_extra = static_cast<size_t>(N / splits) * (kTileM * R * 2 + R * 4);
+      f.b_stage = smem_for(g.stages, N, static_cast<int>(stage_extra)) <= kSmemBudget ? 1 : 0;
+      const size_t smem = smem_for(g.stages, N, f.b_stage ? static_cast<int>(stage_extra) : 0);
+      const uint64_t key = (static_cast<uint64_t>(splits) << 32) | static_cast<uint64_t>(smem);
+      if (p->fused_key != key) {
+        p->fused_key = key;
+        p->fused_max_ctas = gemm_fused_max_ctas(splits, smem);
+      }
+      const int spare = std::max(0, std::min(p->fused_max_ctas - grid, 32) / splits * splits);
+      if (spare > 0) {  // every CTA resident at once, and a spare CTA to publish the routing plan
+        const int n_teams = 2 * spare + grid;
+        const int n_ksteps = (h_in + kShrinkStepElems - 1) / kShrinkStepElems;
+        int ks = std::max(1, std::min(kMaxZSplits, n_ksteps / 4));
+        while (ks > 1 && T * (R / 8) * ks > 2 * n_teams) ks >>= 1;
+        f.n_ctas = spare;
+        f.ks = ks;
+        f.x_wait = 1;  // x may be the output of the call before this one
+        f.A_pool = p->A_pool;
+        f.x = x;
+        f.z = p->zws;
+        f.sync = p->group_counters + kDecodeMaxT * 8 + 8;
+        f.pv = plan->pv;
+        ProfScope ps(p, 3, stream);
+        CUDA_TRY(launch_gemm_fused(mr, mc, g, f, smem, p->opt_pdl != 0, stream));
+        ++launches;
+        fused = true;
+        p->last_info[2] = grid + spare;
+        p->last_info[3] = splits;
+      }
+    }
+    if (!fused) {
+      rc = launch_shrink();
+      if (rc) return rc;
+    }
+    if (!fused) {
       ProfScope ps(p, 3, stream);
       // With one CTA per SM the base product cannot start beside the shrink (both fill an SM's
       // shared memory), and an early launch then only costs: measured 178 vs 122 us per step on
       // the 14336 -> 4096, T = 256 workload.
       CUDA_TRY(launch_gemm(mr, mc, mb, g, grid, smem_for(g.stages, N), pdl && ctas_per_sm == 2, stream));
       ++launches;
+      p->last_info[2] = grid;
+      p->last_info[3] = splits;
     }
-    p->last_info[2] = grid;
-    p->last_info[3] = splits;
   } else {
     // ---------------------------------------------------------------- prefill
     if (ids_dev) {

@@ -81,7 +81,9 @@ struct edgelora_pool {
   uint32_t *status_dev = nullptr;
   std::vector<TmapEntry> tmaps;
   size_t tmap_next = 0;
-  int opt_regime = 0, opt_profile = 0, opt_pdl = 1;
+  int opt_regime = 0, opt_profile = 0, opt_pdl = 1, opt_fused_decode = 1;
+  uint64_t fused_key = 0;  // launch shape the occupancy answer below belongs to
+  int fused_max_ctas = 0;
   long long wait_cycles = edgelora::ptx::kWaitLimitCycles;
   int64_t last_info[8] = {0};
   int64_t total_launches = 0;

@@ -72,6 +72,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity,
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }
+// Untiled bulk copy global -> this CTA's shared memory (no multicast): both addresses 16-byte
+// aligned, bytes a multiple of 16; completes on the mbarrier like a tiled load.
+__device__ __forceinline__ void bulk_load_1d(void *smem_dst, const void *gmem_src, uint32_t bytes, uint64_t *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(smem_dst)),
+               "l"(reinterpret_cast<uint64_t>(gmem_src)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
 // 2D tiled load, no multicast.  c0 is the innermost (contiguous) coordinate.
 __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *m, uint64_t *bar,
                                             int32_t c0, int32_t c1) {

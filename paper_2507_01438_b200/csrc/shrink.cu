@@ -5,6 +5,7 @@
 // tiles of the tile kernel (gemm.cu).
 #include <cuda_fp16.h>
 
+#include "decode_route.cuh"
 #include "internal.cuh"
 #include "launch.cuh"
 #include "ptx.cuh"
@@ -34,35 +35,6 @@ __device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
   f[2] = ptx::bf16_lo(v.y); f[3] = ptx::bf16_hi(v.y);
   f[4] = ptx::bf16_lo(v.z); f[5] = ptx::bf16_hi(v.z);
   f[6] = ptx::bf16_lo(v.w); f[7] = ptx::bf16_hi(v.w);
-}
-
-// Exclusive prefix sum of one int per thread over the 256-thread CTA; `total` gets the sum.
-__device__ __forceinline__ int block_scan_256(int v, int *wt /* smem[9] */, int &total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int incl = v;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const int o = __shfl_up_sync(0xffffffffu, incl, d);
-    if (lane >= d) incl += o;
-  }
-  if (lane == 31) wt[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    const int w = lane < 8 ? wt[lane] : 0;
-    int wi = w;
-#pragma unroll
-    for (int d = 1; d < 8; d <<= 1) {
-      const int o = __shfl_up_sync(0xffffffffu, wi, d);
-      if (lane >= d) wi += o;
-    }
-    if (lane < 8) wt[lane] = wi - w;
-    if (lane == 7) wt[8] = wi;
-  }
-  __syncthreads();
-  const int res = wt[warp] + incl - v;
-  total = wt[8];
-  __syncthreads();
-  return res;
 }
 
 constexpr int kDsMaxDepth = 5;                      // ring stages per warp: up to 5, or 2 for small batches
@@ -296,59 +268,7 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
 
   // ---- the last CTA publishes the plan in canonical order (ids ascending, -1 first): everything
   // is worked out in shared memory and registers first, the stores come after the wait
-  if (publisher) {
-    const uint32_t key = (static_cast<uint32_t>(a + 1) << 16) | static_cast<uint32_t>(tid);
-    int rp = 0;
-    if (tid < T)
-      for (int u = 0; u < T; ++u)
-        rp += (((static_cast<uint32_t>(s_id[u] + 1) << 16) | static_cast<uint32_t>(u)) < key) ? 1 : 0;
-    __syncthreads();  // every thread is done with s_cnt as a counter
-    if (tid < T) s_cnt[rp] = tid;  // s_cnt now holds the tokens in canonical order
-    __syncthreads();
-    int ida = -2, tok = 0;
-    bool head = false;
-    if (tid < T) {
-      tok = s_cnt[tid];
-      ida = s_id[tok];
-      head = tid == 0 || s_id[s_cnt[tid - 1]] != ida;
-    }
-    int n_groups;
-    const int gi = block_scan_256(head ? 1 : 0, s_wt, n_groups);
-    const int has_base = (T > 0 && s_id[s_cnt[0]] < 0) ? 1 : 0;
-    const bool shead = tid < T && (tid == 0 || s_id[tid - 1] != a);
-    int n_segs;
-    const int si = block_scan_256(shead ? 1 : 0, s_wt, n_segs);
-
-    ptx::pdl_wait_prior_grids();
-    if (any_bad && tid == 0) atomicOr(pv.status, EDGELORA_STATUS_BAD_ADAPTER_ID);
-    if (tid < T) {
-      pv.ids_valid[tid] = a;
-      pv.perm[tid] = tok;
-      pv.perm_short[tid] = tok;
-      if (head) {
-        pv.group_start[gi] = tid;
-        pv.gs_short[gi] = tid;
-        pv.group_adapter[gi] = ida;
-        if (ida >= 0) pv.lg_adapter[gi - has_base] = ida;
-      }
-      pv.tok_seg[tid] = si + (shead ? 1 : 0) - 1;
-      if (shead) {
-        pv.seg_start[si] = tid;
-        pv.seg_adapter[si] = a;
-      }
-    }
-    if (tid == 0) {
-      pv.group_start[n_groups] = T;
-      pv.gs_short[n_groups] = T;
-      pv.seg_start[n_segs] = T;
-      pv.counts[0] = n_groups;
-      pv.counts[1] = n_segs;
-      pv.counts[2] = 0;
-      pv.counts[3] = T;
-      pv.counts[4] = n_groups - has_base;
-      pv.counts[5] = KS;
-    }
-  }
+  if (publisher) publish_decode_plan(pv, a, T, any_bad, KS, s_id, s_cnt, s_wt);
 
   // ---- per-warp work items, no CTA-wide synchronisation from here on
   const int n_items = NB * KS * n_rgn;
