@@ -48,13 +48,16 @@ typedef enum {
   EDGELORA_ERR_SLOT_EMPTY = -7,
   EDGELORA_ERR_TIMEOUT = -8,
   EDGELORA_ERR_TOO_MANY_TOKENS = -9,
-  EDGELORA_ERR_CACHE_FULL = -10
+  EDGELORA_ERR_CACHE_FULL = -10,
+  EDGELORA_ERR_BOUNDS = -11
 } edgelora_status;
 
 /* Bits of the device status word returned by edgelora_pool_sync_status(). */
 #define EDGELORA_STATUS_BAD_ADAPTER_ID 0x1u /* an id outside [-1, n_slots) was seen     */
 #define EDGELORA_STATUS_SLOT_EMPTY 0x2u     /* an id named a slot with nothing loaded   */
 #define EDGELORA_STATUS_TIMEOUT 0x4u        /* a bounded in-kernel wait gave up         */
+#define EDGELORA_STATUS_BOUNDS 0x8u         /* checked build only: a kernel met an index outside
+                                               its array and skipped the access            */
 
 typedef struct edgelora_pool edgelora_pool_t; /* opaque, owned by the library */
 typedef struct edgelora_plan edgelora_plan_t; /* opaque, owned by the library */
@@ -293,6 +296,21 @@ int edgelora_pool_set_option(edgelora_pool_t *pool, int32_t option, int32_t valu
  * Only with EDGELORA_OPT_WAIT_CYCLES lowered to at most 16384 (16 M cycles); otherwise
  * EDGELORA_ERR_INVALID_ARG and nothing is launched. */
 int edgelora_pool_selftest_wait(edgelora_pool_t *pool, void *stream);
+
+/* The checked build of the library (compiled with -DEDGELORA_CHECKED, for finding memory errors
+ * where no memory-checking tool can be run; the paper has no counterpart).  It differs in two ways.
+ * The kernels test the indices they read from device memory (adapter ids in the routing plan's lists,
+ * token indices, tile descriptors, ranks) against their arrays' sizes; a failed test skips the
+ * access and raises EDGELORA_STATUS_BOUNDS, which edgelora_pool_sync_status reports as
+ * EDGELORA_ERR_BOUNDS.  And every device buffer the library allocates has 256 guard bytes of a fixed
+ * value in front and behind.
+ *   edgelora_build_is_checked  1 for the checked build, 0 for the normal one.
+ *   edgelora_check_guards      synchronises the current device and compares every guard zone on it
+ *                              with its value: EDGELORA_OK, or EDGELORA_ERR_BOUNDS when a kernel or
+ *                              copy wrote outside a buffer.  The normal build has no zones and
+ *                              returns EDGELORA_OK. */
+int edgelora_build_is_checked(void);
+int edgelora_check_guards(void);
 
 /* Launch bookkeeping for measurement.  info_out[0] = kernels launched by the last
  * edgelora_lora_linear call, [1] = regime used (1 decode, 2 prefill), [2] = grid of the

@@ -12,12 +12,16 @@ from typing import Optional
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libedgelora.so")
+# EDGELORA_CHECKED=1 in the environment selects the checked build of the library (index tests in the
+# kernels, guard zones around its device buffers; `python -m paper_2507_01438_b200.build --checked`)
+LIB_PATH = os.path.join(_HERE, "libedgelora_checked.so" if os.environ.get("EDGELORA_CHECKED") == "1"
+                        else "libedgelora.so")
 
 OK = 0
 ERR_INVALID_ARG, ERR_BAD_SLOT, ERR_RANK_TOO_LARGE, ERR_ARENA_TOO_SMALL = -1, -2, -3, -4
 ERR_CUDA, ERR_BAD_ADAPTER_ID, ERR_SLOT_EMPTY, ERR_TIMEOUT, ERR_TOO_MANY_TOKENS = -5, -6, -7, -8, -9
-STATUS_BAD_ADAPTER_ID, STATUS_SLOT_EMPTY, STATUS_TIMEOUT = 0x1, 0x2, 0x4
+ERR_CACHE_FULL, ERR_BOUNDS = -10, -11
+STATUS_BAD_ADAPTER_ID, STATUS_SLOT_EMPTY, STATUS_TIMEOUT, STATUS_BOUNDS = 0x1, 0x2, 0x4, 0x8
 OPT_REGIME, OPT_PROFILE, OPT_PDL, OPT_DECODE_SPLITS, OPT_SHRINK_ITEMS, OPT_WAIT_CYCLES = 1, 2, 3, 4, 5, 6
 OPT_GATHER_SPLITS, OPT_GATHER_MIN_T, OPT_SHRINK_DEPTH, OPT_FUSED_DECODE = 7, 8, 9, 10
 KERNEL_NAMES = ("plan", "shrink_small_decode", "shrink_tiles", "base_gemm")
@@ -37,6 +41,7 @@ EXPORTS = (
     "edgelora_siteset_run_host", "edgelora_siteset_plan",
     "edgelora_cache_prefill", "edgelora_pool_load_slot_q8", "edgelora_pool_load_slot_pinned", "edgelora_batcher_create", "edgelora_batcher_destroy", "edgelora_batcher_submit",
     "edgelora_batcher_next_batch", "edgelora_batcher_complete_step", "edgelora_batcher_finished",
+    "edgelora_build_is_checked", "edgelora_check_guards",
 )
 
 
@@ -108,6 +113,8 @@ def lib() -> ctypes.CDLL:
     L.edgelora_siteset_plan.argtypes = [vp, cp(vp)]
     L.edgelora_plan_sync_status.argtypes = [vp, vp, cp(ctypes.c_uint32)]
     L.edgelora_pool_selftest_wait.argtypes = [vp, vp]
+    L.edgelora_build_is_checked.argtypes = []
+    L.edgelora_check_guards.argtypes = []
     L.edgelora_pool_sync_status.argtypes = [vp, cp(ctypes.c_uint32)]
     L.edgelora_pool_set_option.argtypes = [vp, i32, i32]
     L.edgelora_pool_last_launch.argtypes = [vp, vp]
@@ -346,6 +353,16 @@ def edgelora_plan_sync_status(plan, stream=None):
     if rc == ERR_CUDA or rc == ERR_INVALID_ARG:
         raise EdgeLoraError(rc, "plan_sync_status")
     return rc, bits.value
+
+
+def edgelora_build_is_checked() -> bool:
+    return bool(lib().edgelora_build_is_checked())
+
+
+def edgelora_check_guards() -> int:
+    """EDGELORA_OK, or ERR_BOUNDS when something wrote outside one of the library's device buffers
+    (checked build; the normal build has no guard zones and always answers OK)."""
+    return lib().edgelora_check_guards()
 
 
 def edgelora_pool_selftest_wait(pool, stream=None) -> int:

@@ -143,6 +143,11 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams &p, int32_t til
       c.row_r = p.sgmv_tiles[4 * st + 0];
       c.nrows = p.sgmv_tiles[4 * st + 1];
       c.slot = p.sgmv_tiles[4 * st + 2];
+      if (!EL_CHECK(p.status, c.row_r >= 0 && c.nrows >= 0 && c.row_r + c.nrows <= p.T && c.slot >= 0 && c.slot < p.n_slots, 4)) {
+        c.row_r = 0;  // a tile of no rows: computed, nothing written
+        c.nrows = 0;
+        c.slot = 0;
+      }
     } else {
       const int n_gt = gather_tiles(p);
       const int gsp = gather_splits(p, n_gt, gridDim.x);
@@ -237,6 +242,10 @@ __device__ __forceinline__ void st_cluster_f32x4(uint32_t addr, float a, float b
 // the partial planes are added in order, values at or past the true rank forced to zero.
 __device__ __forceinline__ void load_z_packed(const GemmParams &p, int32_t t, int32_t rank,
                                               uint4 (&out)[8]) {
+  if (!EL_CHECK(p.status, rank <= p.R_pad && t >= 0 && t < p.max_tokens, 3)) {
+    rank = 0;  // all zeros, read from row 0
+    t = 0;
+  }
   const int nch = p.R_pad >> 3;
   const float *zt = p.zws + static_cast<size_t>(t) * p.R_pad;
   const size_t plane = static_cast<size_t>(p.max_tokens) * p.R_pad;
@@ -314,7 +323,10 @@ __device__ __forceinline__ bool gather_pass_copies(const GemmParams &jp, const T
       my_quad = item - tc.ng;
 #pragma unroll
       for (int i = 0; i < 4; ++i)  // rows past the pass's last token repeat it (they land in unused columns)
+      {
         tok[i] = jp.perm_short[tc.tok0 + t0 + min(my_quad * 4 + i, n - 1)];
+        if (!EL_CHECK(jp.status, tok[i] >= 0 && tok[i] < jp.T, 5)) tok[i] = 0;
+      }
     }
   }
   for (int32_t kb = tc.kb0; kb < tc.kb1; ++kb) {
@@ -701,6 +713,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         const LoraList ll = lora_list(p, tc, s_lg, s_nlg);
         for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
           const int32_t a = ll.list[e];
+          if (!EL_CHECK(p.status, a >= 0 && a < p.n_slots, 1)) continue;
           if (p.mode != kModeDecode && p.slots[a].rank <= 0) continue;
           if (!wait_empty()) {
             ok = false;
@@ -807,6 +820,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
           const LoraList ll = lora_list(p, tc, s_lg, s_nlg);
           for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
             const int32_t a = ll.list[e];
+            if (!EL_CHECK(p.status, a >= 0 && a < p.n_slots, 1)) continue;
             if (p.mode != kModeDecode && p.slots[a].rank <= 0) continue;
             if (!ptx::mbar_wait(&full_bar[stage], phase, wl) ||
                 !ptx::mbar_wait(&zfull_bar[stage], (zphase >> stage) & 1u, wl) || *abort_flag) {
@@ -997,6 +1011,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
           for (int q = 0; q < 8; ++q) {
             const int c = q * 32 + lane;
             tok[q] = c < n ? jp.perm_short[tc.tok0 + t0 + c] : 0;
+            if (!EL_CHECK(jp.status, tok[q] >= 0 && tok[q] < jp.max_tokens, 6)) tok[q] = 0;
           }
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                                  acc * static_cast<uint32_t>(p.acc_cols);
@@ -1331,6 +1346,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         if (kMinBlocks == 1) id_hi = s_vid[btid + 128];  // the two-per-SM variant runs with BN <= 128
       } else if (tok0 + btid < p.T) {
         id_lo = p.ids_valid[tok0 + btid];
+        if (!EL_CHECK(p.status, id_lo >= -1 && id_lo < p.n_slots, 2)) id_lo = -1;
       }
       uint4 z_lo[8], z_hi[8];
       if (ll.e0 < ll.e1) {
@@ -1339,6 +1355,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       }
       for (int32_t e = ll.e0; e < ll.e1; e += ll.de) {
         const int32_t a = ll.list[e];
+        if (!EL_CHECK(p.status, a >= 0 && a < p.n_slots, 1)) continue;
         if (p.mode != kModeDecode && p.slots[a].rank <= 0) continue;
         const uint32_t stage = count % nstages;
         ++count;

@@ -20,6 +20,22 @@ constexpr int kMaxZSplits = 16;    // partial z planes (K splits of the shrink);
 constexpr int kShrinkThreads = 256;
 constexpr int kShrinkStepElems = 256;  // K elements of one shrink step (512 bytes of a row)
 
+// Checked build: EL_CHECK(status, cond, site) is `cond`, and when it is false raises
+// EDGELORA_STATUS_BOUNDS in the status word and records `site` (a number naming the test) in the
+// word after it, first failure only; the caller skips the access.  In the normal build it is `true`
+// and costs nothing.  Every role of a kernel evaluates the same tests on the same data, so a skipped
+// K block is skipped by all of them.
+#ifdef EDGELORA_CHECKED
+__device__ __forceinline__ bool el_check_fail(uint32_t *status, uint32_t site) {
+  atomicOr(status, EDGELORA_STATUS_BOUNDS);
+  atomicCAS(status + 1, 0u, site);
+  return false;
+}
+#define EL_CHECK(status, cond, site) ((cond) ? true : ::edgelora::el_check_fail((status), (site)))
+#else
+#define EL_CHECK(status, cond, site) (true)
+#endif
+
 // One row of the slot table (paper Section 3.3: one fixed block per resident adapter).
 struct SlotRow {
   int32_t rank;        // 0 = empty

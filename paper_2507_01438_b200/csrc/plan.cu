@@ -134,7 +134,8 @@ plan_kernel(const int32_t *__restrict__ ids, int32_t T, int32_t n_slots, PlanVie
   });
   for (int t = tid; t < T; t += kPlanThreads) {
     const int s = pv.tok_seg[t];
-    pv.perm[out_start[inv[s]] + (t - pv.seg_start[s])] = t;
+    const int pos = out_start[inv[s]] + (t - pv.seg_start[s]);
+    if (EL_CHECK(pv.status, s >= 0 && s < n_segs && pos >= 0 && pos < T, 30)) pv.perm[pos] = t;
   }
   auto is_ghead = [&](int j) { return (j == 0 || (keys[j] >> 16) != (keys[j - 1] >> 16)) ? 1 : 0; };
   const int has_base = (n_segs > 0 && (keys[0] >> 16) == 0) ? 1 : 0;  // the group of id -1 sorts first
@@ -172,7 +173,8 @@ plan_kernel(const int32_t *__restrict__ ids, int32_t T, int32_t n_slots, PlanVie
   for (int t = tid; t < T; t += kPlanThreads) {
     const int s = pv.tok_seg[t];
     const int len = pv.seg_start[s + 1] - pv.seg_start[s];
-    if (all_short || len < kSegMin) pv.perm_short[out_start[inv[s]] + (t - pv.seg_start[s])] = t;
+    const int pos = out_start[inv[s]] + (t - pv.seg_start[s]);
+    if ((all_short || len < kSegMin) && EL_CHECK(pv.status, pos >= 0 && pos < T, 31)) pv.perm_short[pos] = t;
   }
   if (tid == 0) {
     pv.gs_short[n_groups] = n_short;

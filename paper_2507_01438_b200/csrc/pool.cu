@@ -13,6 +13,7 @@
 #include <utility>
 #include <vector>
 
+#include "guard.h"
 #include "pool.h"
 
 using namespace edgelora;
@@ -166,7 +167,7 @@ int plan_alloc(edgelora_plan *pl) {
   const size_t n_mt = (mt + kTileM - 1) / kTileM;
   const size_t ints = 7 * mt + 4 * (mt + 1) + 4 * static_cast<size_t>(max_tiles) + (n_mt + 1) +
                       n_mt * kTileM + 8 + 4;
-  CUDA_TRY(cudaMalloc(&pl->block, ints * 4));
+  CUDA_TRY(el_malloc(&pl->block, ints * 4));
   CUDA_TRY(cudaMemset(pl->block, 0, ints * 4));
   int32_t *q = static_cast<int32_t *>(pl->block);
   PlanView &v = pl->pv;
@@ -205,6 +206,8 @@ const char *edgelora_strerror(int code) {
     case EDGELORA_ERR_BAD_ADAPTER_ID: return "an adapter id outside [-1, n_slots) was seen (token computed base-only)";
     case EDGELORA_ERR_SLOT_EMPTY: return "an adapter id named an empty slot (token computed base-only)";
     case EDGELORA_ERR_TIMEOUT: return "a bounded in-kernel wait gave up";
+    case EDGELORA_ERR_BOUNDS:
+      return "checked build: a kernel met an index outside its array, or a guard zone around a device buffer was overwritten";
     case EDGELORA_ERR_TOO_MANY_TOKENS: return "T exceeds max_tokens (or max_tokens exceeds 32768)";
     case EDGELORA_ERR_CACHE_FULL: return "every block of the adapter cache is held by a running request";
     default: return "unknown error";
@@ -229,7 +232,7 @@ int edgelora_plan_create(int32_t max_tokens, int32_t n_slots, edgelora_plan_t **
   pl->n_slots = n_slots;
   int rc = plan_alloc(pl);
   if (rc != EDGELORA_OK) {
-    if (pl->block) cudaFree(pl->block);
+    if (pl->block) el_free(pl->block);
     delete pl;
     return rc;
   }
@@ -241,7 +244,7 @@ int edgelora_plan_create(int32_t max_tokens, int32_t n_slots, edgelora_plan_t **
 int edgelora_plan_destroy(edgelora_plan_t *plan) {
   if (!plan) return EDGELORA_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
-  if (plan->block) cudaFree(plan->block);
+  if (plan->block) el_free(plan->block);
   delete plan;
   return EDGELORA_OK;
 }
@@ -338,14 +341,14 @@ int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool
   if (cfg->arena_dev) {
     p->arena = static_cast<uint8_t *>(cfg->arena_dev);
   } else {
-    POOL_TRY(cudaMalloc(&p->arena, need));
+    POOL_TRY(el_malloc(&p->arena, need));
     p->owns_arena = true;
   }
   p->A_pool = reinterpret_cast<uint16_t *>(p->arena);
   p->B_pool = p->A_pool + p->a_block * cfg->n_slots;
-  POOL_TRY(cudaMalloc(&p->slots_dev, sizeof(SlotRow) * cfg->n_slots));
+  POOL_TRY(el_malloc(&p->slots_dev, sizeof(SlotRow) * cfg->n_slots));
   POOL_TRY(cudaMemset(p->slots_dev, 0, sizeof(SlotRow) * cfg->n_slots));
-  POOL_TRY(cudaMalloc(&p->status_dev, 16));
+  POOL_TRY(el_malloc(&p->status_dev, 16));
   POOL_TRY(cudaMemset(p->status_dev, 0, 16));
   // room for a block in its own layout or, for Q8_0 loads, A and B as 8-bit blocks (+ alignment)
   const size_t b_q8_bytes = static_cast<size_t>(cfg->h_out) * ((p->R_pad + 31) / 32) * 34;
@@ -358,8 +361,8 @@ int edgelora_pool_create(const edgelora_pool_config *cfg, edgelora_pool_t **pool
   POOL_TRY(cudaEventCreateWithFlags(&p->load_ev, cudaEventDisableTiming));
   POOL_TRY(cudaEventCreateWithFlags(&p->use_ev, cudaEventDisableTiming));
   // partial planes [0, kMaxZSplits) plus the final plane of the decode shrink
-  POOL_TRY(cudaMalloc(&p->zws, sizeof(float) * (kMaxZSplits + 1) * static_cast<size_t>(p->cfg.max_tokens) * p->R_pad));
-  POOL_TRY(cudaMalloc(&p->group_counters, sizeof(int32_t) * (kDecodeMaxT * 8 + 32)));
+  POOL_TRY(el_malloc(&p->zws, sizeof(float) * (kMaxZSplits + 1) * static_cast<size_t>(p->cfg.max_tokens) * p->R_pad));
+  POOL_TRY(el_malloc(&p->group_counters, sizeof(int32_t) * (kDecodeMaxT * 8 + 32)));
   POOL_TRY(cudaMemset(p->group_counters, 0, sizeof(int32_t) * (kDecodeMaxT * 8 + 32)));
   POOL_TRY(gemm_set_smem_limit(kSmemBudget));
   POOL_TRY(shrink_set_smem_limit());
@@ -377,9 +380,9 @@ int edgelora_pool_destroy(edgelora_pool_t *p) {
   if (!p) return EDGELORA_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
   if (p->plan) edgelora_plan_destroy(p->plan);
-  if (p->owns_arena && p->arena) cudaFree(p->arena);
-  if (p->slots_dev) cudaFree(p->slots_dev);
-  if (p->status_dev) cudaFree(p->status_dev);
+  if (p->owns_arena && p->arena) el_free(p->arena);
+  if (p->slots_dev) el_free(p->slots_dev);
+  if (p->status_dev) el_free(p->status_dev);
   for (auto &sb : p->staging) {
     if (sb.host) cudaFreeHost(sb.host);
     if (sb.done) cudaEventDestroy(sb.done);
@@ -387,9 +390,9 @@ int edgelora_pool_destroy(edgelora_pool_t *p) {
   if (p->side) cudaStreamDestroy(p->side);
   if (p->load_ev) cudaEventDestroy(p->load_ev);
   if (p->use_ev) cudaEventDestroy(p->use_ev);
-  if (p->zws) cudaFree(p->zws);
-  if (p->q8_dev) cudaFree(p->q8_dev);
-  if (p->group_counters) cudaFree(p->group_counters);
+  if (p->zws) el_free(p->zws);
+  if (p->q8_dev) el_free(p->q8_dev);
+  if (p->group_counters) el_free(p->group_counters);
   for (auto &r : p->prof) {
     cudaEventDestroy(r.start);
     cudaEventDestroy(r.stop);
@@ -397,13 +400,13 @@ int edgelora_pool_destroy(edgelora_pool_t *p) {
   if (p->hx) cudaFreeHost(p->hx);
   if (p->hy) cudaFreeHost(p->hy);
   if (p->hids) cudaFreeHost(p->hids);
-  if (p->dx) cudaFree(p->dx);
-  if (p->dy) cudaFree(p->dy);
-  if (p->dids) cudaFree(p->dids);
+  if (p->dx) el_free(p->dx);
+  if (p->dy) el_free(p->dy);
+  if (p->dids) el_free(p->dids);
   for (int b = 0; b < 2; ++b) {
-    if (p->pdx[b]) cudaFree(p->pdx[b]);
-    if (p->pdy[b]) cudaFree(p->pdy[b]);
-    if (p->pdids[b]) cudaFree(p->pdids[b]);
+    if (p->pdx[b]) el_free(p->pdx[b]);
+    if (p->pdy[b]) el_free(p->pdy[b]);
+    if (p->pdids[b]) el_free(p->pdids[b]);
     if (p->ev_in[b]) cudaEventDestroy(p->ev_in[b]);
     if (p->ev_done[b]) cudaEventDestroy(p->ev_done[b]);
     if (p->ev_out[b]) cudaEventDestroy(p->ev_out[b]);
@@ -520,7 +523,7 @@ int edgelora_pool_load_slot_q8(edgelora_pool_t *p, int32_t slot, int32_t rank, f
   const size_t b_off = (a_bytes + 15) & ~static_cast<size_t>(15);
   const size_t scratch = static_cast<size_t>(p->cfg.max_rank) * (h_in / 32) * 34 + 16 +
                          static_cast<size_t>(h_out) * ((p->cfg.max_rank + 31) / 32) * 34;
-  if (!p->q8_dev) CUDA_TRY(cudaMalloc(&p->q8_dev, scratch));
+  if (!p->q8_dev) CUDA_TRY(el_malloc(&p->q8_dev, scratch));
   StagingBuf &sb = p->staging[p->next_staging];
   p->next_staging = (p->next_staging + 1) % kStagingBuffers;
   if (sb.in_flight) {
@@ -695,13 +698,21 @@ int edgelora_pool_sync_status(edgelora_pool_t *p, uint32_t *bits_out) {
   CUDA_TRY(cudaMemcpy(&a, p->status_dev, 4, cudaMemcpyDeviceToHost));
   CUDA_TRY(cudaMemcpy(&b, p->plan->pv.status, 4, cudaMemcpyDeviceToHost));
   CUDA_TRY(cudaMemset(p->status_dev, 0, 4));
-  CUDA_TRY(cudaMemset(p->plan->pv.status, 0, 4));
+  CUDA_TRY(cudaMemset(p->plan->pv.status, 0, 8));
   const uint32_t bits = a | b;
   if (bits_out) *bits_out = bits;
   // a wait that ran out can leave arrival counters between their values: nothing is in flight now
   if (bits & EDGELORA_STATUS_TIMEOUT)
     CUDA_TRY(cudaMemset(p->group_counters, 0, sizeof(int32_t) * (kDecodeMaxT * 8 + 32)));
+  if (bits & EDGELORA_STATUS_BOUNDS) {  // checked build: which test failed first
+    uint32_t site = 0;
+    CUDA_TRY(cudaMemcpy(&site, p->status_dev + 1, 4, cudaMemcpyDeviceToHost));
+    CUDA_TRY(cudaMemset(p->status_dev + 1, 0, 4));
+    snprintf(g_last_error, sizeof g_last_error, "a kernel's index test failed (test %u)", site);
+    return EDGELORA_ERR_BOUNDS;
+  }
   if (bits & EDGELORA_STATUS_TIMEOUT) return EDGELORA_ERR_TIMEOUT;
+  if (edgelora_check_guards() != EDGELORA_OK) return EDGELORA_ERR_BOUNDS;  // always intact in the normal build
   if (bits & EDGELORA_STATUS_BAD_ADAPTER_ID) return EDGELORA_ERR_BAD_ADAPTER_ID;
   if (bits & EDGELORA_STATUS_SLOT_EMPTY) return EDGELORA_ERR_SLOT_EMPTY;
   return EDGELORA_OK;
@@ -715,6 +726,7 @@ int edgelora_plan_sync_status(edgelora_plan_t *plan, void *stream, uint32_t *bit
   CUDA_TRY(cudaMemcpy(&bits, plan->pv.status, 4, cudaMemcpyDeviceToHost));
   CUDA_TRY(cudaMemset(plan->pv.status, 0, 4));
   if (bits_out) *bits_out = bits;
+  if (bits & EDGELORA_STATUS_BOUNDS) return EDGELORA_ERR_BOUNDS;
   if (bits & EDGELORA_STATUS_TIMEOUT) return EDGELORA_ERR_TIMEOUT;
   if (bits & EDGELORA_STATUS_BAD_ADAPTER_ID) return EDGELORA_ERR_BAD_ADAPTER_ID;
   if (bits & EDGELORA_STATUS_SLOT_EMPTY) return EDGELORA_ERR_SLOT_EMPTY;
@@ -1203,9 +1215,9 @@ int edgelora_lora_linear_host(edgelora_pool_t *p, const void *W_dev, const uint1
     CUDA_TRY(cudaMallocHost(&p->hx, mt * p->cfg.h_in * 2));
     CUDA_TRY(cudaMallocHost(&p->hy, mt * p->cfg.h_out * 2));
     CUDA_TRY(cudaMallocHost(&p->hids, mt * 4));
-    CUDA_TRY(cudaMalloc(&p->dx, mt * p->cfg.h_in * 2));
-    CUDA_TRY(cudaMalloc(&p->dy, mt * p->cfg.h_out * 2));
-    CUDA_TRY(cudaMalloc(&p->dids, mt * 4));
+    CUDA_TRY(el_malloc(&p->dx, mt * p->cfg.h_in * 2));
+    CUDA_TRY(el_malloc(&p->dy, mt * p->cfg.h_out * 2));
+    CUDA_TRY(el_malloc(&p->dids, mt * 4));
   }
   const size_t xb = static_cast<size_t>(T) * p->cfg.h_in * 2, yb = static_cast<size_t>(T) * p->cfg.h_out * 2;
   memcpy(p->hx, x_host, xb);
@@ -1233,9 +1245,9 @@ int edgelora_lora_linear_host_async(edgelora_pool_t *p, const void *W_dev, const
     CUDA_TRY(cudaStreamCreateWithFlags(&p->h2d_stream, cudaStreamNonBlocking));
     CUDA_TRY(cudaStreamCreateWithFlags(&p->d2h_stream, cudaStreamNonBlocking));
     for (int b = 0; b < 2; ++b) {
-      CUDA_TRY(cudaMalloc(&p->pdx[b], mt * p->cfg.h_in * 2));
-      CUDA_TRY(cudaMalloc(&p->pdy[b], mt * p->cfg.h_out * 2));
-      CUDA_TRY(cudaMalloc(&p->pdids[b], mt * 4));
+      CUDA_TRY(el_malloc(&p->pdx[b], mt * p->cfg.h_in * 2));
+      CUDA_TRY(el_malloc(&p->pdy[b], mt * p->cfg.h_out * 2));
+      CUDA_TRY(el_malloc(&p->pdids[b], mt * 4));
       CUDA_TRY(cudaEventCreateWithFlags(&p->ev_in[b], cudaEventDisableTiming));
       CUDA_TRY(cudaEventCreateWithFlags(&p->ev_done[b], cudaEventDisableTiming));
       CUDA_TRY(cudaEventCreateWithFlags(&p->ev_out[b], cudaEventDisableTiming));

@@ -387,7 +387,7 @@ decode_shrink_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         ptx::pdl_wait_prior_grids();
         waited = true;
       }
-      if (q < nt)
+      if (q < nt && EL_CHECK(status, s_gtok[tb + q] >= 0 && s_gtok[tb + q] < max_tokens && ad >= 0 && ad < n_slots, 20))
         zws[(KS > 1 ? c : kMaxZSplits) * zplane + static_cast<size_t>(s_gtok[tb + q]) * R_pad + r] =
             scale * acc[0];
     }

@@ -11,6 +11,7 @@
 #include <new>
 #include <vector>
 
+#include "guard.h"
 #include "pool.h"
 
 using namespace edgelora;
@@ -117,10 +118,10 @@ int edgelora_siteset_destroy(edgelora_siteset_t *s) {
   if (!s) return EDGELORA_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
   if (s->plan) edgelora_plan_destroy(s->plan);
-  for (auto *q : s->dx) if (q) cudaFree(q);
-  for (auto *q : s->dy) if (q) cudaFree(q);
-  for (auto &e : s->dy_scratch) if (e.second) cudaFree(e.second);
-  if (s->dids) cudaFree(s->dids);
+  for (auto *q : s->dx) if (q) el_free(q);
+  for (auto *q : s->dy) if (q) el_free(q);
+  for (auto &e : s->dy_scratch) if (e.second) el_free(e.second);
+  if (s->dids) el_free(s->dids);
   cudaGetLastError();
   delete s;
   return EDGELORA_OK;
@@ -168,21 +169,21 @@ int edgelora_siteset_run_host(edgelora_siteset_t *s, const uint16_t *const *x_ho
   for (int i = 0; i < s->n_inputs; ++i) {
     if (!s->in_width[i]) continue;
     if (!x_host[i]) return EDGELORA_ERR_INVALID_ARG;
-    if (!s->dx[i]) SET_TRY(cudaMalloc(&s->dx[i], mt * s->in_width[i] * 2));
+    if (!s->dx[i]) SET_TRY(el_malloc(&s->dx[i], mt * s->in_width[i] * 2));
   }
-  if (!s->dids) SET_TRY(cudaMalloc(&s->dids, mt * 4));
+  if (!s->dids) SET_TRY(el_malloc(&s->dids, mt * 4));
   std::vector<void *> y_dev(n, nullptr);
   for (int i = 0; i < n; ++i) {
     const int32_t h_out = s->pools[i]->cfg.h_out;
     if (y_host[i]) {
-      if (!s->dy[i]) SET_TRY(cudaMalloc(&s->dy[i], mt * h_out * 2));
+      if (!s->dy[i]) SET_TRY(el_malloc(&s->dy[i], mt * h_out * 2));
       y_dev[i] = s->dy[i];
     } else {
       uint16_t *buf = nullptr;
       for (auto &e : s->dy_scratch)
         if (e.first == h_out) buf = e.second;
       if (!buf) {
-        SET_TRY(cudaMalloc(&buf, mt * h_out * 2));
+        SET_TRY(el_malloc(&buf, mt * h_out * 2));
         s->dy_scratch.emplace_back(h_out, buf);
       }
       y_dev[i] = buf;

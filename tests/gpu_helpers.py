@@ -5,6 +5,9 @@ from paper_2507_01438_b200 import binding as B
 from paper_2507_01438_b200 import workloads as wl
 
 
+SENTINEL = 0x7FA5   # bfloat16 bits of a NaN payload that no result takes
+
+
 def to_dev_bf16(bits: np.ndarray):
     import torch
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
@@ -34,10 +37,17 @@ def run_gpu(w: "wl.Workload", regime: int = 0, pool=None, return_plan=False, opt
         W = to_dev_bf16(w.W)
         x = to_dev_bf16(w.x)
         ids = torch.from_numpy(w.ids).cuda()
-        y = torch.full((w.T, w.h_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+        # y sits between two sentinel rows (a bit pattern no result takes): writes outside y show there
+        framed = torch.full((w.T + 2, w.h_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+        framed[0].view(torch.int16).fill_(SENTINEL)
+        framed[-1].view(torch.int16).fill_(SENTINEL)
+        y = framed[1:w.T + 1]
         B.edgelora_lora_linear(pool.handle, W, x, ids, y)
         rc, bits = pool.status()
         assert rc == 0 and bits == 0, f"status rc={rc} bits={bits:#x}"
+        edges = framed[[0, -1]].view(torch.int16).cpu().numpy()
+        assert (edges == SENTINEL).all(), "the rows in front of or behind y were written"
+        assert B.edgelora_check_guards() == B.OK       # guard zones of the library's buffers (checked build)
         out = from_dev_bf16(y)
         if return_plan:
             plan = B.edgelora_plan_export(B.edgelora_pool_plan(pool.handle), w.T)

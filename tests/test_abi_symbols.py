@@ -45,6 +45,17 @@ def test_every_declared_symbol_is_exported(lib):
         getattr(lib, n)                                          # raises AttributeError if missing
 
 
+def test_checked_build_exports_the_same_symbols():
+    # the checked variant (-DEDGELORA_CHECKED) is the same sources and must offer the same boundary
+    if not (shutil.which("nvcc") or os.path.exists(libbuild.NVCC)):
+        pytest.skip("no nvcc to build the checked variant with")
+    path = libbuild.build(checked=True)
+    checked = ctypes.CDLL(path)
+    for n in declared_symbols():
+        getattr(checked, n)
+    assert checked.edgelora_build_is_checked() == 1
+
+
 def test_host_only_calls(lib):
     assert B.strerror(0) == "ok" and "rank" in B.strerror(B.ERR_RANK_TOO_LARGE)
     # 2 * R_pad * (h_in + h_out) bytes per slot, ranks padded to 16 / 32 / 64
