@@ -81,9 +81,11 @@ __device__ __forceinline__ int32_t gather_tiles(const GemmParams &p) {
 // first token tile go to those CTAs (as their first tile): in a serving batch the first token tile
 // holds the decode tokens (one token per generating request, many adapters, so many LoRA K blocks),
 // and its tiles are the longest of the launch.  Returns how many tiles are placed that way.
+// Only for launches of a site set (heavy_first): the placed tiles touch every W tile in the first
+// wave, which a batch without such a first tile pays for with a second read of W from HBM.
 __device__ __forceinline__ int32_t heavy_slots(const GemmParams &p, int32_t grid) {
   const int32_t total = p.n_mtiles * p.n_ntiles, rem = total % grid;
-  if (p.mode != kModePrefill || p.n_mtiles < 2 || total <= grid || rem == 0) return 0;
+  if (p.mode != kModePrefill || !p.heavy_first || p.n_mtiles < 2 || total <= grid || rem == 0) return 0;
   return min(p.n_ntiles, grid - rem);
 }
 

@@ -1118,6 +1118,7 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
     int BN = (tiles256 * 4 >= p->sms || h_out <= 128) ? 256 : 128;
     BN = std::min(BN, round_up(h_out, 32));
     g.mode = kModePrefill;
+    g.heavy_first = in_set ? 1 : 0;  // a serving batch: decode tokens first (see heavy_slots in gemm.cu)
     g.BN = BN;
     g.ring_rows = BN;
     g.acc_cols = BN;
