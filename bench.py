@@ -555,7 +555,7 @@ def bench_site(name, ctx, steps=None, warmup=None, pdl=None, graph=True, cpu_bud
         gemm_bytes = 2 * w.h_in * w.h_out + 2 * w.T * (w.h_in + w.h_out) + \
             sum(2 * w.adapters[a].rank * w.h_out for a in w.distinct_adapters())
         kernel_name = "lora_gemm_kernel (decode mode)"
-        if "shrink_small_decode" not in kt and "shrink_tiles" not in kt:
+        if not any(kt.get(k, {}).get("launches", 0) for k in ("shrink_small_decode", "shrink_tiles", "plan")):
             # one launch per call: the same kernel also reads every distinct A_a (its shrink teams)
             gemm_bytes = ws_bytes
             kernel_name = "lora_gemm_kernel (decode mode with the shrink teams in its grid: the whole call)"

@@ -594,6 +594,19 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     *abort_flag = 0;
     *s_nlg = 0;
     ptx::fence_barrier_init();
+    if (kFused && f.x_wait) {
+      // W is not written by any kernel of this library: this thread (lane 0 of the producer warp, which
+      // has just initialised the barriers) requests the W tiles of the first ring revolution at once,
+      // before the tensor-memory allocation and the CTA-wide barrier; the producer adds the x tiles
+      // after its dependency wait
+      const TileCoord tc0 = tile_coord(p, bid);
+      const int32_t npre = min(p.stages, tc0.kb1 - tc0.kb0);
+      for (int32_t i = 0; i < npre; ++i) {
+        ptx::mbar_arrive_expect_tx(&full_bar[i], r_bytes + c_bytes);
+        ptx::tma_load_2d(smem + static_cast<size_t>(i) * stage_bytes, &tmap_r, &full_bar[i], (tc0.kb0 + i) * kBlockK,
+                         tc0.row_r);
+      }
+    }
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, static_cast<uint32_t>(p.tmem_cols));
@@ -665,14 +678,9 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         int32_t kb_first = tc.kb0;
         if (kFused && f.x_wait && !x_waited) {
           // x may be an output of the kernel before this one, W is not: the W tiles of the first ring
-          // revolution are requested before the dependency wait, the x tiles after it
+          // revolution were requested in the prologue (with the bytes of both tiles announced), the x
+          // tiles follow the dependency wait
           const int32_t npre = min(static_cast<int32_t>(nstages), tc.kb1 - tc.kb0);  // the ring is empty: no waits
-          if (lane == 0)
-            for (int32_t i = 0; i < npre; ++i) {
-              ptx::mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
-              ptx::tma_load_2d(smem + static_cast<size_t>(i) * stage_bytes, mr, &full_bar[i], (tc.kb0 + i) * kBlockK,
-                               tc.row_r);
-            }
           ptx::pdl_wait_prior_grids();
           if (lane == 0)
             for (int32_t i = 0; i < npre; ++i)
@@ -1419,12 +1427,19 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     const bool have_acc = sender && !*abort_flag;  // this CTA's accumulator is complete (tfull waited)
     const bool z_ok = fused_z_ok;  // fused launches: the wait for the shrink teams ended in time
     float4 *z_stage = reinterpret_cast<float4 *>(b_stage + static_cast<size_t>(cols_per) * kTileM * p.R_pad * 2);
+    // The partial tiles land in the operand ring, which is idle once every CTA of the cluster is past
+    // its main loop: hence the first barrier.  A fused launch with room to spare (b_stage == 2) has a
+    // buffer of its own behind the staged rows instead, and sends at once.
+    const bool own_buf = kFused && f.b_stage == 2;
+    uint8_t *red = own_buf ? b_stage + ((static_cast<size_t>(cols_per) * (kTileM * p.R_pad * 2 + p.R_pad * 4) + 1023) &
+                                        ~static_cast<size_t>(1023))
+                           : smem;
     __syncwarp();
-    cluster_sync_all();
+    if (!own_buf) cluster_sync_all();
     if (have_acc) {
       ptx::tc_fence_after_sync();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-      const uint32_t local = ptx::smem_u32(smem) +
+      const uint32_t local = ptx::smem_u32(red) +
                              ((my_rank * cols_per) * kTileM + row_in_tile) * 4u;
       const uint32_t qpo = static_cast<uint32_t>(cols_per) >> 2;  // token quads per owner
       for (int32_t c0 = c_first; c0 < p.BN; c0 += c_step) {
@@ -1444,7 +1459,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
             const int col = c0 + g4 * 4;
             const uint32_t owner = static_cast<uint32_t>(col >> shift);
             const uint32_t quad_i = static_cast<uint32_t>(col & (cols_per - 1)) >> 2;
-            const uint32_t addr = ptx::smem_u32(smem) + ((my_rank * qpo + quad_i) * kTileM + row_in_tile) * 16u;
+            const uint32_t addr = ptx::smem_u32(red) + ((my_rank * qpo + quad_i) * kTileM + row_in_tile) * 16u;
             st_cluster_f32x4(map_to_cta(addr, owner), v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
           }
         }
@@ -1453,7 +1468,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     __syncwarp();
     cluster_sync_all();
     if (epi || wide) {
-      const float *buf = reinterpret_cast<const float *>(smem);
+      const float *buf = reinterpret_cast<const float *>(red);
       const int n_units = cols_per * 32;  // unit = (token, 4 adjacent W rows)
       const int row0 = bid / p.splits * kTileM;
       auto sum_partials = [&](int cl, int r4) {
@@ -1474,7 +1489,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         // unit = (token quad, W row): the splits' partial sums are 16 bytes each, lanes take
         // adjacent rows, so a warp writes 64 bytes in a row of y per token
         const int qpo = cols_per >> 2;
-        const float4 *buf4 = reinterpret_cast<const float4 *>(smem);
+        const float4 *buf4 = reinterpret_cast<const float4 *>(red);
         ptx::pdl_wait_prior_grids();  // warps 0 and 1 have not waited yet; earlier kernels may read y
         for (int u = threadIdx.x; u < qpo * kTileM; u += kGemmThreads) {
           const int qd = u >> 7, r = u & (kTileM - 1);
@@ -1497,7 +1512,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
         // needs is in shared memory by now: B_a[row][0..R_pad) of each token's adapter (lanes take
         // adjacent rows: 32-byte pieces side by side) and the tokens' z (the same for every lane).
         const int qpo = cols_per >> 2;
-        const float4 *buf4 = reinterpret_cast<const float4 *>(smem);
+        const float4 *buf4 = reinterpret_cast<const float4 *>(red);
         const int n_units = qpo * kTileM;  // at most 4 per thread (cols_per <= 16)
         const int nch = p.R_pad >> 3;
         float4 base[4];

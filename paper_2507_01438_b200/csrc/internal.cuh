@@ -123,7 +123,8 @@ struct FusedDecode {
   int32_t ks;              // K chunks of the shrink = partial z planes the expand adds, in order
   int32_t x_wait;          // 1: x may be an output of the kernel before this one: wait before reading it
   int32_t b_stage;         // 1: the launch's shared memory has room, behind the ring and the barriers, for the
-                           // B_a rows (tokens per owner x 128 rows x R_pad) and z of an owner's tokens
+                           // B_a rows (tokens per owner x 128 rows x R_pad) and z of an owner's tokens;
+                           // 2: also for the buffer of the cluster reduction
   const uint16_t *A_pool;  // [S][R_pad][h_in]
   const uint16_t *x;       // [T][h_in]
   float *z;                // [ks][max_tokens][R_pad]

@@ -1045,8 +1045,14 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
         !p->a_q8 && h_in % 8 == 0) {
       FusedDecode f{};
       // room behind the ring for the B_a rows and z of an owner's tokens, when it fits
-      const size_t stage_extra = static_cast<size_t>(N / splits) * (kTileM * R * 2 + R * 4);
+      // (2: and for the cluster reduction's buffer, which then does not have to wait for the ring)
+      size_t stage_extra = static_cast<size_t>(N / splits) * (kTileM * R * 2 + R * 4);
       f.b_stage = smem_for(g.stages, N, static_cast<int>(stage_extra)) <= kSmemBudget ? 1 : 0;
+      const size_t with_buf = ((stage_extra + 1023) & ~static_cast<size_t>(1023)) + static_cast<size_t>(N) * kTileM * 4;
+      if (f.b_stage && smem_for(g.stages, N, static_cast<int>(with_buf)) <= kSmemBudget) {
+        f.b_stage = 2;
+        stage_extra = with_buf;
+      }
       const size_t smem = smem_for(g.stages, N, f.b_stage ? static_cast<int>(stage_extra) : 0);
       const uint64_t key = (static_cast<uint64_t>(splits) << 32) | static_cast<uint64_t>(smem);
       if (p->fused_key != key) {
