@@ -104,7 +104,13 @@ typedef struct {
 #define EDGELORA_OPT_SHRINK_DEPTH 9  /* tuning: ring depth of the decode shrink for batches above 64 tokens:
                                         2 (default, two CTAs per SM) or 4 (one CTA per SM); 0 = default */
 #define EDGELORA_OPT_FUSED_DECODE 10 /* 1 (default): batches of at most 64 tokens take one launch, the shrink
-                                        on otherwise idle warps of the base product's grid; 0: two launches */
+                                        on otherwise idle warps of the base product's grid; 0: two launches.
+                                        The CTAs of such a launch wait (bounded) for one another, so all of
+                                        them must be resident at once: the library checks that against the
+                                        device's occupancy figure.  Set 0 for pools whose calls run at the
+                                        same time as another pool's on a stream of different priority: two
+                                        such grids could each hold SMs the other needs, and the wait would
+                                        end in EDGELORA_ERR_TIMEOUT */
 #define EDGELORA_OPT_WAIT_CYCLES 6   /* limit of every bounded in-kernel wait of the layer, in units
                                         of 1024 SM clock cycles; 0 = default (about two seconds).
                                         A wait that runs out raises EDGELORA_STATUS_TIMEOUT           */
