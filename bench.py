@@ -726,12 +726,20 @@ def bench_full_set(ctx, steps=None, warmup=None, cpu_budget=12.0, layers=wl.LLAM
         step()
     torch.cuda.synchronize()
     kt = {}
+    per_site = {}     # site name -> [device ms of its base-product launches, launches, flops of one launch]
     for s in sites:
         for kname, v in B.edgelora_pool_kernel_times(s[4].handle, reset=True).items():
             acc = kt.setdefault(kname, {"ms": 0.0, "launches": 0})
             acc["ms"] += v["ms"]
             acc["launches"] += v["launches"]
+            if kname == "base_gemm":
+                ps = per_site.setdefault(s[0], [0.0, 0, 2.0 * T * s[1] * s[2]])
+                ps[0] += v["ms"]
+                ps[1] += v["launches"]
         B.edgelora_pool_set_option(s[4].handle, B.OPT_PROFILE, 0)
+    per_site_us = {k: {"kernel_us": 1e3 * v[0] / max(v[1], 1),
+                       "base_tflops": v[2] / (1e-3 * v[0] / max(v[1], 1)) / 1e12 if v[0] > 0 else None}
+                   for k, v in per_site.items()}
     # kernels of one step in the timed configuration
     before = sum(B.edgelora_pool_last_launch(s[4].handle)["total_launches"] for s in sites)
     with torch.cuda.stream(stream):
@@ -766,6 +774,9 @@ def bench_full_set(ctx, steps=None, warmup=None, cpu_budget=12.0, layers=wl.LLAM
                      "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS, "nominal": "2.25 PFLOP/s dense bf16"},
         "e2e": e2e,
         "kernel_ms_profiled": {k: v for k, v in kt.items() if v["launches"]},
+        # per projection site, mean over the layers: serialised device time of its launch (its base product
+        # and the next site's shrink tiles) and the base product's flops over that time
+        "per_site": per_site_us,
     }
     if ctx["rank"] == 0 and world == 1 and cpu_budget > 0:
         res["cpu_baseline"] = full_set_oracle_sample(cpu_budget)
@@ -977,7 +988,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic"}
     for k in ("config", "launch_info", "clocks", "e2e", "gpu_launches", "roofline", "step_work", "step_roofline_frac",
               "step_roofline_frac_of_nominal", "iterations", "variants", "warm_l2", "single_call_latency",
-              "kernel_ms_profiled", "adapter_swaps", "cpu_baseline"):
+              "kernel_ms_profiled", "per_site", "adapter_swaps", "cpu_baseline"):
         if k in head:
             line[k] = head[k]
     if per_config:
