@@ -303,6 +303,21 @@ int edgelora_pool_set_option(edgelora_pool_t *pool, int32_t option, int32_t valu
  * EDGELORA_ERR_INVALID_ARG and nothing is launched. */
 int edgelora_pool_selftest_wait(edgelora_pool_t *pool, void *stream);
 
+/* Section 5.1, model table (base models stored in Q8_0 or Q4_0): decodes a base weight matrix kept in
+ * one of the two published block formats into the bfloat16 matrix W [h_out][h_in] that the layer
+ * calls take, on the device, so that the stored form is what crosses to the GPU (34/64 or 18/64 of
+ * the bfloat16 bytes).  Both formats block 32 consecutive values of a row (h_in % 32 == 0), a
+ * half-precision scale d first (little endian): Q8_0 has 32 signed bytes q after it, value d * q
+ * (34 bytes); Q4_0 has 16 bytes, byte j holding value j in its low and value j + 16 in its high four
+ * bits as codes c, value d * (c - 8) (18 bytes).  Each value is rounded to nearest even bfloat16.
+ * W_blocks_dev: device memory, [h_out][h_in / 32] blocks, read only; W_dev: device memory the caller
+ * owns, 16-byte aligned, written on `stream`.  EDGELORA_ERR_INVALID_ARG for an unknown format, a null
+ * pointer or h_in % 32 != 0; EDGELORA_ERR_CUDA if the launch fails. */
+#define EDGELORA_WEIGHTS_Q8_0 0
+#define EDGELORA_WEIGHTS_Q4_0 1
+int edgelora_weights_decode(int32_t format, const void *W_blocks_dev, int32_t h_out, int32_t h_in,
+                            uint16_t *W_dev, void *stream);
+
 /* The checked build of the library (compiled with -DEDGELORA_CHECKED, for finding memory errors
  * where no memory-checking tool can be run; the paper has no counterpart).  It differs in two ways.
  * The kernels test the indices they read from device memory (adapter ids in the routing plan's lists,

@@ -7,6 +7,12 @@ The layer with such adapters is the layer of Section 3.4 with A and B replaced b
 values; this file decodes in float64 (exactly: d has 11 significant bits, q 7) and evaluates the
 low-rank term token by token in float64 on top of the base product of the C oracle.
 
+Section 5.1's model table also stores the base weights in Q8_0 or Q4_0.  Q4_0 is the published ggml
+format of 18 bytes per 32 consecutive values: the half-precision scale d, then 16 bytes; byte j holds
+value j in its low four bits and value j + 16 in its high four bits, each an unsigned code c with
+value d * (c - 8).  `weights_decode` turns a matrix kept in either format into float64 values; the
+layer then rounds each to bfloat16 (nearest even), which is the W of Section 3.4.
+
 Readings: A is blocked along h_in (each of its `rank` rows is h_in / 32 blocks); B is blocked
 along the rank (each of its h_out rows is ceil(rank / 32) blocks, entries past the rank ignored),
 since the format blocks the contiguous dimension of a matrix.
@@ -34,6 +40,34 @@ def q8_0_decode(blocks: np.ndarray, n_values: int) -> np.ndarray:
                 q = int(blk[2 + i]) - 256 if blk[2 + i] >= 128 else int(blk[2 + i])
                 flat_o[r, b * BLOCK + i] = d * q
     return out[..., :n_values]
+
+
+Q4_BLOCK_BYTES = 18
+
+
+def q4_0_decode(blocks: np.ndarray, n_values: int) -> np.ndarray:
+    """blocks: uint8 [..., n_blocks, 18] -> float64 [..., n_values] (n_values <= 32 * n_blocks)."""
+    blocks = np.asarray(blocks, dtype=np.uint8)
+    assert blocks.shape[-1] == Q4_BLOCK_BYTES
+    lead = blocks.shape[:-2]
+    out = np.zeros(lead + (blocks.shape[-2] * BLOCK,), dtype=np.float64)
+    flat_b = blocks.reshape(-1, blocks.shape[-2], Q4_BLOCK_BYTES)
+    flat_o = out.reshape(-1, blocks.shape[-2] * BLOCK)
+    for r in range(flat_b.shape[0]):
+        for b in range(flat_b.shape[1]):
+            blk = flat_b[r, b]
+            d = float(np.frombuffer(blk[:2].tobytes(), dtype="<f2")[0])
+            for j in range(16):
+                byte = int(blk[2 + j])
+                flat_o[r, b * BLOCK + j] = d * ((byte & 0x0F) - 8)
+                flat_o[r, b * BLOCK + j + 16] = d * ((byte >> 4) - 8)
+    return out[..., :n_values]
+
+
+def weights_decode(fmt: str, blocks: np.ndarray, h_in: int) -> np.ndarray:
+    """fmt "q8_0" or "q4_0"; blocks uint8 [h_out, h_in / 32, 34 or 18] -> float64 [h_out, h_in]."""
+    assert h_in % BLOCK == 0 and blocks.shape[1] == h_in // BLOCK
+    return q8_0_decode(blocks, h_in) if fmt == "q8_0" else q4_0_decode(blocks, h_in)
 
 
 def lora_linear_q8(W_bits, x_bits, ids, adapters):

@@ -41,7 +41,7 @@ EXPORTS = (
     "edgelora_siteset_run_host", "edgelora_siteset_plan",
     "edgelora_cache_prefill", "edgelora_pool_load_slot_q8", "edgelora_pool_load_slot_pinned", "edgelora_batcher_create", "edgelora_batcher_destroy", "edgelora_batcher_submit",
     "edgelora_batcher_next_batch", "edgelora_batcher_complete_step", "edgelora_batcher_finished",
-    "edgelora_build_is_checked", "edgelora_check_guards",
+    "edgelora_build_is_checked", "edgelora_check_guards", "edgelora_weights_decode",
 )
 
 
@@ -114,6 +114,7 @@ def lib() -> ctypes.CDLL:
     L.edgelora_plan_sync_status.argtypes = [vp, vp, cp(ctypes.c_uint32)]
     L.edgelora_pool_selftest_wait.argtypes = [vp, vp]
     L.edgelora_build_is_checked.argtypes = []
+    L.edgelora_weights_decode.argtypes = [i32, vp, i32, i32, vp, vp]
     L.edgelora_check_guards.argtypes = []
     L.edgelora_pool_sync_status.argtypes = [vp, cp(ctypes.c_uint32)]
     L.edgelora_pool_set_option.argtypes = [vp, i32, i32]
@@ -353,6 +354,15 @@ def edgelora_plan_sync_status(plan, stream=None):
     if rc == ERR_CUDA or rc == ERR_INVALID_ARG:
         raise EdgeLoraError(rc, "plan_sync_status")
     return rc, bits.value
+
+
+WEIGHTS_Q8_0, WEIGHTS_Q4_0 = 0, 1
+
+
+def edgelora_weights_decode(fmt: int, W_blocks, h_out: int, h_in: int, W, stream=None) -> None:
+    """W_blocks: torch uint8 CUDA tensor [h_out, h_in / 32, 34 or 18]; W: torch bf16 CUDA tensor [h_out, h_in]."""
+    _check(lib().edgelora_weights_decode(fmt, W_blocks.data_ptr(), h_out, h_in, _dev_ptr(W, 2, "W"),
+                                         _stream_ptr(stream)), "weights_decode")
 
 
 def edgelora_build_is_checked() -> bool:

@@ -155,6 +155,7 @@ cudaError_t shrink_set_smem_limit();
 cudaError_t launch_q8_to_block(const uint8_t *A_q8, const uint8_t *B_q8, uint16_t *A_blk, uint16_t *B_blk,
                                int32_t rank, int32_t R_pad, int32_t h_in, int32_t h_out, int32_t sms,
                                cudaStream_t stream);
+void set_last_cuda_error(cudaError_t e, const char *what);
 cudaError_t launch_wait_selftest(uint32_t *status, long long wait_cycles, cudaStream_t stream);
 cudaError_t launch_decode_shrink(const CUtensorMap &tmap_a, const CUtensorMap &tmap_d, const CUtensorMap &tmap_x,
                                  const int32_t *ids, const SlotRow *slots, const PlanView &pv,

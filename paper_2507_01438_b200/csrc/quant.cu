@@ -9,6 +9,8 @@
 // side stream, and the layer kernels read the block as they read any other.
 #include <cuda_fp16.h>
 
+#include <algorithm>
+
 #include "internal.cuh"
 #include "ptx.cuh"
 
@@ -54,6 +56,53 @@ q8_to_block_kernel(const uint8_t *__restrict__ A_q8, const uint8_t *__restrict__
   }
 }
 
+// Base weights stored in a block format (paper Section 5.1, model table: base models in Q8_0 or
+// Q4_0).  Q4_0 is the published ggml format of 18 bytes per 32 consecutive values of a row: a
+// half-precision scale d, then 16 bytes; byte j holds value j in its low four bits and value j + 16
+// in its high four bits, each as an unsigned code c with value d * (c - 8).  One thread decodes one
+// block into 32 bfloat16 values (round to nearest even; d * code is exact in fp32).
+template <int kFormat>  // 0: Q8_0, 1: Q4_0
+__global__ void __launch_bounds__(256)
+weights_decode_kernel(const uint8_t *__restrict__ Wq, uint16_t *__restrict__ W, size_t n_blocks) {
+  constexpr int kBytes = kFormat == 0 ? kQ8Bytes : 18;
+  for (size_t b = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; b < n_blocks;
+       b += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const uint8_t *blk = Wq + b * kBytes;
+    const float d = __half2float(__ushort_as_half(static_cast<unsigned short>(blk[0] | (blk[1] << 8))));
+    float v[32];
+    if (kFormat == 0) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = d * static_cast<float>(static_cast<int8_t>(blk[2 + i]));
+    } else {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const int byte = blk[2 + j];
+        v[j] = d * static_cast<float>((byte & 0xF) - 8);
+        v[j + 16] = d * static_cast<float>((byte >> 4) - 8);
+      }
+    }
+    uint4 *dst = reinterpret_cast<uint4 *>(W + b * 32);  // blocks follow one another along the rows
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint4 o;
+      o.x = ptx::pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
+      o.y = ptx::pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
+      o.z = ptx::pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
+      o.w = ptx::pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
+      dst[q] = o;
+    }
+  }
+}
+
+cudaError_t launch_weights_decode(int32_t format, const uint8_t *Wq, uint16_t *W, size_t n_blocks, cudaStream_t stream) {
+  const int grid = static_cast<int>(std::min<size_t>((n_blocks + 255) / 256, 148 * 8));
+  if (format == 0)
+    weights_decode_kernel<0><<<grid, 256, 0, stream>>>(Wq, W, n_blocks);
+  else
+    weights_decode_kernel<1><<<grid, 256, 0, stream>>>(Wq, W, n_blocks);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_q8_to_block(const uint8_t *A_q8, const uint8_t *B_q8, uint16_t *A_blk, uint16_t *B_blk,
                                int32_t rank, int32_t R_pad, int32_t h_in, int32_t h_out, int32_t sms,
                                cudaStream_t stream) {
@@ -62,3 +111,18 @@ cudaError_t launch_q8_to_block(const uint8_t *A_q8, const uint8_t *B_q8, uint16_
 }
 
 }  // namespace edgelora
+
+extern "C" int edgelora_weights_decode(int32_t format, const void *W_blocks_dev, int32_t h_out, int32_t h_in,
+                                       uint16_t *W_dev, void *stream) {
+  if ((format != EDGELORA_WEIGHTS_Q8_0 && format != EDGELORA_WEIGHTS_Q4_0) || !W_blocks_dev || !W_dev || h_out <= 0 ||
+      h_in <= 0 || h_in % 32 != 0)
+    return EDGELORA_ERR_INVALID_ARG;
+  const size_t n_blocks = static_cast<size_t>(h_out) * (h_in / 32);
+  const cudaError_t e = edgelora::launch_weights_decode(format, static_cast<const uint8_t *>(W_blocks_dev), W_dev, n_blocks,
+                                                        static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) {
+    edgelora::set_last_cuda_error(e, "weights_decode_kernel");
+    return EDGELORA_ERR_CUDA;
+  }
+  return EDGELORA_OK;
+}

@@ -269,3 +269,26 @@ def q8_0_encode(values: np.ndarray) -> np.ndarray:
     out[..., 0:2] = np.ascontiguousarray(d.astype("<f2"))[..., None].view(np.uint8)   # little endian
     out[..., 2:] = q.view(np.uint8)
     return out
+
+
+def q4_0_encode(values: np.ndarray) -> np.ndarray:
+    """Packs rows of float32 values into Q4_0 blocks (input preparation for base weights that arrive in
+    the paper's storage format): per 32 values the element of largest magnitude m fixes d = m / -8 (half
+    precision), codes c = clamp(round(v / d) + 8, 0, 15); byte j = c[j] | c[j + 16] << 4.  The row length
+    must be a multiple of 32.  Returns uint8 [..., n_blocks, 18]."""
+    v = np.asarray(values, dtype=np.float32)
+    n = v.shape[-1]
+    assert n % 32 == 0
+    blk = v.reshape(v.shape[:-1] + (n // 32, 32))
+    idx = np.abs(blk).argmax(axis=-1)
+    m = np.take_along_axis(blk, idx[..., None], axis=-1)[..., 0]
+    d = (m / np.float32(-8.0)).astype(np.float16)
+    df = d.astype(np.float32)
+    inv = np.zeros_like(df)
+    nz = df != 0
+    inv[nz] = np.float32(1.0) / df[nz]
+    c = np.clip(np.floor(blk * inv[..., None] + np.float32(8.5)), 0, 15).astype(np.uint8)
+    out = np.zeros(v.shape[:-1] + (n // 32, 18), dtype=np.uint8)
+    out[..., 0:2] = np.ascontiguousarray(d.astype("<f2"))[..., None].view(np.uint8)
+    out[..., 2:] = c[..., :16] | (c[..., 16:] << 4)
+    return out

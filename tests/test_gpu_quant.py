@@ -99,3 +99,36 @@ def test_q8_pool_needs_a_width_of_256():
     with pytest.raises(B.EdgeLoraError) as e:
         B.Pool(320, 256, 2, 16, max_tokens=16, flags=B.FLAG_A_Q8)
     assert e.value.code == B.ERR_INVALID_ARG
+
+
+# ------------------------------------------------------------------ base weights stored in Q8_0 / Q4_0
+@pytest.mark.parametrize("fmt,code,encode", [("q8_0", B.WEIGHTS_Q8_0, wl.q8_0_encode), ("q4_0", B.WEIGHTS_Q4_0, wl.q4_0_encode)])
+def test_base_weights_decode_is_bit_exact_and_feeds_the_layer(fmt, code, encode):
+    # The decode kernel against the oracle's decode: d * code is exact in both, so after rounding to
+    # bfloat16 the bits must agree.  Then the layer over the decoded W against the layer oracle.
+    import torch
+    from oracle.quant import weights_decode
+    from gpu_helpers import to_dev_bf16, from_dev_bf16, make_pool
+    from helpers import assert_parity, oracle_of
+    from test_gpu_parity import random_workload
+    w = random_workload(8800, 40, 512, 392, ranks=[16, 8, 12], max_rank=16)
+    Wf = wl.bf16_bits_to_f32(w.W)
+    blocks = encode(Wf)                                              # [h_out, h_in / 32, 34 or 18]
+    want_bits = wl.f32_to_bf16_bits(weights_decode(fmt, blocks, w.h_in).astype(np.float32))
+    Wq = torch.from_numpy(blocks).cuda()
+    W = torch.zeros((w.h_out, w.h_in), dtype=torch.bfloat16, device="cuda")
+    B.edgelora_weights_decode(code, Wq, w.h_out, w.h_in, W)
+    torch.cuda.synchronize()
+    got_bits = W.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(got_bits, want_bits)
+    w2 = wl.Workload(f"{fmt}_weights", w.h_in, w.h_out, w.n_slots, w.max_rank, want_bits, w.x, w.ids, w.adapters)
+    pool = make_pool(w2, 64)
+    try:
+        y = pool.linear(W, to_dev_bf16(w2.x), torch.from_numpy(w2.ids).cuda())
+        assert pool.status() == (0, 0)
+        assert_parity(from_dev_bf16(y), oracle_of(w2), f"layer over W decoded from {fmt}")
+    finally:
+        pool.close()
+    with pytest.raises(B.EdgeLoraError) as e:
+        B.edgelora_weights_decode(7, Wq, w.h_out, w.h_in, W)
+    assert e.value.code == B.ERR_INVALID_ARG

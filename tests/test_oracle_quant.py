@@ -56,3 +56,37 @@ def test_layer_with_q8_adapters_equals_the_bf16_layer_on_values_both_formats_hol
     assert np.allclose(got, want, rtol=1e-12, atol=1e-12)
     base = oracle.lora_linear(W, x, np.full(T, -1, np.int32), adapter_set(2, {}))
     assert np.array_equal(got[ids < 0], base[ids < 0]) and not np.allclose(got[ids >= 0], base[ids >= 0])
+
+
+# ------------------------------------------------------------------ base weights in Q4_0 / Q8_0
+def test_q4_0_hand_written_block():
+    from oracle.quant import q4_0_decode
+    fx = golden("q4_0_block.json")
+    blk = np.array(fx["block_bytes"], dtype=np.uint8).reshape(1, 18)
+    assert np.array_equal(q4_0_decode(blk, 32), np.array(fx["values"], dtype=np.float64))
+    # a shorter row takes the leading values only
+    assert np.array_equal(q4_0_decode(blk, 20), np.array(fx["values"][:20], dtype=np.float64))
+
+
+def test_q4_0_encoder_round_trip_is_within_half_a_step():
+    from oracle.quant import q4_0_decode, weights_decode
+    rng = np.random.Generator(np.random.PCG64(9))
+    v = (rng.standard_normal((6, 128)) * 0.05).astype(np.float32)
+    blocks = wl.q4_0_encode(v)
+    assert blocks.shape == (6, 4, 18)
+    back = q4_0_decode(blocks, 128)
+    m = np.abs(v.reshape(6, 4, 32)).max(axis=-1)
+    step = np.repeat(m / 8.0, 32, axis=1)
+    # half a step, except at the end of the range opposite to the largest element (code 15 = +7 steps)
+    assert np.all(np.abs(back - v) <= 1.0 * step * (1 + 2e-3) + 1e-12)
+    inner = np.abs(v) <= 6.5 * step
+    assert np.all(np.abs(back - v)[inner] <= 0.5 * step[inner] * (1 + 4e-3) + 1e-12)
+    assert np.all(q4_0_decode(wl.q4_0_encode(np.zeros((2, 32), np.float32)), 32) == 0.0)
+    # multiples of a power-of-two step with the extreme at -8 steps survive exactly
+    exact = (rng.integers(-7, 8, size=(3, 64)) * 0.125).astype(np.float32)
+    exact[:, 0], exact[:, 32] = -8 * 0.125, -8 * 0.125
+    assert np.array_equal(q4_0_decode(wl.q4_0_encode(exact), 64), exact.astype(np.float64))
+    assert np.array_equal(weights_decode("q4_0", wl.q4_0_encode(exact), 64), exact.astype(np.float64))
+    exact8 = (rng.integers(-127, 128, size=(3, 64)) * 0.25).astype(np.float32)
+    exact8[:, 0], exact8[:, 32] = 127 * 0.25, -127 * 0.25          # d = 1/4 exactly
+    assert np.array_equal(weights_decode("q8_0", wl.q8_0_encode(exact8), 64), exact8.astype(np.float64))
