@@ -766,7 +766,7 @@ def bench_full_set(ctx, steps=None, warmup=None, cpu_budget=12.0, layers=wl.LLAM
         "step_roofline_frac": step_tflops / peak,
         "step_roofline_frac_of_nominal": step_tflops / NOMINAL_BF16_TFLOPS,
         "roofline": {"bound": "tensor", "kernel": "lora_gemm_kernel (prefill mode), all 224 sites of a step",
-                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": (ncu_traffic("full_projection_set_per_layer") or 0) * layers or None,
                      "algorithmic_flops": flops, "kernel_us": 1e3 * gemm_ms / max(kt["base_gemm"]["launches"], 1),
                      "kernel_us_is": "serialised latency of one launch between two CUDA events (launch gap included), "
                                      "mean over the 224 sites; with events between the kernels nothing overlaps",
