@@ -78,11 +78,10 @@ __device__ __forceinline__ int32_t gather_tiles(const GemmParams &p) {
 
 // Prefill jobs: tiles are dealt round-robin to the CTAs of the persistent grid, so when the tile count
 // is not a multiple of the grid the CTAs from (count % grid) on get one tile fewer.  The tiles of the
-// first token tile go to those CTAs (as their first tile): in a serving batch the first token tile
-// holds the decode tokens (one token per generating request, many adapters, so many LoRA K blocks),
-// and its tiles are the longest of the launch.  Returns how many tiles are placed that way.
-// Only for launches of a site set (heavy_first): the placed tiles touch every W tile in the first
-// wave, which a batch without such a first tile pays for with a second read of W from HBM.
+// first token tile go to those CTAs: in a serving batch the first token tile holds the decode tokens
+// (one token per generating request, many adapters, so many LoRA K blocks), and its tiles are the
+// longest of the launch.  Returns how many tiles are placed that way (tile_coord says where).
+// Only for launches of a site set (heavy_first).
 __device__ __forceinline__ int32_t heavy_slots(const GemmParams &p, int32_t grid) {
   const int32_t total = p.n_mtiles * p.n_ntiles, rem = total % grid;
   if (p.mode != kModePrefill || !p.heavy_first || p.n_mtiles < 2 || total <= grid || rem == 0) return 0;
@@ -107,18 +106,33 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams &p, int32_t til
     int m, n;
     const int32_t H = heavy_slots(p, gridDim.x);
     const int32_t rem = (p.n_mtiles * p.n_ntiles) % static_cast<int32_t>(gridDim.x);
-    if (H > 0 && tile >= rem && tile < rem + H) {  // first-wave positions of the CTAs with a tile fewer
-      m = 0;
-      n = tile - rem;
-    } else if (H > 0) {  // the other tiles in their usual order, the H placed ones taken out
-      const int32_t u = tile < rem ? tile : tile - H;
-      if (u < H * (p.n_mtiles - 1)) {
-        n = u / (p.n_mtiles - 1);
-        m = 1 + u % (p.n_mtiles - 1);
-      } else {
-        const int32_t o = u + H;
-        n = o / p.n_mtiles;
-        m = o % p.n_mtiles;
+    if (H > 0) {
+      // Position `tile` is step tile / grid of CTA tile % grid.  The tile (0, j) sits on CTA rem + j, at
+      // the step at which the sweep over the other tiles (column by column, below) is at column j, so
+      // that the W tile it needs is the one the launch is reading anyway.  pos(j) grows with j: the
+      // number of placed tiles in front of a position is found by bisection.
+      const int32_t grid = static_cast<int32_t>(gridDim.x);
+      const int32_t last_step = (p.n_mtiles * p.n_ntiles) / grid - 1;  // last step of a CTA with a tile fewer
+      auto pos = [&](int32_t j) { return min(last_step, (j * (p.n_mtiles - 1)) / grid) * grid + rem + j; };
+      int32_t lo = 0, hi = H;
+      while (lo < hi) {
+        const int32_t mid = (lo + hi) >> 1;
+        if (pos(mid) < tile) lo = mid + 1;
+        else hi = mid;
+      }
+      if (lo < H && pos(lo) == tile) {
+        m = 0;
+        n = lo;
+      } else {  // the other tiles in their usual order, the H placed ones taken out
+        const int32_t u = tile - lo;
+        if (u < H * (p.n_mtiles - 1)) {
+          n = u / (p.n_mtiles - 1);
+          m = 1 + u % (p.n_mtiles - 1);
+        } else {
+          const int32_t o = u + H;
+          n = o / p.n_mtiles;
+          m = o % p.n_mtiles;
+        }
       }
     } else {
       m = tile % p.n_mtiles;
