@@ -636,20 +636,42 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
 
   if (p.mode == kModeSgmv) ptx::pdl_wait_prior_grids();  // tile list comes from the plan kernel
   const int32_t n_tiles0 = total_tiles(p);
-  // the second job's tiles start behind the CTAs that took the first token tile's tiles (above)
+  // Where the second job's tiles go.  Positions continue after the first job's, round-robin over the
+  // CTAs, so the first of them fall on the CTAs that got one tile fewer (or none).  Those CTAs are free
+  // for about a tile's time: they take fill_rounds of the second job's tiles each before the others
+  // get any (the positions of the others are holes in those rounds); the CTAs that took the first
+  // token tile's tiles, which are longer, sit out the first round (n_hole).
   const int32_t n_hole = has2 ? heavy_slots(p, gridDim.x) : 0;
-  const int32_t n_tiles = n_tiles0 + n_hole + (has2 ? p2.n_mtiles : 0);
+  const int32_t rem0 = (has2 && p.mode == kModePrefill) ? n_tiles0 % ngrid : 0;
+  const int32_t n_short = rem0 > 0 ? ngrid - rem0 : 0;
+  const int32_t fill = max(1, p.fill_rounds);
+  const int32_t n_tiles = n_tiles0 + (has2 ? p2.n_mtiles + (n_short > 0 ? n_short + (fill - 1) * ngrid : 0) : 0);
   const uint32_t nstages = static_cast<uint32_t>(p.stages);
   // Every role walks the same tile sequence: tiles below n_tiles0 belong to the first job; for the
   // others the true count of the second job is read once (after griddepcontrol.wait: the plan may
   // come from a kernel this one was allowed to start under) and the walk ends at it.
   int32_t n2_true = -1;
-  auto second_job_tile = [&](int32_t tile) -> int32_t {  // local tile index, or -1 = stop
+  auto second_job_tile = [&](int32_t tile) -> int32_t {  // local tile index, -2 = a hole, -1 = stop
+    const int32_t q = tile - n_tiles0;
+    int32_t local;
+    if (n_short == 0) {
+      local = q;
+    } else if (q < n_short) {
+      if (q < n_hole) return -2;
+      local = q - n_hole;
+    } else {
+      const int32_t q2 = q - n_short, round = q2 / ngrid + 1, c = q2 % ngrid;
+      if (round < fill) {
+        if (c < rem0) return -2;
+        local = (n_short - n_hole) + (round - 1) * n_short + (c - rem0);
+      } else {
+        local = (n_short - n_hole) + (fill - 1) * n_short + (round - fill) * ngrid + c;
+      }
+    }
     if (n2_true < 0) {
       ptx::pdl_wait_prior_grids();
       n2_true = total_tiles(p2);
     }
-    const int32_t local = tile - n_tiles0 - n_hole;
     return local < n2_true ? local : -1;
   };
 
@@ -675,8 +697,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       for (int32_t tile = bid; ok && tile < n_tiles; tile += ngrid) {
         const bool second = tile >= n_tiles0;
         int32_t local = tile;
-        if (second && tile < n_tiles0 + n_hole) continue;
-        if (second && (local = second_job_tile(tile)) < 0) break;
+        if (second && (local = second_job_tile(tile)) < 0) {
+          if (local == -2) continue;
+          break;
+        }
         const GemmParams &jp = second ? p2 : p;
         const CUtensorMap *mr = second ? &tmap_r2 : &tmap_r, *mc = second ? &tmap_c2 : &tmap_c;
         const TileCoord tc = tile_coord(jp, local);
@@ -774,8 +798,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
       for (int32_t tile = bid; ok && tile < n_tiles; tile += ngrid) {
         const bool second = tile >= n_tiles0;
         int32_t local = tile;
-        if (second && tile < n_tiles0 + n_hole) continue;
-        if (second && (local = second_job_tile(tile)) < 0) break;
+        if (second && (local = second_job_tile(tile)) < 0) {
+          if (local == -2) continue;
+          break;
+        }
         const GemmParams &jp = second ? p2 : p;
         const TileCoord tc = tile_coord(jp, local);
         const int32_t n_pass = tile_passes(jp, tc);
@@ -996,8 +1022,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     for (int32_t tile = bid; ok && tile < n_tiles; tile += ngrid) {
       const bool second = tile >= n_tiles0;
       int32_t local = tile;
-      if (second && tile < n_tiles0 + n_hole) continue;
-      if (second && (local = second_job_tile(tile)) < 0) break;
+      if (second && (local = second_job_tile(tile)) < 0) {
+        if (local == -2) continue;
+        break;
+      }
       const GemmParams &jp = second ? p2 : p;
       const TileCoord tc = tile_coord(jp, local);
       if (kShrink && tc.kind == 1) {
@@ -1342,8 +1370,8 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tmap_r, const __grid_consta
     }
     for (int32_t tile = bid; ok && tile < n_tiles; tile += ngrid) {
       if (kShrink && tile >= n_tiles0) {  // a tile of the second job: no LoRA blocks
-        if (tile < n_tiles0 + n_hole) continue;
         const int32_t local = second_job_tile(tile);
+        if (local == -2) continue;
         if (local < 0) break;
         ok = shrink_tile(p2, local, &tmap_c2, &tmap_g2);
         continue;

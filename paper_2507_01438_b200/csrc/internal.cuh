@@ -78,6 +78,8 @@ struct GemmParams {
   int32_t ring_rows;   // rows of the C region of a ring stage (>= BN; wider when gather passes need it)
   int32_t acc_cols;    // TMEM columns between the accumulators (>= BN, >= gN)
   int32_t y_tma;       // prefill: y leaves through a shared-memory stage and TMA stores (needs the y map)
+  int32_t fill_rounds; // prefill with a second job: how many of that job's tiles a CTA with a tile fewer (or none)
+                       // takes before the other CTAs get any: about (K blocks of a tile) / (K blocks of such an item)
   int32_t heavy_first; // prefill: the first token tile holds the batch's decode tokens (many LoRA K blocks per
                        // output tile): its tiles go to the CTAs that get one tile fewer (see heavy_slots)
   int32_t kb_total;    // K blocks of 64 covering h_in

@@ -1156,6 +1156,8 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
         if (rc) return rc;
         fuse_next = true;
         grid = std::min(p->sms, g.n_mtiles * g.n_ntiles + nj.s.n_mtiles);
+        // CTAs that get one tile fewer (or none) are free for about a tile's time: that many shrink items
+        g.fill_rounds = std::max(1, std::min(8, kb_total / std::max(1, nj.s.kb_per)));
       } else {  // cannot share the ring (a tiny site): on its own, before this site's base product
         rc = shrink_job(q, next->x, false, 0, &nj);
         if (rc) return rc;
