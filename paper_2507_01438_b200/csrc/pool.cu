@@ -1087,10 +1087,12 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
     }
     if (!fused) {
       ProfScope ps(p, 3, stream);
-      // With one CTA per SM the base product cannot start beside the shrink (both fill an SM's
-      // shared memory), and an early launch then only costs: measured 178 vs 122 us per step on
-      // the 14336 -> 4096, T = 256 workload.
-      CUDA_TRY(launch_gemm(mr, mc, mb, g, grid, smem_for(g.stages, N), pdl && ctas_per_sm == 2, stream));
+      // Launched under the shrink's tail: a base-product CTA cannot share an SM with the shrink's CTAs
+      // (shared memory), but the shrink's CTAs end at different times, and on the SMs that are free
+      // early the base K blocks, which need no z, start at once (14336 -> 4096, T = 256: 99 us per
+      // step against 104; with the one-CTA-per-SM shrink of four ring stages it was the other way
+      // round, 178 against 122 us).
+      CUDA_TRY(launch_gemm(mr, mc, mb, g, grid, smem_for(g.stages, N), pdl, stream));
       ++launches;
       p->last_info[2] = grid;
       p->last_info[3] = splits;
