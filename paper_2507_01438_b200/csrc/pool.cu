@@ -945,7 +945,11 @@ int lora_linear_impl(edgelora_pool *p, edgelora_plan *plan, const int32_t *ids_d
         // the 200-adapter down_proj: 45.8 us against 49.8 us with depth 4)
         const int shrink_depth = T <= 64 ? 2 : (p->opt_shrink_depth == 4 ? 4 : 2);
         const int cta_cap = shrink_depth == 2 && T > 64 ? 2 * p->sms : p->sms;
-        const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : (overlapped ? 1 : 4 * 8 * cta_cap);
+        // Large batches: few, long items (about 0.6 per warp) beat many short ones, whose ring ramp-up and
+        // chunk sums add up: 92 us per step with 2 K chunks on the 1000-adapter down_proj, 96 with 3-4,
+        // 100 with 12, 104 with 1.  Small batches: four items per warp.
+        const int auto_target = T > 64 ? 5 * cta_cap : 4 * 8 * cta_cap;
+        const int target = p->opt_shrink_items > 0 ? p->opt_shrink_items : (overlapped ? 1 : auto_target);
         // at most T token blocks x (R / 8) row groups x K chunks warp items, eight warps per CTA
         const int n_ksteps = (h_in + kShrinkStepElems - 1) / kShrinkStepElems;
         const int max_chunks = target == 1 ? 1 : std::max(1, std::min(kMaxZSplits, n_ksteps / 4));
