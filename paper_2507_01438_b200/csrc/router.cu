@@ -15,9 +15,14 @@
 namespace edgelora {
 
 constexpr int kRouterThreads = 256;
-constexpr int kRouterReq = 8;  // prompts per pass over a row
-constexpr int kRouterUnroll = 8;
+constexpr int kRouterReq = 8;      // prompts per pass over a row
+constexpr int kRouterUnroll = 16;  // 16-byte loads per lane in flight: a whole row of 4096 values
 
+// A warp asks for (the first 8 KB of) its first row before the prompts are staged in shared memory, so
+// that the rows are on their way while the CTA synchronises: the kernel is a few microseconds long and
+// what it waits for is the first round trip to HBM.  Up to eight prompts share a pass over W_r; the
+// loop over them is rolled (the row stays in registers), because code that runs once or twice per
+// launch costs its instruction fetch: lane q ends up with the score of prompt b0 + q.
 __global__ void __launch_bounds__(kRouterThreads)
 router_scores_kernel(const uint16_t *__restrict__ Wr, const float *__restrict__ bias,
                      const uint16_t *__restrict__ h, int32_t B, int32_t n, int32_t hidden,
@@ -25,61 +30,52 @@ router_scores_kernel(const uint16_t *__restrict__ Wr, const float *__restrict__ 
   extern __shared__ uint4 s_h[];  // [min(B, 8)][hidden / 8]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int n8 = hidden >> 3;
+  const int j_first = blockIdx.x * (kRouterThreads / 32) + warp, j_step = gridDim.x * (kRouterThreads / 32);
   ptx::pdl_launch_dependents();
-  ptx::pdl_wait_prior_grids();  // h comes from earlier work on the stream
+  auto load_chunk = [&](int j, int k0, uint4 (&wv)[kRouterUnroll]) {
+    const uint4 *row = reinterpret_cast<const uint4 *>(Wr + static_cast<size_t>(j) * hidden);
+#pragma unroll
+    for (int u = 0; u < kRouterUnroll; ++u)
+      wv[u] = (k0 + 32 * u < n8) ? __ldg(row + k0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
+  };
+  uint4 wv[kRouterUnroll];
+  if (j_first < n) load_chunk(j_first, lane, wv);  // W_r is not written by anything on the stream
+  ptx::pdl_wait_prior_grids();                      // h comes from earlier work on the stream
   for (int b0 = 0; b0 < B; b0 += kRouterReq) {
     const int nb = min(kRouterReq, B - b0);
     __syncthreads();
     for (int i = threadIdx.x; i < nb * n8; i += kRouterThreads)
       s_h[i] = __ldg(reinterpret_cast<const uint4 *>(h + static_cast<size_t>(b0) * hidden) + i);
     __syncthreads();
-    for (int j = blockIdx.x * (kRouterThreads / 32) + warp; j < n; j += gridDim.x * (kRouterThreads / 32)) {
-      const uint4 *row = reinterpret_cast<const uint4 *>(Wr + static_cast<size_t>(j) * hidden);
-      float acc[kRouterReq];
-#pragma unroll
-      for (int q = 0; q < kRouterReq; ++q) acc[q] = 0.f;
-      // kRouterUnroll loads of 16 bytes per lane in flight: a row is a few KB, so what matters is
-      // how many requests a warp has outstanding, not how fast it adds
+    for (int j = j_first; j < n; j += j_step) {
+      float v = 0.f;  // lane q: W_r[j] . h[b0 + q]
       for (int k0 = lane; k0 < n8; k0 += 32 * kRouterUnroll) {
-        uint4 wv[kRouterUnroll];
+        if (!(b0 == 0 && j == j_first && k0 == lane)) load_chunk(j, k0, wv);  // the first chunk is already here
+#pragma unroll 1
+        for (int q = 0; q < nb; ++q) {
+          const uint4 *hq = s_h + q * n8 + k0;
+          float s = 0.f;
 #pragma unroll
-        for (int u = 0; u < kRouterUnroll; ++u)
-          wv[u] = (k0 + 32 * u < n8) ? __ldg(row + k0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-        for (int u = 0; u < kRouterUnroll; ++u) {
-          const int k = k0 + 32 * u;
-          if (k >= n8) break;
-          const uint4 w = wv[u];
-          const float w0 = ptx::bf16_lo(w.x), w1 = ptx::bf16_hi(w.x), w2 = ptx::bf16_lo(w.y), w3 = ptx::bf16_hi(w.y);
-          const float w4 = ptx::bf16_lo(w.z), w5 = ptx::bf16_hi(w.z), w6 = ptx::bf16_lo(w.w), w7 = ptx::bf16_hi(w.w);
-#pragma unroll
-          for (int q = 0; q < kRouterReq; ++q) {
-            if (q < nb) {
-              const uint4 x = s_h[q * n8 + k];
-              float s = acc[q];
-              s = fmaf(w0, ptx::bf16_lo(x.x), s); s = fmaf(w1, ptx::bf16_hi(x.x), s);
-              s = fmaf(w2, ptx::bf16_lo(x.y), s); s = fmaf(w3, ptx::bf16_hi(x.y), s);
-              s = fmaf(w4, ptx::bf16_lo(x.z), s); s = fmaf(w5, ptx::bf16_hi(x.z), s);
-              s = fmaf(w6, ptx::bf16_lo(x.w), s); s = fmaf(w7, ptx::bf16_hi(x.w), s);
-              acc[q] = s;
+          for (int u = 0; u < kRouterUnroll; ++u) {
+            if (k0 + 32 * u < n8) {  // (values past the row are zero: nothing to add)
+              const uint4 w = wv[u], x = hq[32 * u];
+              s = fmaf(ptx::bf16_lo(w.x), ptx::bf16_lo(x.x), s); s = fmaf(ptx::bf16_hi(w.x), ptx::bf16_hi(x.x), s);
+              s = fmaf(ptx::bf16_lo(w.y), ptx::bf16_lo(x.y), s); s = fmaf(ptx::bf16_hi(w.y), ptx::bf16_hi(x.y), s);
+              s = fmaf(ptx::bf16_lo(w.z), ptx::bf16_lo(x.z), s); s = fmaf(ptx::bf16_hi(w.z), ptx::bf16_hi(x.z), s);
+              s = fmaf(ptx::bf16_lo(w.w), ptx::bf16_lo(x.w), s); s = fmaf(ptx::bf16_hi(w.w), ptx::bf16_hi(x.w), s);
             }
           }
+#pragma unroll
+          for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+          if (lane == q) v += s;
         }
       }
-#pragma unroll
-      for (int q = 0; q < kRouterReq; ++q)
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], d);
       if (lane < nb) {
-        float v = 0.f;
-#pragma unroll
-        for (int q = 0; q < kRouterReq; ++q)
-          if (q == lane) v = acc[q];
         if (bias) v += bias[j];
         // sigmoid without overflow on either side
         const float e = __expf(-fabsf(v));
-        const float s = v >= 0.f ? 1.f / (1.f + e) : e / (1.f + e);
-        scores[static_cast<size_t>(b0 + lane) * n + j] = s;
+        const float sg = v >= 0.f ? 1.f / (1.f + e) : e / (1.f + e);
+        scores[static_cast<size_t>(b0 + lane) * n + j] = sg;
       }
     }
   }
