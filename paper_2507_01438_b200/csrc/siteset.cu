@@ -28,6 +28,8 @@ struct edgelora_siteset {
   int32_t *dids = nullptr;
   std::vector<uint16_t *> dy;             // [n_sites] device results of the sites that are read back
   std::vector<std::pair<int32_t, uint16_t *>> dy_scratch;  // (h_out, buffer) for the others
+  cudaStream_t copy_stream = nullptr;     // read-back of results beside the sites that follow
+  std::vector<cudaEvent_t> done_ev;       // [n_sites] recorded behind a site whose result is read back
 };
 
 namespace {
@@ -41,8 +43,9 @@ bool capturing(cudaStream_t s) {
   return st != cudaStreamCaptureStatusNone;
 }
 
+// after: optional, one event per site (or null): recorded on the stream behind that site's launch.
 int run_sites(edgelora_siteset *s, const void *const *x_dev, const int32_t *ids_dev, int32_t T,
-              void *const *y_dev, cudaStream_t stream) {
+              void *const *y_dev, cudaStream_t stream, const std::vector<cudaEvent_t> *after = nullptr) {
   int rc = edgelora_plan_build(s->plan, ids_dev, T, stream);
   if (rc != EDGELORA_OK) return rc;
   const int n = static_cast<int>(s->pools.size());
@@ -61,6 +64,7 @@ int run_sites(edgelora_siteset *s, const void *const *x_dev, const int32_t *ids_
     rc = lora_linear_impl(s->pools[i], s->plan, nullptr, s->W[i], x_dev[s->input_of[i]], T, y_dev[i], stream,
                           pipelined && i > 0, next.pool ? &next : nullptr, !pipelined && i > 0);
     if (rc != EDGELORA_OK) return rc;
+    if (after && (*after)[i] && cudaEventRecord((*after)[i], stream) != cudaSuccess) return EDGELORA_ERR_CUDA;
   }
   if (pipelined && !capturing(stream)) {  // slot loads issued later wait for this step
     for (auto *p : s->pools) {
@@ -122,6 +126,8 @@ int edgelora_siteset_destroy(edgelora_siteset_t *s) {
   for (auto *q : s->dy) if (q) el_free(q);
   for (auto &e : s->dy_scratch) if (e.second) el_free(e.second);
   if (s->dids) el_free(s->dids);
+  for (auto e : s->done_ev) if (e) cudaEventDestroy(e);
+  if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
   cudaGetLastError();
   delete s;
   return EDGELORA_OK;
@@ -195,13 +201,26 @@ int edgelora_siteset_run_host(edgelora_siteset_t *s, const uint16_t *const *x_ho
                               cudaMemcpyHostToDevice, st));
   SET_TRY(cudaMemcpyAsync(s->dids, adapter_id_host, static_cast<size_t>(T) * 4, cudaMemcpyHostToDevice, st));
   std::vector<const void *> xd(s->dx.begin(), s->dx.end());
-  int rc = run_sites(s, xd.data(), s->dids, T, y_dev.data(), st);
+  // A result goes back to the host on a second stream as soon as its site is done, beside the sites
+  // that follow (an event behind a launch keeps the next launch from starting under it, which is
+  // paid only for the sites that are read back).
+  if (!s->copy_stream) SET_TRY(cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking));
+  if (s->done_ev.empty()) s->done_ev.assign(n, nullptr);
+  for (int i = 0; i < n; ++i)
+    if (y_host[i] && !s->done_ev[i]) SET_TRY(cudaEventCreateWithFlags(&s->done_ev[i], cudaEventDisableTiming));
+  std::vector<cudaEvent_t> after(n, nullptr);
+  for (int i = 0; i < n; ++i)
+    if (y_host[i]) after[i] = s->done_ev[i];
+  int rc = run_sites(s, xd.data(), s->dids, T, y_dev.data(), st, &after);
   if (rc != EDGELORA_OK) return rc;
   for (int i = 0; i < n; ++i)
-    if (y_host[i])
+    if (y_host[i]) {
+      SET_TRY(cudaStreamWaitEvent(s->copy_stream, s->done_ev[i], 0));
       SET_TRY(cudaMemcpyAsync(y_host[i], s->dy[i], static_cast<size_t>(T) * s->pools[i]->cfg.h_out * 2,
-                              cudaMemcpyDeviceToHost, st));
+                              cudaMemcpyDeviceToHost, s->copy_stream));
+    }
   SET_TRY(cudaStreamSynchronize(st));
+  SET_TRY(cudaStreamSynchronize(s->copy_stream));
 #undef SET_TRY
   return EDGELORA_OK;
 }
