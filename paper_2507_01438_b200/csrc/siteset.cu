@@ -30,6 +30,7 @@ struct edgelora_siteset {
   std::vector<std::pair<int32_t, uint16_t *>> dy_scratch;  // (h_out, buffer) for the others
   cudaStream_t copy_stream = nullptr;     // read-back of results beside the sites that follow
   std::vector<cudaEvent_t> done_ev;       // [n_sites] recorded behind a site whose result is read back
+  std::vector<cudaEvent_t> up_ev;         // [n_inputs] an input uploaded on the second stream has arrived
 };
 
 namespace {
@@ -44,8 +45,10 @@ bool capturing(cudaStream_t s) {
 }
 
 // after: optional, one event per site (or null): recorded on the stream behind that site's launch.
+// before: optional, one event per site (or null): the stream waits for it in front of that site's launch.
 int run_sites(edgelora_siteset *s, const void *const *x_dev, const int32_t *ids_dev, int32_t T,
-              void *const *y_dev, cudaStream_t stream, const std::vector<cudaEvent_t> *after = nullptr) {
+              void *const *y_dev, cudaStream_t stream, const std::vector<cudaEvent_t> *after = nullptr,
+              const std::vector<cudaEvent_t> *before = nullptr) {
   int rc = edgelora_plan_build(s->plan, ids_dev, T, stream);
   if (rc != EDGELORA_OK) return rc;
   const int n = static_cast<int>(s->pools.size());
@@ -59,6 +62,7 @@ int run_sites(edgelora_siteset *s, const void *const *x_dev, const int32_t *ids_
       next.pool = s->pools[i + 1];
       next.x = static_cast<const uint16_t *>(x_dev[s->input_of[i + 1]]);
     }
+    if (before && (*before)[i] && cudaStreamWaitEvent(stream, (*before)[i], 0) != cudaSuccess) return EDGELORA_ERR_CUDA;
     // (decode-sized batches: the sites are independent given their inputs and results, so a
     // site's shrink may start under the previous site's base product)
     rc = lora_linear_impl(s->pools[i], s->plan, nullptr, s->W[i], x_dev[s->input_of[i]], T, y_dev[i], stream,
@@ -127,6 +131,7 @@ int edgelora_siteset_destroy(edgelora_siteset_t *s) {
   for (auto &e : s->dy_scratch) if (e.second) el_free(e.second);
   if (s->dids) el_free(s->dids);
   for (auto e : s->done_ev) if (e) cudaEventDestroy(e);
+  for (auto e : s->up_ev) if (e) cudaEventDestroy(e);
   if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
   cudaGetLastError();
   delete s;
@@ -195,23 +200,43 @@ int edgelora_siteset_run_host(edgelora_siteset_t *s, const uint16_t *const *x_ho
       y_dev[i] = buf;
     }
   }
-  for (int i = 0; i < s->n_inputs; ++i)
-    if (s->in_width[i])
-      SET_TRY(cudaMemcpyAsync(s->dx[i], x_host[i], static_cast<size_t>(T) * s->in_width[i] * 2,
-                              cudaMemcpyHostToDevice, st));
+  // An input that the first launches do not need is uploaded on the second stream, beside them; the
+  // launch in front of its first consumer waits for it (a launch also carries the next site's shrink,
+  // hence one launch earlier).
+  if (!s->copy_stream) SET_TRY(cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking));
+  if (s->up_ev.empty()) s->up_ev.assign(s->n_inputs, nullptr);
+  std::vector<cudaEvent_t> before(n, nullptr);
   SET_TRY(cudaMemcpyAsync(s->dids, adapter_id_host, static_cast<size_t>(T) * 4, cudaMemcpyHostToDevice, st));
+  for (int i = 0; i < s->n_inputs; ++i) {
+    if (!s->in_width[i]) continue;
+    int first = n;
+    for (int k = 0; k < n; ++k)
+      if (s->input_of[k] == i) {
+        first = k;
+        break;
+      }
+    const int at = first - 1;  // the launch that may already read it
+    const size_t bytes = static_cast<size_t>(T) * s->in_width[i] * 2;
+    if (at <= 0 || first >= n || before[at]) {
+      SET_TRY(cudaMemcpyAsync(s->dx[i], x_host[i], bytes, cudaMemcpyHostToDevice, st));
+    } else {
+      if (!s->up_ev[i]) SET_TRY(cudaEventCreateWithFlags(&s->up_ev[i], cudaEventDisableTiming));
+      SET_TRY(cudaMemcpyAsync(s->dx[i], x_host[i], bytes, cudaMemcpyHostToDevice, s->copy_stream));
+      SET_TRY(cudaEventRecord(s->up_ev[i], s->copy_stream));
+      before[at] = s->up_ev[i];
+    }
+  }
   std::vector<const void *> xd(s->dx.begin(), s->dx.end());
   // A result goes back to the host on a second stream as soon as its site is done, beside the sites
   // that follow (an event behind a launch keeps the next launch from starting under it, which is
   // paid only for the sites that are read back).
-  if (!s->copy_stream) SET_TRY(cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking));
   if (s->done_ev.empty()) s->done_ev.assign(n, nullptr);
   for (int i = 0; i < n; ++i)
     if (y_host[i] && !s->done_ev[i]) SET_TRY(cudaEventCreateWithFlags(&s->done_ev[i], cudaEventDisableTiming));
   std::vector<cudaEvent_t> after(n, nullptr);
   for (int i = 0; i < n; ++i)
     if (y_host[i]) after[i] = s->done_ev[i];
-  int rc = run_sites(s, xd.data(), s->dids, T, y_dev.data(), st, &after);
+  int rc = run_sites(s, xd.data(), s->dids, T, y_dev.data(), st, &after, &before);
   if (rc != EDGELORA_OK) return rc;
   for (int i = 0; i < n; ++i)
     if (y_host[i]) {
