@@ -253,7 +253,9 @@ int edgelora_siteset_run(edgelora_siteset_t *set, const void *const *x_dev, cons
 /* The same with HOST buffers (page-locked for full copy speed): copies the inputs and the ids to
  * the device, runs the set, copies back y of every site whose y_host entry is not NULL (the others
  * stay on the device and are overwritten by the next site of the same width) and synchronises
- * `stream` before returning.  Allocates its device mirrors on first use. */
+ * `stream` before returning.  Allocates its device mirrors on first use.  Copies that the running
+ * sites do not wait for (a result that is complete, an input that only later sites read) go through
+ * a second stream of the set's own, beside the kernels; that stream is synchronised too. */
 int edgelora_siteset_run_host(edgelora_siteset_t *set, const uint16_t *const *x_host,
                               const int32_t *adapter_id_host, int32_t T, uint16_t *const *y_host,
                               void *stream);
