@@ -138,3 +138,36 @@ def test_one_set_run_three_times_gives_the_same_bits():
         B.edgelora_siteset_destroy(s)
         for p in pools:
             p.close()
+
+
+def test_host_buffer_call_twice_on_one_set():
+    # the set's second stream, its events and its device mirrors are reused by the second call, which
+    # has other inputs and another batch size: both calls must match the oracle
+    import torch
+    ranks = [16, 8, 16]
+    shapes = [(256, 264), (512, 128), (256, 520)]
+    pin = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a).view(dt)).pin_memory()
+    ids1 = mixed_ids(31, 30, [(1, 280)], len(ranks))
+    ids2 = mixed_ids(32, 12, [(0, 150), (2, 200)], len(ranks))
+    xs1, sites1 = make_sites(41, len(ids1), shapes, ranks, 16, ids1)
+    rng = np.random.Generator(np.random.PCG64(43))
+    xs2 = {h: wl.normal_bf16(rng, (len(ids2), h), 1.0) for h in xs1}       # the same W and adapters, other inputs
+    sites2 = [wl.Workload(w.name, w.h_in, w.h_out, w.n_slots, w.max_rank, w.W, xs2[w.h_in], ids2, w.adapters)
+              for w in sites1]
+    widths = sorted(xs1)
+    pools = [make_pool(w, 512) for w in sites1]
+    Ws = [to_dev_bf16(w.W) for w in sites1]
+    s = B.edgelora_siteset_create([p.handle for p in pools], Ws, [widths.index(w.h_in) for w in sites1],
+                                  len(widths), 512)
+    try:
+        for xs, ids, sites in ((xs1, ids1, sites1), (xs2, ids2, sites2)):
+            ys = [torch.zeros((len(ids), w.h_out), dtype=torch.int16).pin_memory() for w in sites]
+            B.edgelora_siteset_run_host(s, [pin(xs[h], np.int16) for h in widths], pin(ids, np.int32), ys)
+            for p in pools:
+                assert p.status() == (0, 0)
+            for w, y in zip(sites, ys):
+                assert_parity(wl.bf16_bits_to_f32(y.numpy().view(np.uint16)), oracle_of(w), w.name)
+    finally:
+        B.edgelora_siteset_destroy(s)
+        for p in pools:
+            p.close()
