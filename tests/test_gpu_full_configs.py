@@ -130,3 +130,26 @@ def test_full_projection_set_sampled_sites():
                 pool.close()
     finally:
         B.edgelora_plan_destroy(plan)
+
+
+def test_largest_batch_a_pool_takes():
+    # T = 32768 (the limit of max_tokens), small widths so that the oracle covers every element:
+    # 256 token tiles, long runs (segment tiles), short runs and scattered tokens (gather tiles), a
+    # ragged last row tile, ragged ranks
+    from test_gpu_parity import random_workload
+    from gpu_helpers import run_gpu
+    T = 32768
+    base = random_workload(9900, 64, 136, 200, ranks=[16, 8, 3, 16, 12, 5, 16, 1], max_rank=16)
+    rng = np.random.Generator(np.random.PCG64(9901))
+    parts, left = [], T
+    while left > 0:
+        n = int(min(left, rng.choice([1, 2, 5, 17, 40, 130, 700, 3000])))
+        parts.append(np.full(n, rng.integers(-1, 8)))
+        left -= n
+    ids = np.concatenate(parts).astype(np.int32)
+    x = wl.normal_bf16(rng, (T, base.h_in), 1.0)
+    w = wl.Workload("max_T", base.h_in, base.h_out, base.n_slots, base.max_rank, base.W, x, ids, base.adapters)
+    y, plan = run_gpu(w, 0, return_plan=True)
+    assert_parity(y, oracle_of(w), "T = 32768")
+    from test_gpu_parity import check_plan
+    check_plan(plan, ids, w.n_slots)
