@@ -153,3 +153,24 @@ def test_largest_batch_a_pool_takes():
     assert_parity(y, oracle_of(w), "T = 32768")
     from test_gpu_parity import check_plan
     check_plan(plan, ids, w.n_slots)
+
+
+@pytest.mark.parametrize("T", [40, 300])
+def test_largest_pool_and_smallest_widths(T):
+    # 65534 slots (the limit), adapters in the first, a middle and the last slot; and the smallest widths
+    # the library takes (8 -> 8), where every operand tile is mostly zero fill
+    from gpu_helpers import run_gpu
+    rng = np.random.Generator(np.random.PCG64(9950 + T))
+    S, h_in, h_out = 65534, 64, 72
+    slots = [0, 1, 32767, 65533]
+    ad = {a: wl.Adapter(wl.normal_bf16(rng, (r, h_in), 0.05), wl.normal_bf16(rng, (h_out, r), 0.05), 1.0)
+          for a, r in zip(slots, [16, 5, 12, 16])}
+    ids = rng.choice(np.array([-1] + slots), size=T).astype(np.int32)
+    w = wl.Workload("max_slots", h_in, h_out, S, 16, wl.normal_bf16(rng, (h_out, h_in), 0.05),
+                    wl.normal_bf16(rng, (T, h_in), 1.0), ids, ad)
+    assert_parity(run_gpu(w, 0), oracle_of(w), f"65534 slots, T = {T}")
+    tiny = {0: wl.Adapter(wl.normal_bf16(rng, (8, 8), 0.3), wl.normal_bf16(rng, (8, 8), 0.3), 2.0),
+            1: wl.Adapter(wl.normal_bf16(rng, (3, 8), 0.3), wl.normal_bf16(rng, (8, 3), 0.3), 0.5)}
+    w8 = wl.Workload("min_widths", 8, 8, 2, 8, wl.normal_bf16(rng, (8, 8), 0.3), wl.normal_bf16(rng, (T, 8), 1.0),
+                     rng.integers(-1, 2, size=T).astype(np.int32), tiny)
+    assert_parity(run_gpu(w8, 0), oracle_of(w8), f"8 -> 8, T = {T}")
